@@ -1,0 +1,100 @@
+"""Seeded synthetic inputs and the benchmark shapes.
+
+Holds no arithmetic of the method: only shapes, random weights / prompts / logits and
+dtype plumbing.  Both the CUDA library's harness and the CPU oracle's tests take their
+inputs from here so that they see identical buffers.
+
+The paper measured on CNN-DM / XSUM prompts with pretrained LayerSkip and Gemma2
+checkpoints; neither is available offline, so random-init models of the configured shapes
+and uniform-random prompts stand in for them.
+"""
+import numpy as np
+import torch
+
+LAYER_KEYS = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "wg", "wu", "wd")
+
+
+def model_cfg(n_layers, d_model, n_q_heads, n_kv_heads, d_ff, vocab, dtype, head_dim=None):
+    return dict(n_layers=n_layers, d_model=d_model, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads,
+                head_dim=head_dim or d_model // n_q_heads, d_ff=d_ff, vocab=vocab, dtype=dtype,
+                rms_eps=1e-5, rope_theta=10000.0)
+
+
+# The five workloads of the benchmark contract (model, exits, T, batch, prompt, n_new, page).
+WORKLOADS = {
+    "tiny3": dict(model=model_cfg(4, 128, 4, 4, 512, 512, "fp32"), exits=(1, 2, 4), T=(3, 2),
+                  batch=1, prompt=16, n_new=64, page=16, weight_seed=1, prompt_seed=1),
+    "accept": dict(batch=64, t=8, vocab=32000, dtype="bf16", target_std=3.0, noise_std=1.0),
+    "1b3": dict(model=model_cfg(16, 2048, 32, 8, 5632, 32000, "bf16"), exits=(4, 8, 16), T=(4, 2),
+                batch=1, prompt=512, n_new=256, page=16, weight_seed=3, prompt_seed=3),
+    "8b3": dict(model=model_cfg(32, 4096, 32, 8, 14336, 32000, "bf16"), exits=(4, 12, 32), T=None,
+                batch=1, prompt=1024, n_new=256, page=16, weight_seed=4, prompt_seed=4),
+    "8b4long": dict(model=model_cfg(32, 4096, 32, 8, 14336, 32000, "bf16"), exits=(2, 6, 16, 32),
+                    T=(2, 2, 3), batch=16, prompt=8192, n_new=512, page=16, weight_seed=4,
+                    prompt_seed=5),
+    # small bf16 stand-in with the 8B-shape's structure (GQA, SwiGLU, 3 levels) that the
+    # CPU oracle finishes in seconds; spans several GEMM tiles and ragged tails.
+    "mini3": dict(model=model_cfg(6, 256, 8, 2, 704, 2048, "bf16", head_dim=32), exits=(1, 3, 6),
+                  T=(3, 2), batch=1, prompt=24, n_new=48, page=16, weight_seed=7, prompt_seed=7),
+}
+
+
+def _gen(seed, device):
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return g
+
+
+def make_weights(cfg, seed, device="cpu", std=0.02):
+    """Matrices N(0, std^2) stored [out_features, in_features]; norm gains 1.  torch tensors in
+    the model's storage dtype on ``device``."""
+    dt = torch.float32 if cfg["dtype"] == "fp32" else torch.bfloat16
+    g = _gen(seed, device)
+    d, hd, ff, V = cfg["d_model"], cfg["head_dim"], cfg["d_ff"], cfg["vocab"]
+    nq, nkv = cfg["n_q_heads"], cfg["n_kv_heads"]
+
+    def mat(rows, cols):
+        return (torch.randn(rows, cols, generator=g, device=device, dtype=torch.float32) * std).to(dt)
+
+    def ones(n):
+        return torch.ones(n, device=device, dtype=dt)
+
+    w = dict(embed=mat(V, d), final_norm=ones(d), lm_head=mat(V, d), layers=[])
+    for _ in range(cfg["n_layers"]):
+        w["layers"].append(dict(attn_norm=ones(d), wq=mat(nq * hd, d), wk=mat(nkv * hd, d),
+                                wv=mat(nkv * hd, d), wo=mat(d, nq * hd), mlp_norm=ones(d),
+                                wg=mat(ff, d), wu=mat(ff, d), wd=mat(d, ff)))
+    return w
+
+
+def weights_to_numpy(w):
+    """fp32 tensors -> float32 arrays; bf16 tensors -> uint16 bit patterns (host copies)."""
+    def conv(t):
+        t = t.detach().cpu().contiguous()
+        return t.view(torch.uint16).numpy() if t.dtype == torch.bfloat16 else t.numpy()
+    out = {k: conv(v) for k, v in w.items() if k != "layers"}
+    out["layers"] = [{k: conv(v) for k, v in layer.items()} for layer in w["layers"]]
+    return out
+
+
+def make_prompts(vocab, batch, length, seed):
+    """Uniform-random token ids, int32 [batch, length] on the CPU."""
+    g = _gen(seed, "cpu")
+    return torch.randint(0, vocab, (batch, length), generator=g, dtype=torch.int32)
+
+
+def make_accept_logits(batch, t, vocab, seed, device="cpu", target_std=3.0, noise_std=1.0,
+                       dtype="bf16"):
+    """Target logits [batch, t+1, vocab] ~ N(0, target_std^2); draft logits [batch, t, vocab] =
+    the first t target rows (before rounding) + N(0, noise_std^2); both rounded to ``dtype``."""
+    g = _gen(seed, device)
+    dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    tgt = torch.randn(batch, t + 1, vocab, generator=g, device=device, dtype=torch.float32) * target_std
+    drf = tgt[:, :t, :] + torch.randn(batch, t, vocab, generator=g, device=device,
+                                      dtype=torch.float32) * noise_std
+    return tgt.to(dt).contiguous(), drf.to(dt).contiguous()
+
+
+def logits_to_numpy(x):
+    """Stored logits -> float32 numpy (bf16 widens exactly)."""
+    return x.detach().cpu().to(torch.float32).numpy()
