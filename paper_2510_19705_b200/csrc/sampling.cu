@@ -1,0 +1,226 @@
+// Sampling kernels of the HSD hot path: level-0 draft sampling (Algorithm 1, base case) and the
+// fused softmax-statistics / acceptance / residual-resample step (Algorithm 2; rule of Section 2).
+#include "sampling.cuh"
+#include "sampling_api.cuh"
+
+namespace hsd {
+
+// ------------------------------------------------------------------------------ draft sampling
+// One block per row: token = inverse-CDF sample of softmax(row) with the purpose-0 uniform.
+template <typename T>
+__global__ void __launch_bounds__(kSampleThreads)
+draft_sample_kernel(const T *__restrict__ logits, int V, const SampleRow *__restrict__ desc,
+                    int regular_rows, u32 regular_serial, u64 seed, int32_t *__restrict__ out) {
+  __shared__ float shf[32];
+  __shared__ u64 sh64[34];
+  SampleRow d;
+  if (desc) {
+    d = desc[blockIdx.x];
+  } else {
+    d.logit_row = blockIdx.x;
+    d.out_index = blockIdx.x;
+    d.j = blockIdx.x % regular_rows;
+    d.seq = blockIdx.x / regular_rows;
+    d.serial = regular_serial;
+    d.level = 0;
+  }
+  const T *row = logits + (size_t)d.logit_row * V;
+  float m = row_max(row, V, shf);
+  u32 U = uniform24(seed, d.j, d.serial, d.level, PURPOSE_DRAFT, d.seq);
+  int tok = block_inverse_cdf(V, U, [&](int k) { return (u64)exp_weight(to_f32(row[k]), m); }, sh64, nullptr);
+  if (threadIdx.x == 0) out[d.out_index] = tok;
+}
+
+// ------------------------------------------------------------------------------ row statistics
+// grid (2 * t_max + 1, batch).  Block (r, b): r <= t_max -> target row r; else draft row
+// r - t_max - 1.  Writes the row maximum, the integer total S and the weight of the drafted token.
+template <typename T>
+__global__ void __launch_bounds__(kStatThreads)
+row_stats_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, const int32_t *__restrict__ tokens,
+                 int V, int t_max, const VerifySeq *__restrict__ desc, int regular_t, RowStat *__restrict__ stats) {
+  __shared__ float shf[32];
+  __shared__ u64 sh64[33];
+  int b = blockIdx.y, r = blockIdx.x;
+  VerifySeq d;
+  if (desc) d = desc[b];
+  else { d.t = regular_t; d.p_row0 = (long long)b * (regular_t + 1); d.q_row0 = (long long)b * regular_t; d.tok_off = (long long)b * regular_t; }
+  const T *row;
+  int tok = -1;
+  if (r <= t_max) {
+    if (r > d.t) return;
+    row = p_logits + (size_t)(d.p_row0 + r) * V;
+    if (r < d.t) tok = tokens[d.tok_off + r];
+  } else {
+    int j = r - t_max - 1;
+    if (j >= d.t) return;
+    row = q_logits + (size_t)(d.q_row0 + j) * V;
+    tok = tokens[d.tok_off + j];
+  }
+  float m = row_max(row, V, shf);
+  u64 local = 0;
+  for (int k = threadIdx.x; k < V; k += blockDim.x) local += exp_weight(to_f32(row[k]), m);
+  u64 total;
+  block_exclusive_scan(local, sh64, &total);
+  if (threadIdx.x == 0) {
+    RowStat s;
+    s.m = m;
+    s.S = total;
+    s.Ex = (tok >= 0 && tok < V) ? exp_weight(to_f32(row[tok]), m) : 0u;
+    stats[(size_t)b * (2 * t_max + 1) + r] = s;
+  }
+}
+
+// ------------------------------------------------------------------------------ decision
+// One block per sequence: accept tests for all positions (each with its own counter-addressed
+// uniform, so the parallel form equals Algorithm 2's sequential loop with break), n = index of the
+// first rejection, then the final draw from the residual of row n (n < t) or from target row t.
+template <typename T>
+__global__ void __launch_bounds__(kSampleThreads)
+decide_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, int32_t *__restrict__ tokens, int V,
+              int t_max, const VerifySeq *__restrict__ desc, int regular_t, u32 regular_serial, u32 regular_level,
+              const RowStat *__restrict__ stats, u64 seed, int32_t *__restrict__ out_tokens /*[B, t_max+1] or null*/,
+              int32_t *__restrict__ out_n /*[B]*/, int write_in_place) {
+  __shared__ u64 sh64[34];
+  __shared__ int sh_first_reject;
+  int b = blockIdx.x;
+  VerifySeq d;
+  if (desc) d = desc[b];
+  else {
+    d.t = regular_t; d.p_row0 = (long long)b * (regular_t + 1); d.q_row0 = (long long)b * regular_t;
+    d.tok_off = (long long)b * regular_t; d.serial = regular_serial; d.seq = b; d.level = regular_level;
+  }
+  const RowStat *st = stats + (size_t)b * (2 * t_max + 1);
+  if (threadIdx.x == 0) sh_first_reject = d.t;
+  __syncthreads();
+  if ((int)threadIdx.x < d.t) {
+    int j = threadIdx.x;
+    RowStat sp = st[j], sq = st[t_max + 1 + j];
+    u64 Pp = fixed_prob(sp.Ex, prob_scale(sp.S));
+    u64 Pq = fixed_prob(sq.Ex, prob_scale(sq.S));
+    u32 U = uniform24(seed, j, d.serial, d.level, PURPOSE_ACCEPT, d.seq);
+    bool ok = (((u64)U * Pq) >> 24) < Pp;                 // u < p(x) / q(x)
+    if (!ok) atomicMin(&sh_first_reject, j);
+  }
+  __syncthreads();
+  int n = sh_first_reject;
+  u32 U = uniform24(seed, 0, d.serial, d.level, PURPOSE_FINAL, d.seq);
+  const T *prow = p_logits + (size_t)(d.p_row0 + n) * V;
+  float mp = st[n].m;
+  int m_tok = -1;
+  if (n < d.t) {
+    const T *qrow = q_logits + (size_t)(d.q_row0 + n) * V;
+    float mq = st[t_max + 1 + n].m;
+    ProbScale psp = prob_scale(st[n].S), psq = prob_scale(st[t_max + 1 + n].S);
+    m_tok = block_inverse_cdf(V, U, [&](int k) {
+      u64 Pp = fixed_prob(exp_weight(to_f32(prow[k]), mp), psp);
+      u64 Pq = fixed_prob(exp_weight(to_f32(qrow[k]), mq), psq);
+      return Pp > Pq ? Pp - Pq : 0ull;
+    }, sh64, nullptr);
+  }
+  if (m_tok < 0)   // bonus token, or an all-zero residual: draw from the verifier's own row
+    m_tok = block_inverse_cdf(V, U, [&](int k) { return (u64)exp_weight(to_f32(prow[k]), mp); }, sh64, nullptr);
+  if (threadIdx.x == 0) {
+    out_n[b] = n;
+    if (write_in_place) tokens[d.tok_off + n] = m_tok;
+  }
+  if (out_tokens) {
+    for (int j = threadIdx.x; j <= t_max; j += blockDim.x) {
+      int v = -1;
+      if (j < n) v = tokens[d.tok_off + j];
+      else if (j == n) v = m_tok;
+      out_tokens[(size_t)b * (t_max + 1) + j] = v;
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------ host launchers
+size_t verify_scratch_bytes(int batch, int t_max) { return (size_t)batch * (2 * t_max + 1) * sizeof(RowStat); }
+
+template <typename T>
+static int launch_draft_sample_t(const void *logits, int V, const SampleRow *desc, int n_rows, int regular_rows,
+                                 u32 regular_serial, u64 seed, int32_t *out, cudaStream_t s) {
+  draft_sample_kernel<T><<<n_rows, kSampleThreads, 0, s>>>((const T *)logits, V, desc, regular_rows, regular_serial, seed, out);
+  return hsd_launch_status();
+}
+
+int launch_draft_sample(const void *logits, int dtype, int V, const SampleRow *desc, int n_rows, int regular_rows,
+                        u32 regular_serial, u64 seed, int32_t *out, cudaStream_t s) {
+  if (n_rows == 0) return HSD_OK;
+  return dtype == HSD_BF16
+             ? launch_draft_sample_t<__nv_bfloat16>(logits, V, desc, n_rows, regular_rows, regular_serial, seed, out, s)
+             : launch_draft_sample_t<float>(logits, V, desc, n_rows, regular_rows, regular_serial, seed, out, s);
+}
+
+template <typename T>
+static int launch_verify_t(const void *p, const void *q, int32_t *tokens, int V, int batch, int t_max,
+                           const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch,
+                           u64 seed, int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s) {
+  RowStat *stats = (RowStat *)scratch;
+  dim3 grid(2 * t_max + 1, batch);
+  row_stats_kernel<T><<<grid, kStatThreads, 0, s>>>((const T *)p, (const T *)q, tokens, V, t_max, desc, regular_t, stats);
+  if (cudaGetLastError() != cudaSuccess) return HSD_E_CUDA;
+  decide_kernel<T><<<batch, kSampleThreads, 0, s>>>((const T *)p, (const T *)q, tokens, V, t_max, desc, regular_t,
+                                                   regular_serial, regular_level, stats, seed, out_tokens, out_n,
+                                                   write_in_place);
+  return hsd_launch_status();
+}
+
+int launch_verify(const void *p, const void *q, int32_t *tokens, int dtype, int V, int batch, int t_max,
+                  const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch, u64 seed,
+                  int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s) {
+  if (batch == 0) return HSD_OK;
+  return dtype == HSD_BF16 ? launch_verify_t<__nv_bfloat16>(p, q, tokens, V, batch, t_max, desc, regular_t, regular_serial,
+                                                            regular_level, scratch, seed, out_tokens, out_n, write_in_place, s)
+                           : launch_verify_t<float>(p, q, tokens, V, batch, t_max, desc, regular_t, regular_serial,
+                                                    regular_level, scratch, seed, out_tokens, out_n, write_in_place, s);
+}
+
+}  // namespace hsd
+
+// ------------------------------------------------------------------------------ C ABI
+extern "C" {
+
+const char *hsd_strerror(int status) {
+  switch (status) {
+    case HSD_OK: return "ok";
+    case HSD_E_INVALID_ARG: return "invalid argument";
+    case HSD_E_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case HSD_E_OUT_OF_PAGES: return "out of KV pages";
+    case HSD_E_CUDA: return "CUDA error";
+    case HSD_E_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case HSD_E_UNSUPPORTED: return "unsupported configuration";
+    case HSD_E_IO: return "I/O error";
+    default: return "unknown status";
+  }
+}
+
+int hsd_draft_sample(const void *logits, int batch, int rows, int vocab, int dtype, uint64_t seed,
+                     uint64_t call_serial, void *stream, int32_t *out_tokens) {
+  if (!logits || !out_tokens || batch <= 0 || rows <= 0 || vocab <= 0) return HSD_E_INVALID_ARG;
+  if (dtype != HSD_F32 && dtype != HSD_BF16) return HSD_E_INVALID_ARG;
+  if ((long long)batch * rows > 0x7FFFFFFFll) return HSD_E_INVALID_ARG;
+  return hsd::launch_draft_sample(logits, dtype, vocab, nullptr, batch * rows, rows, (u32)call_serial, seed, out_tokens,
+                                  (cudaStream_t)stream);
+}
+
+size_t hsd_verify_workspace_bytes(int batch, int t) {
+  if (batch <= 0 || t < 0) return 0;
+  return hsd::verify_scratch_bytes(batch, t);
+}
+
+int hsd_verify_level(int level, const void *target_logits, const void *draft_logits, const int32_t *draft_tokens,
+                     int batch, int t, int vocab, int dtype, uint64_t seed, uint64_t call_serial, void *workspace,
+                     size_t workspace_bytes, void *stream, int32_t *out_tokens, int32_t *out_n_accepted) {
+  if (!target_logits || !out_tokens || !out_n_accepted || !workspace) return HSD_E_INVALID_ARG;
+  if (batch <= 0 || t < 0 || vocab <= 0 || level < 0 || level > 255) return HSD_E_INVALID_ARG;
+  if (t > 0 && (!draft_logits || !draft_tokens)) return HSD_E_INVALID_ARG;
+  if (t >= hsd::kSampleThreads || batch > 65535) return HSD_E_INVALID_ARG;
+  if (dtype != HSD_F32 && dtype != HSD_BF16) return HSD_E_INVALID_ARG;
+  if (((uintptr_t)workspace & 15) != 0) return HSD_E_INVALID_ARG;
+  if (workspace_bytes < hsd::verify_scratch_bytes(batch, t)) return HSD_E_WORKSPACE_TOO_SMALL;
+  return hsd::launch_verify(target_logits, draft_logits, const_cast<int32_t *>(draft_tokens), dtype, vocab, batch, t,
+                            nullptr, t, (u32)call_serial, (u32)level, workspace, seed, out_tokens, out_n_accepted, 0,
+                            (cudaStream_t)stream);
+}
+
+}  // extern "C"

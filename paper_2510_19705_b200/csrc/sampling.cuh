@@ -1,0 +1,143 @@
+// Device-side decision arithmetic of the speculative-sampling rule (Section 2, Algorithm 2):
+// Philox4x32-10 uniforms, integer softmax numerators, fixed-point probabilities, block-wide
+// inverse CDF.  Everything that decides an integer is integer arithmetic on values produced by a
+// fixed sequence of IEEE fp32 operations, so the outcome does not depend on thread count or
+// summation order.
+#pragma once
+#include "common.cuh"
+
+namespace hsd {
+
+enum { PURPOSE_DRAFT = 0, PURPOSE_ACCEPT = 1, PURPOSE_FINAL = 2 };
+
+// ---- Philox4x32-10 (Salmon et al., SC'11): 10 rounds, key bumped by the Weyl constants.
+__device__ __forceinline__ u32 philox_word0(u32 c0, u32 c1, u32 c2, u32 c3, u32 k0, u32 k1) {
+  const u32 M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    if (r > 0) { k0 += W0; k1 += W1; }
+    u32 hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    u32 hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    u32 n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+  }
+  return c0;
+}
+
+// 24-bit integer uniform of the decision addressed (j, serial, level, purpose, seq).
+__device__ __forceinline__ u32 uniform24(u64 seed, u32 j, u32 serial, u32 level, u32 purpose, u32 seq) {
+  return philox_word0(j, serial, (level & 0xFFu) | (purpose << 8), seq, (u32)seed, (u32)(seed >> 32)) >> 8;
+}
+
+// ---- E = min(floor(exp(l - m) * 2^32), 2^32 - 1): every step is one fp32 operation, never fused.
+__device__ __forceinline__ u32 exp_weight(float l, float m) {
+  float x = __fsub_rn(l, m);
+  x = fmaxf(x, -32.0f);
+  float t = __fmul_rn(x, __uint_as_float(0x3FB8AA3Bu));     // * log2(e)
+  float j = rintf(t);                                      // half to even
+  float f = __fsub_rn(t, j);                               // exact, in [-1/2, 1/2]
+  float p = __uint_as_float(0x3AADDD0Au);
+  p = __fadd_rn(__fmul_rn(p, f), __uint_as_float(0x3C1E7544u));
+  p = __fadd_rn(__fmul_rn(p, f), __uint_as_float(0x3D635BA9u));
+  p = __fadd_rn(__fmul_rn(p, f), __uint_as_float(0x3E75FCDEu));
+  p = __fadd_rn(__fmul_rn(p, f), __uint_as_float(0x3F317215u));
+  p = __fadd_rn(__fmul_rn(p, f), 1.0f);
+  int e = (int)j + 32;                                     // in [-14, 32]
+  float w = __fmul_rn(p, __int_as_float((e + 127) << 23)); // exact power-of-two scaling
+  return __float2uint_rz(w);                               // floor; saturates at 2^32 - 1
+}
+
+// Fixed-point probabilities in units of 2^-40: P = (E * rinv) >> shift.
+struct ProbScale { u32 rinv; int shift; };
+__device__ __forceinline__ ProbScale prob_scale(u64 S) {
+  ProbScale ps;
+  int z = __clzll((long long)S);
+  u64 s_top = (S << z) >> 32;                              // in [2^31, 2^32)
+  ps.rinv = (u32)(0x7FFFFFFFFFFFFFFFull / s_top);
+  ps.shift = 55 - z;
+  return ps;
+}
+__device__ __forceinline__ u64 fixed_prob(u32 E, ProbScale ps) { return ((u64)E * ps.rinv) >> ps.shift; }
+
+// (U * total) >> 24 without overflow (U < 2^24, total < 2^64).
+__device__ __forceinline__ u64 cdf_threshold(u32 U, u64 total) {
+  return (u64)U * (total >> 24) + (((u64)U * (total & 0xFFFFFFull)) >> 24);
+}
+
+// ---- block-wide reductions (blockDim.x a multiple of 32, at most 1024)
+__device__ __forceinline__ float block_max(float v, float *sh /*[32]*/) {
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+  __syncthreads();
+  if (l == 0) sh[w] = v;
+  __syncthreads();
+  float r = (l < nw) ? sh[l] : -INFINITY;
+  for (int o = 16; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xFFFFFFFFu, r, o));
+  return r;
+}
+
+// Exclusive prefix sum of one u64 per thread in thread order; *total receives the block sum.
+__device__ __forceinline__ u64 block_exclusive_scan(u64 v, u64 *sh /*[33]*/, u64 *total) {
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+  u64 inc = v;
+  for (int o = 1; o < 32; o <<= 1) {
+    u64 n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+    if (l >= o) inc += n;
+  }
+  __syncthreads();
+  if (l == 31) sh[w] = inc;
+  __syncthreads();
+  if (w == 0) {
+    u64 t = (l < nw) ? sh[l] : 0ull, ti = t;
+    for (int o = 1; o < 32; o <<= 1) {
+      u64 n = __shfl_up_sync(0xFFFFFFFFu, ti, o);
+      if (l >= o) ti += n;
+    }
+    if (l < nw) sh[l] = ti - t;          // exclusive warp offsets
+    if (l == 31) sh[32] = ti;            // block total
+  }
+  __syncthreads();
+  *total = sh[32];
+  return sh[w] + inc - v;
+}
+
+// Row maximum of stored logits (value only).
+template <typename T>
+__device__ __forceinline__ float row_max(const T *row, int V, float *sh) {
+  float m = -INFINITY;
+  for (int k = threadIdx.x; k < V; k += blockDim.x) m = fmaxf(m, to_f32(row[k]));
+  return block_max(m, sh);
+}
+
+// Inverse CDF in ascending token id over integer weights weight(k), k in [0, V):
+// returns the smallest k whose inclusive prefix sum exceeds (U * total) >> 24, or -1 if the
+// total is zero.  Each thread owns a contiguous chunk of tokens.  All threads get the result.
+template <class WeightFn>
+__device__ __forceinline__ int block_inverse_cdf(int V, u32 U, WeightFn weight, u64 *sh64 /*[34]*/, u64 *total_out) {
+  int chunk = (V + blockDim.x - 1) / blockDim.x;
+  int k0 = threadIdx.x * chunk, k1 = min(V, k0 + chunk);
+  u64 local = 0;
+  for (int k = k0; k < k1; ++k) local += weight(k);
+  u64 total;
+  u64 excl = block_exclusive_scan(local, sh64, &total);
+  if (total_out) *total_out = total;
+  int *result = reinterpret_cast<int *>(&sh64[33]);
+  if (threadIdx.x == 0) *result = -1;
+  __syncthreads();
+  if (total != 0) {
+    u64 tau = cdf_threshold(U, total);
+    if (tau >= excl && tau < excl + local) {       // exactly one thread
+      u64 c = excl;
+      for (int k = k0; k < k1; ++k) {
+        c += weight(k);
+        if (c > tau) { *result = k; break; }
+      }
+    }
+  }
+  __syncthreads();
+  int r = *result;
+  __syncthreads();
+  return r;
+}
+
+}  // namespace hsd
