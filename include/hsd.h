@@ -80,6 +80,78 @@ int hsd_verify_level(int level, const void *target_logits, const void *draft_log
                      uint64_t seed, uint64_t call_serial, void *workspace, size_t workspace_bytes,
                      void *stream, int32_t *out_tokens, int32_t *out_n_accepted);
 
+
+/* ---------------------------------------------------------------------------------------
+ * The hierarchy: models M_0..M_K as early exits of one decoder-only transformer (Section 5.1:
+ * level i = the first exit_layers[i] layers followed by the shared final norm and the shared
+ * output head), parameters T_0..T_{K-1} (Algorithm 1).
+ *
+ * Network (the paper uses pretrained checkpoints and does not describe it; this is the
+ * Llama-style decoder of the benchmark shapes): pre-norm residual blocks, RMSNorm with gain,
+ * rotary embedding with half-split pairing, causal attention with grouped KV heads, SwiGLU MLP,
+ * untied output head, softmax at temperature 1 over the whole vocabulary.  Matrices are stored
+ * [out_features, in_features] row-major in `dtype`.
+ */
+typedef struct hsd_ctx hsd_ctx; /* opaque; owns host bookkeeping only */
+
+typedef struct {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+  int32_t dtype;                     /* HSD_F32 or HSD_BF16 */
+  float rms_eps, rope_theta;
+  int32_t max_batch, max_seq;        /* capacity: sequences, tokens per sequence (prompt + generated + drafts) */
+  int32_t page_size;                 /* tokens per KV page (0 = 16) */
+  const void *embed;                 /* device [vocab, d_model] */
+  const void *final_norm;            /* device [d_model] */
+  const void *lm_head;               /* device [vocab, d_model] */
+  const void *const *layer_weights;  /* HOST array [n_layers * 9] of device pointers, per layer:
+                                        attn_norm[d], wq[nq*hd, d], wk[nkv*hd, d], wv[nkv*hd, d], wo[d, nq*hd],
+                                        mlp_norm[d], wg[ff, d], wu[ff, d], wd[d, ff] */
+} hsd_model_desc;
+
+/* Per-level counters accumulated over one hsd_generate call.  Level 0: calls = HSD(0) calls,
+ * emitted = drafted tokens.  Level i >= 1: calls = Verify calls, drafted = tokens received,
+ * tested = accept tests of Algorithm 2's sequential loop, accepted = sum of n, emitted = sum of n+1.
+ * rows = token rows pushed through the level's forward passes (drafts + catch-up rows);
+ * forwards = forward passes; ms = device time of those passes. */
+typedef struct {
+  int64_t calls, rows, drafted, tested, accepted, emitted, forwards;
+  double ms;
+} hsd_level_stats;
+
+/* Device workspace needed by hsd_create for this model / hierarchy (KV pages, token buffers,
+ * per-level logits rows, activations, scratch).  0 on invalid arguments. */
+size_t hsd_workspace_bytes(const hsd_model_desc *model, const int32_t *exit_layers, int n_levels, const int32_t *T);
+
+/* Build a context.  exit_layers [n_levels] ascending, last == n_layers; T [n_levels - 1], each >= 1
+ * (n_levels == 1: plain autoregressive sampling from the target; n_levels == 2: single-draft
+ * speculative decoding).  workspace: device, 256-byte aligned, >= hsd_workspace_bytes(), must
+ * outlive the context, as must the weights.  The descriptor itself is only read during the call.
+ * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL, UNSUPPORTED (head_dim not in {32,64,128}, ...), CUDA. */
+int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_levels, const int32_t *T,
+               void *workspace, size_t workspace_bytes, hsd_ctx **out);
+
+/* Generate n_new tokens per sequence with Algorithm 1 called at idx = K until enough tokens exist
+ * (the first n_new are returned).  Sequence b produces exactly the tokens it would produce alone
+ * with the same seed (uniforms are keyed by b).
+ *   prompt_ids  device int32 [batch, prompt_len], prompt_len >= 1
+ *   out_tokens  device int32 [batch, n_new]
+ *   stats       host [n_levels] or NULL; overwritten
+ *   timing_ms   host [2] or NULL: device time of the prompt pass and of the generation loop
+ * Blocks until done (the host reads one accept count per verification).  Requires
+ * prompt_len + n_new + sum(T) + n_levels + 1 <= max_seq and batch <= max_batch.
+ * Errors: INVALID_ARG, OUT_OF_PAGES, CUDA, IO (trace file). */
+int hsd_generate(hsd_ctx *ctx, const int32_t *prompt_ids, int batch, int prompt_len, int n_new, uint64_t seed,
+                 void *stream, int32_t *out_tokens, hsd_level_stats *stats, double *timing_ms);
+
+/* Decision log for parity checks: every level-0 call and every verification appends one binary
+ * record to `path` (NULL closes the log).  Record = 12 int32 {0x48534454, level, sequence, serial,
+ * context length, t, n, forward rows, logit rows, has_logits, vocab, dtype} + t drafted tokens (level 0:
+ * the T_0 sampled tokens) + [level >= 1: the final token m] + [the call's own logit rows, raw, if
+ * has_logits].  Logits are included for the first `logit_calls` records only. */
+int hsd_set_trace(hsd_ctx *ctx, const char *path, int logit_calls);
+
+void hsd_destroy(hsd_ctx *ctx);
+
 #ifdef __cplusplus
 }
 #endif

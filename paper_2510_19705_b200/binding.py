@@ -100,3 +100,129 @@ def hsd_verify_level(level, target_logits, draft_logits, draft_tokens, seed, cal
                                       _dtype_code(target_logits), seed, call_serial, _dev(workspace),
                                       workspace.numel(), _stream(), _dev(out_tokens), _dev(out_n_accepted)))
     return out_tokens, out_n_accepted
+
+
+# ------------------------------------------------------------------------------------- engine
+class _ModelDesc(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("d_model", ctypes.c_int32), ("n_q_heads", ctypes.c_int32),
+                ("n_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("d_ff", ctypes.c_int32),
+                ("vocab", ctypes.c_int32), ("dtype", ctypes.c_int32), ("rms_eps", ctypes.c_float),
+                ("rope_theta", ctypes.c_float), ("max_batch", ctypes.c_int32), ("max_seq", ctypes.c_int32),
+                ("page_size", ctypes.c_int32), ("embed", ctypes.c_void_p), ("final_norm", ctypes.c_void_p),
+                ("lm_head", ctypes.c_void_p), ("layer_weights", ctypes.POINTER(ctypes.c_void_p))]
+
+
+class LevelStats(ctypes.Structure):
+    _fields_ = [("calls", ctypes.c_int64), ("rows", ctypes.c_int64), ("drafted", ctypes.c_int64),
+                ("tested", ctypes.c_int64), ("accepted", ctypes.c_int64), ("emitted", ctypes.c_int64),
+                ("forwards", ctypes.c_int64), ("ms", ctypes.c_double)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+_LAYER_KEYS = ("attn_norm", "wq", "wk", "wv", "wo", "mlp_norm", "wg", "wu", "wd")
+
+
+def _declare_engine(lib):
+    c = ctypes
+    vp, i32, u64, sz = c.c_void_p, c.c_int, c.c_uint64, c.c_size_t
+    lib.hsd_workspace_bytes.restype = sz
+    lib.hsd_workspace_bytes.argtypes = [c.POINTER(_ModelDesc), c.POINTER(c.c_int32), i32, c.POINTER(c.c_int32)]
+    lib.hsd_create.restype = i32
+    lib.hsd_create.argtypes = [c.POINTER(_ModelDesc), c.POINTER(c.c_int32), i32, c.POINTER(c.c_int32), vp, sz,
+                               c.POINTER(vp)]
+    lib.hsd_generate.restype = i32
+    lib.hsd_generate.argtypes = [vp, vp, i32, i32, i32, u64, vp, vp, c.POINTER(LevelStats), c.POINTER(c.c_double)]
+    lib.hsd_set_trace.restype = i32
+    lib.hsd_set_trace.argtypes = [vp, c.c_char_p, i32]
+    lib.hsd_destroy.restype = None
+    lib.hsd_destroy.argtypes = [vp]
+
+
+class Hsd:
+    """A hierarchy M_0..M_K of early exits of one decoder (hsd_create / hsd_generate / hsd_destroy).
+
+    cfg: dict as produced by inputs.model_cfg; weights: dict of CUDA tensors (inputs.make_weights);
+    exits: exit layer per level (last == n_layers); T: T_0..T_{K-1}."""
+
+    def __init__(self, cfg, weights, exits, T, max_batch, max_seq, page_size=16):
+        lib = library()
+        _declare_engine(lib)
+        self._lib = lib
+        self.cfg, self.exits, self.T = dict(cfg), list(exits), list(T)
+        self.weights = weights                      # keep the device buffers alive
+        n_layers = cfg["n_layers"]
+        ptrs = (ctypes.c_void_p * (n_layers * 9))()
+        for l, layer in enumerate(weights["layers"]):
+            for k, name in enumerate(_LAYER_KEYS):
+                t = layer[name]
+                assert t.is_cuda and t.is_contiguous()
+                ptrs[l * 9 + k] = t.data_ptr()
+        self._ptrs = ptrs
+        d = _ModelDesc(n_layers, cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"],
+                       cfg["vocab"], HSD_BF16 if cfg["dtype"] == "bf16" else HSD_F32, cfg["rms_eps"],
+                       cfg["rope_theta"], max_batch, max_seq, page_size, weights["embed"].data_ptr(),
+                       weights["final_norm"].data_ptr(), weights["lm_head"].data_ptr(), ptrs)
+        self._desc = d
+        n_levels = len(self.exits)
+        ex = (ctypes.c_int32 * n_levels)(*self.exits)
+        tt = (ctypes.c_int32 * max(1, n_levels - 1))(*(self.T or [1]))
+        need = lib.hsd_workspace_bytes(ctypes.byref(d), ex, n_levels, tt)
+        if need == 0:
+            raise HsdError("hsd_workspace_bytes rejected the configuration")
+        self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=weights["embed"].device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        ctx = ctypes.c_void_p()
+        _check(lib.hsd_create(ctypes.byref(d), ex, n_levels, tt, ctypes.c_void_p(base), need, ctypes.byref(ctx)))
+        self._ctx = ctx
+        self.n_levels = n_levels
+        self.workspace_bytes = need
+
+    def set_trace(self, path, logit_calls=0):
+        _check(self._lib.hsd_set_trace(self._ctx, path.encode() if path else None, logit_calls))
+
+    def generate(self, prompt_ids, n_new, seed):
+        """prompt_ids: CUDA int32 [batch, prompt_len] -> (tokens CUDA int32 [batch, n_new], [per-level stats
+        dicts], (prompt_ms, generate_ms))."""
+        batch, plen = prompt_ids.shape
+        out = torch.empty(batch, n_new, dtype=torch.int32, device=prompt_ids.device)
+        stats = (LevelStats * self.n_levels)()
+        timing = (ctypes.c_double * 2)()
+        _check(self._lib.hsd_generate(self._ctx, _dev(prompt_ids), batch, plen, n_new, seed, _stream(), _dev(out),
+                                      stats, timing))
+        return out, [s.as_dict() for s in stats], (timing[0], timing[1])
+
+    def close(self):
+        if getattr(self, "_ctx", None):
+            self._lib.hsd_destroy(self._ctx)
+            self._ctx = None
+
+    def __del__(self):
+        self.close()
+
+
+def read_trace(path):
+    """Parse a decision log written by hsd_set_trace into a list of dicts (numpy logits as float32)."""
+    import numpy as np
+    recs = []
+    with open(path, "rb") as f:
+        while True:
+            hdr = f.read(48)
+            if len(hdr) < 48:
+                break
+            h = np.frombuffer(hdr, dtype=np.int32)
+            assert int(h[0]) == 0x48534454
+            level, seq, serial, ctx_len, t, n, rows, lrows, has_logits, V, dtype = (int(v) for v in h[1:12])
+            n_tok = (n if level == 0 else t + 1)
+            toks = np.frombuffer(f.read(4 * n_tok), dtype=np.int32).copy()
+            logits = None
+            if has_logits:
+                if dtype == HSD_BF16:
+                    raw = np.frombuffer(f.read(2 * lrows * V), dtype=np.uint16)
+                    logits = (raw.astype(np.uint32) << 16).view(np.float32).reshape(lrows, V)
+                else:
+                    logits = np.frombuffer(f.read(4 * lrows * V), dtype=np.float32).reshape(lrows, V).copy()
+            recs.append(dict(level=level, seq=seq, serial=serial, ctx_len=ctx_len, t=t, n=n, rows=rows,
+                             tokens=toks, logits=logits))
+    return recs

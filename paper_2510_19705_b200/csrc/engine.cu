@@ -1,0 +1,656 @@
+// Host control of the HSD hot path: Algorithm 1's recursion (level-synchronous over a batch of
+// independent sequences), the per-level verification step (multi-row forward -> acceptance /
+// resample -> KV rollback), KV paging, workspace carving, statistics and the decision log.
+#include <stdio.h>
+#include <math.h>
+#include <algorithm>
+#include <new>
+#include <vector>
+
+#include "forward.cuh"
+#include "sampling_api.cuh"
+
+using namespace hsd;
+
+namespace {
+
+constexpr int kRingSlots = 48;
+constexpr int kTimerPairs = 64;
+constexpr int kAttnBlocksTarget = 512;
+constexpr int kMaxSplits = 64;
+constexpr int kPrefillRows = 128;
+constexpr uint32_t kTraceMagic = 0x48534454u;
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+size_t elem_size(int dtype) { return dtype == HSD_BF16 ? 2 : 4; }
+
+// Workspace layout, shared by hsd_workspace_bytes and hsd_create.
+struct Layout {
+  size_t tokens, cos_tab, sin_tab, page_table, k_pool, v_pool, pool_layer_stride, x, h, qkv, q, att, act, partials, hf,
+      vscratch, n_acc, ring, total;
+  std::vector<size_t> logits;
+  std::vector<int> slots;
+  int max_rows, pages_per_seq, n_pages, partial_rows;
+  size_t ring_slot;
+};
+
+bool valid_model(const hsd_model_desc *m, const int32_t *exits, int n_levels, const int32_t *T) {
+  if (!m || !exits || n_levels < 1 || n_levels > 16) return false;
+  if (n_levels > 1 && !T) return false;
+  if (m->n_layers < 1 || m->d_model < 8 || m->n_q_heads < 1 || m->n_kv_heads < 1 || m->head_dim < 2 || m->d_ff < 8 ||
+      m->vocab < 2)
+    return false;
+  if (m->dtype != HSD_F32 && m->dtype != HSD_BF16) return false;
+  if (m->max_batch < 1 || m->max_seq < 4 || m->page_size < 0) return false;
+  if (m->n_q_heads % m->n_kv_heads != 0 || (m->head_dim & 1)) return false;
+  for (int i = 0; i < n_levels; ++i) {
+    if (exits[i] < 1 || exits[i] > m->n_layers) return false;
+    if (i > 0 && exits[i] <= exits[i - 1]) return false;
+  }
+  if (exits[n_levels - 1] != m->n_layers) return false;
+  for (int i = 0; i + 1 < n_levels; ++i)
+    if (T[i] < 1 || T[i] > 64) return false;
+  return true;
+}
+
+Layout make_layout(const hsd_model_desc *m, int n_levels, const int32_t *T) {
+  Layout L;
+  const size_t es = elem_size(m->dtype);
+  const int page = m->page_size ? m->page_size : 16;
+  const int B = m->max_batch, d = m->d_model, hd = m->head_dim, nq = m->n_q_heads, nkv = m->n_kv_heads;
+  int sumT = 0;
+  L.slots.resize(n_levels);
+  for (int i = 0; i < n_levels; ++i) {
+    if (i + 1 < n_levels) sumT += T[i];
+    L.slots[i] = (i + 1 < n_levels ? sumT : sumT) + 1;      // level i keeps at most sum_{j<=i} T_j (+1) rows
+  }
+  if (n_levels == 1) L.slots[0] = 1;
+  // rows of one forward: drafts of the level below + catch-up rows (<= n_levels), per sequence
+  int decode_rows = B * (sumT + n_levels + 1);
+  L.max_rows = std::max(kPrefillRows, decode_rows);
+  L.pages_per_seq = (m->max_seq + page - 1) / page;
+  L.n_pages = B * L.pages_per_seq;
+  L.partial_rows = L.max_rows + kAttnRows * kAttnBlocksTarget / nkv + kAttnRows * kMaxSplits;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  L.tokens = take((size_t)B * m->max_seq * 4);
+  L.cos_tab = take((size_t)m->max_seq * (hd / 2) * 4);
+  L.sin_tab = take((size_t)m->max_seq * (hd / 2) * 4);
+  L.page_table = take((size_t)B * L.pages_per_seq * 4);
+  L.pool_layer_stride = align_up((size_t)L.n_pages * nkv * page * hd * es, 256);
+  L.k_pool = take(L.pool_layer_stride * m->n_layers);
+  L.v_pool = take(L.pool_layer_stride * m->n_layers);
+  L.x = take((size_t)L.max_rows * d * 4);
+  L.h = take((size_t)L.max_rows * d * es);
+  L.qkv = take((size_t)L.max_rows * (nq + 2 * nkv) * hd * 4);
+  L.q = take((size_t)L.max_rows * nq * hd * es);
+  L.att = take((size_t)L.max_rows * nq * hd * es);
+  L.act = take((size_t)L.max_rows * m->d_ff * es);
+  L.partials = take((size_t)L.partial_rows * nq * (hd + 2) * 4);
+  int max_logit_rows = 0;
+  L.logits.resize(n_levels);
+  for (int i = 0; i < n_levels; ++i) {
+    L.logits[i] = take((size_t)B * L.slots[i] * m->vocab * es);
+    max_logit_rows = std::max(max_logit_rows, B * L.slots[i]);
+  }
+  L.hf = take((size_t)max_logit_rows * d * es);
+  L.vscratch = take(verify_scratch_bytes(B, sumT + 1));
+  L.n_acc = take((size_t)B * 4);
+  L.ring_slot = align_up((size_t)L.max_rows * 40 + (size_t)B * 96 + 1024, 256);
+  L.ring = take(L.ring_slot * kRingSlots);
+  L.total = off;
+  return L;
+}
+
+struct SeqWork {
+  int b, start, end;     // rows = positions [start, end)
+  int logit_first;       // first position whose output row is wanted (-1: none); rows up to end - 1
+  int slot0;             // destination slot of that first row in the level's logits buffer
+};
+
+struct TimerPair { cudaEvent_t a, b; int level; };
+
+}  // namespace
+
+struct hsd_ctx {
+  ModelDims md;
+  int n_levels, max_batch;
+  std::vector<int> exits, T;
+  Layout lay;
+  char *ws;
+  const void *embed, *final_norm, *lm_head;
+  std::vector<const void *> lw;
+  // pinned host mirrors
+  char *ring_host;
+  int *n_acc_host;
+  int *page_table_host;
+  int ring_next, ring_in_flight;
+  // per-sequence state
+  std::vector<int> buf_len;
+  std::vector<std::vector<int>> len_g;        // [b][level]: leading positions whose KV in group `level` is valid
+  std::vector<std::vector<uint32_t>> serial;  // [b][level]
+  std::vector<int> n_pages_of;
+  std::vector<int> free_pages;
+  std::vector<char> pt_dirty;
+  // statistics / timing
+  std::vector<hsd_level_stats> stats;
+  TimerPair timers[kTimerPairs];
+  int timers_used;
+  bool timers_ok;
+  // decision log
+  FILE *trace;
+  int trace_logit_calls, trace_records;
+  cudaStream_t stream;
+  uint64_t seed;
+
+  template <typename U> U *dev(size_t off) const { return reinterpret_cast<U *>(ws + off); }
+};
+
+namespace {
+
+int sync_stream(hsd_ctx *c) {
+  if (cudaStreamSynchronize(c->stream) != cudaSuccess) return HSD_E_CUDA;
+  c->ring_in_flight = 0;
+  for (int i = 0; i < c->timers_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->timers[i].a, c->timers[i].b) == cudaSuccess) c->stats[c->timers[i].level].ms += ms;
+  }
+  c->timers_used = 0;
+  return HSD_OK;
+}
+
+// A slot of the descriptor ring: host pointer to fill + matching device address.
+int ring_acquire(hsd_ctx *c, char **host, char **devp) {
+  if (c->ring_in_flight >= kRingSlots) {
+    int st = sync_stream(c);
+    if (st) return st;
+  }
+  int s = c->ring_next;
+  c->ring_next = (c->ring_next + 1) % kRingSlots;
+  c->ring_in_flight++;
+  *host = c->ring_host + (size_t)s * c->lay.ring_slot;
+  *devp = c->ws + c->lay.ring + (size_t)s * c->lay.ring_slot;
+  return HSD_OK;
+}
+
+int ensure_pages(hsd_ctx *c, int b, int upto_len) {
+  const int page = c->md.page;
+  int need = (upto_len + page - 1) / page;
+  if (need > c->md.pages_per_seq) return HSD_E_INVALID_ARG;
+  while (c->n_pages_of[b] < need) {
+    if (c->free_pages.empty()) return HSD_E_OUT_OF_PAGES;
+    int pg = c->free_pages.back();
+    c->free_pages.pop_back();
+    c->page_table_host[(size_t)b * c->md.pages_per_seq + c->n_pages_of[b]] = pg;
+    c->n_pages_of[b]++;
+    c->pt_dirty[b] = 1;
+  }
+  return HSD_OK;
+}
+
+void trim_pages(hsd_ctx *c, int b, int keep_len) {
+  const int page = c->md.page;
+  int keep = (keep_len + page - 1) / page;
+  while (c->n_pages_of[b] > keep) {
+    c->n_pages_of[b]--;
+    c->free_pages.push_back(c->page_table_host[(size_t)b * c->md.pages_per_seq + c->n_pages_of[b]]);
+  }
+}
+
+int upload_page_tables(hsd_ctx *c) {
+  for (int b = 0; b < c->max_batch; ++b) {
+    if (!c->pt_dirty[b]) continue;
+    size_t off = (size_t)b * c->md.pages_per_seq;
+    HSD_CUDA_OK(cudaMemcpyAsync(c->dev<int>(c->lay.page_table) + off, c->page_table_host + off,
+                                (size_t)c->n_pages_of[b] * 4, cudaMemcpyHostToDevice, c->stream));
+    c->pt_dirty[b] = 0;
+  }
+  return HSD_OK;
+}
+
+// One forward pass of level `level` (layers 1..exit) over the given rows; logits of the wanted
+// rows go to the level's logits buffer.  KV of every processed position is (re)written.
+int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
+  const ModelDims &md = c->md;
+  const Layout &L = c->lay;
+  int R = 0, n_attn = 0, n_logit = 0, max_kv = 0;
+  for (const SeqWork &w : work) {
+    int rows = w.end - w.start;
+    if (rows <= 0 || w.start < 0 || w.end > md.max_seq) return HSD_E_INVALID_ARG;
+    R += rows;
+    n_attn += (rows + kAttnRows - 1) / kAttnRows;
+    if (w.logit_first >= 0) {
+      if (w.logit_first < w.start || w.logit_first >= w.end) return HSD_E_INVALID_ARG;
+      n_logit += w.end - w.logit_first;
+    }
+    max_kv = std::max(max_kv, w.end);
+    int st = ensure_pages(c, w.b, w.end);
+    if (st) return st;
+  }
+  if (R == 0) return HSD_OK;
+  if (R > L.max_rows) return HSD_E_INVALID_ARG;
+  char *host, *devp;
+  int st = ring_acquire(c, &host, &devp);
+  if (st) return st;
+  // slot layout: row_seq[R] | row_pos[R] | attn int4[n_attn] | lrow_src[n_logit] | lrow_dst int64[n_logit]
+  size_t o_seq = 0, o_pos = align_up(o_seq + (size_t)R * 4, 16), o_attn = align_up(o_pos + (size_t)R * 4, 16),
+         o_src = align_up(o_attn + (size_t)n_attn * 16, 16), o_dst = align_up(o_src + (size_t)n_logit * 4, 16),
+         bytes = o_dst + (size_t)n_logit * 8;
+  if (bytes > L.ring_slot) return HSD_E_INVALID_ARG;
+  int *row_seq = (int *)(host + o_seq), *row_pos = (int *)(host + o_pos), *lsrc = (int *)(host + o_src);
+  int4 *attn = (int4 *)(host + o_attn);
+  long long *ldst = (long long *)(host + o_dst);
+  int r = 0, ia = 0, il = 0;
+  for (const SeqWork &w : work) {
+    for (int p0 = w.start; p0 < w.end; p0 += kAttnRows) {
+      int rows = std::min(kAttnRows, w.end - p0);
+      attn[ia++] = make_int4(r + (p0 - w.start), rows, w.b, p0);
+    }
+    for (int p = w.start; p < w.end; ++p, ++r) {
+      row_seq[r] = w.b;
+      row_pos[r] = p;
+      if (w.logit_first >= 0 && p >= w.logit_first) {
+        lsrc[il] = r;
+        ldst[il] = (long long)w.b * L.slots[level] + w.slot0 + (p - w.logit_first);
+        if (w.slot0 + (p - w.logit_first) >= L.slots[level]) return HSD_E_INVALID_ARG;
+        ++il;
+      }
+    }
+  }
+  HSD_CUDA_OK(cudaMemcpyAsync(devp, host, bytes, cudaMemcpyHostToDevice, c->stream));
+  st = upload_page_tables(c);
+  if (st) return st;
+  RowBatch rb;
+  rb.R = R;
+  rb.row_seq = (const int *)(devp + o_seq);
+  rb.row_pos = (const int *)(devp + o_pos);
+  rb.n_attn = n_attn;
+  rb.attn = (const int4 *)(devp + o_attn);
+  rb.max_kv_len = max_kv;
+  rb.L = n_logit;
+  rb.lrow_src = (const int *)(devp + o_src);
+  rb.lrow_dst = (const long long *)(devp + o_dst);
+
+  // attention split: enough blocks to fill the GPU, never more partial rows than the buffer holds
+  int n_splits = std::max(1, std::min(kMaxSplits, kAttnBlocksTarget / std::max(1, n_attn * md.nkv)));
+  int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, kAttnKeyTile);
+  n_splits = (max_kv + keys_per_split - 1) / keys_per_split;
+  if ((size_t)R * n_splits > (size_t)L.partial_rows) return HSD_E_INVALID_ARG;
+
+  TimerPair *tp = nullptr;
+  if (c->timers_ok && c->timers_used < kTimerPairs) {
+    tp = &c->timers[c->timers_used++];
+    tp->level = level;
+    cudaEventRecord(tp->a, c->stream);
+  }
+  cudaStream_t s = c->stream;
+  float *x = c->dev<float>(L.x);
+  void *h = c->dev<void>(L.h), *q = c->dev<void>(L.q), *att = c->dev<void>(L.att), *act = c->dev<void>(L.act);
+  float *qkv = c->dev<float>(L.qkv);
+  const int *pt = c->dev<int>(L.page_table);
+#define HSD_TRY(e) do { int st__ = (e); if (st__) return st__; } while (0)
+  HSD_TRY(launch_embed(md, c->embed, c->dev<int>(L.tokens), rb, x, s));
+  for (int l = 0; l < c->exits[level]; ++l) {
+    const void *const *w = &c->lw[(size_t)l * 9];
+    void *kp = c->ws + L.k_pool + L.pool_layer_stride * l, *vp = c->ws + L.v_pool + L.pool_layer_stride * l;
+    HSD_TRY(launch_rmsnorm(md, x, w[0], nullptr, R, h, s));
+    GemmSegs qkv_segs = {{w[1], w[2], w[3]}, {md.nq * md.hd, md.nkv * md.hd, md.nkv * md.hd}, 3};
+    HSD_TRY(launch_gemm_simt(md, h, R, md.d, qkv_segs, GEMM_STORE_F32, qkv, nullptr, nullptr, s));
+    HSD_TRY(launch_rope_kv(md, qkv, rb, c->dev<float>(L.cos_tab), c->dev<float>(L.sin_tab), pt, kp, vp, q, s));
+    HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(L.partials), keys_per_split, n_splits, att, s));
+    GemmSegs o_segs = {{w[4], nullptr, nullptr}, {md.d, 0, 0}, 1};
+    HSD_TRY(launch_gemm_simt(md, att, R, md.nq * md.hd, o_segs, GEMM_ADD_F32, x, nullptr, nullptr, s));
+    HSD_TRY(launch_rmsnorm(md, x, w[5], nullptr, R, h, s));
+    GemmSegs gu_segs = {{w[6], w[7], nullptr}, {md.ff, md.ff, 0}, 2};
+    HSD_TRY(launch_gemm_simt(md, h, R, md.d, gu_segs, GEMM_SWIGLU_T, nullptr, act, nullptr, s));
+    GemmSegs d_segs = {{w[8], nullptr, nullptr}, {md.d, 0, 0}, 1};
+    HSD_TRY(launch_gemm_simt(md, act, R, md.ff, d_segs, GEMM_ADD_F32, x, nullptr, nullptr, s));
+  }
+  if (n_logit > 0) {
+    void *hf = c->dev<void>(L.hf);
+    HSD_TRY(launch_rmsnorm(md, x, c->final_norm, rb.lrow_src, n_logit, hf, s));
+    GemmSegs lm_segs = {{c->lm_head, nullptr, nullptr}, {md.V, 0, 0}, 1};
+    HSD_TRY(launch_gemm_simt(md, hf, n_logit, md.d, lm_segs, GEMM_STORE_T_SCATTER, nullptr, c->ws + L.logits[level],
+                             rb.lrow_dst, s));
+  }
+  if (tp) cudaEventRecord(tp->b, s);
+  c->stats[level].forwards++;
+  c->stats[level].rows += R;
+  for (const SeqWork &w : work)
+    for (int g = 0; g <= level; ++g) c->len_g[w.b][g] = w.end;
+  return HSD_OK;
+}
+
+// ---------------------------------------------------------------------------- decision log
+int fetch_tokens(hsd_ctx *c, int b, int pos0, int n, std::vector<int32_t> &out) {
+  size_t base = out.size();
+  out.resize(base + n);
+  if (n == 0) return HSD_OK;
+  if (cudaMemcpyAsync(out.data() + base, c->dev<int>(c->lay.tokens) + (size_t)b * c->md.max_seq + pos0, (size_t)n * 4,
+                      cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
+    return HSD_E_CUDA;
+  return cudaStreamSynchronize(c->stream) == cudaSuccess ? HSD_OK : HSD_E_CUDA;
+}
+
+int trace_write(hsd_ctx *c, int level, int b, uint32_t serial, int ctx_len, int t, int n, int fwd_rows, int logit_rows,
+                long long logit_row0, const std::vector<int32_t> &toks) {
+  if (!c->trace) return HSD_OK;
+  const ModelDims &md = c->md;
+  int has_logits = c->trace_records < c->trace_logit_calls;
+  int32_t hdr[12] = {(int32_t)kTraceMagic, level, b, (int32_t)serial, ctx_len, t, n, fwd_rows, logit_rows, has_logits, md.V,
+                     md.dtype};
+  std::vector<char> rows;
+  if (has_logits) {
+    rows.resize((size_t)logit_rows * md.V * elem_size(md.dtype));
+    if (cudaMemcpyAsync(rows.data(), c->ws + c->lay.logits[level] + (size_t)logit_row0 * md.V * elem_size(md.dtype),
+                        rows.size(), cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
+      return HSD_E_CUDA;
+    if (cudaStreamSynchronize(c->stream) != cudaSuccess) return HSD_E_CUDA;
+  }
+  if (fwrite(hdr, 4, 12, c->trace) != 12) return HSD_E_IO;
+  if (!toks.empty() && fwrite(toks.data(), 4, toks.size(), c->trace) != toks.size()) return HSD_E_IO;
+  if (has_logits && fwrite(rows.data(), 1, rows.size(), c->trace) != rows.size()) return HSD_E_IO;
+  c->trace_records++;
+  return HSD_OK;
+}
+
+// ---------------------------------------------------------------------------- Algorithm 1
+// Level 0: T_0 single-step forwards, each followed by the draft sample written into the token
+// buffer on the device (no host round trip inside the loop).
+int run_level0(hsd_ctx *c, const std::vector<int> &act) {
+  const Layout &L = c->lay;
+  const int steps = c->n_levels > 1 ? c->T[0] : 1;
+  std::vector<int> ctx0(act.size());
+  std::vector<uint32_t> ser(act.size());
+  for (size_t i = 0; i < act.size(); ++i) {
+    ctx0[i] = c->buf_len[act[i]];
+    ser[i] = c->serial[act[i]][0]++;
+  }
+  for (int j = 0; j < steps; ++j) {
+    std::vector<SeqWork> work;
+    for (int b : act) {
+      int len = c->buf_len[b];
+      int start = std::min(c->len_g[b][0], len - 1);
+      work.push_back({b, start, len, len - 1, j});
+    }
+    HSD_TRY(forward(c, 0, work));
+    char *host, *devp;
+    HSD_TRY(ring_acquire(c, &host, &devp));
+    SampleRow *rows = (SampleRow *)host;
+    for (size_t i = 0; i < act.size(); ++i) {
+      int b = act[i];
+      rows[i].logit_row = (long long)b * L.slots[0] + j;
+      rows[i].out_index = (long long)b * c->md.max_seq + c->buf_len[b];
+      rows[i].j = j; rows[i].serial = ser[i]; rows[i].seq = b; rows[i].level = 0;
+      c->buf_len[b]++;
+    }
+    HSD_CUDA_OK(cudaMemcpyAsync(devp, host, act.size() * sizeof(SampleRow), cudaMemcpyHostToDevice, c->stream));
+    HSD_TRY(launch_draft_sample(c->ws + L.logits[0], c->md.dtype, c->md.V, (const SampleRow *)devp, (int)act.size(), 1, 0,
+                                c->seed, c->dev<int>(L.tokens), c->stream));
+  }
+  for (size_t i = 0; i < act.size(); ++i) {
+    hsd_level_stats &st = c->stats[0];
+    st.calls++;
+    st.emitted += steps;
+    if (c->trace) {
+      std::vector<int32_t> toks;
+      HSD_TRY(fetch_tokens(c, act[i], ctx0[i], steps, toks));
+      HSD_TRY(trace_write(c, 0, act[i], ser[i], ctx0[i], 0, steps, steps, steps, (long long)act[i] * L.slots[0], toks));
+    }
+  }
+  return HSD_OK;
+}
+
+// Verify(level) for the active sequences: drafts are tokens [ctx[b], buf_len[b]) with draft rows in
+// the lower level's slots 0..t-1; this level's rows go to its slots count[b]..count[b]+t.
+int run_verify(hsd_ctx *c, int level, const std::vector<int> &act, const std::vector<int> &ctx, std::vector<int> &count) {
+  const Layout &L = c->lay;
+  std::vector<SeqWork> work;
+  int t_max = 0;
+  for (int b : act) {
+    int t = c->buf_len[b] - ctx[b];
+    if (t < 1 || ctx[b] < 1) return HSD_E_INVALID_ARG;
+    int start = std::min(c->len_g[b][level], ctx[b] - 1);
+    work.push_back({b, start, c->buf_len[b], ctx[b] - 1, count[b]});
+    t_max = std::max(t_max, t);
+  }
+  HSD_TRY(forward(c, level, work));
+  char *host, *devp;
+  HSD_TRY(ring_acquire(c, &host, &devp));
+  VerifySeq *vs = (VerifySeq *)host;
+  std::vector<uint32_t> ser(act.size());
+  for (size_t i = 0; i < act.size(); ++i) {
+    int b = act[i];
+    ser[i] = c->serial[b][level]++;
+    vs[i].p_row0 = (long long)b * L.slots[level] + count[b];
+    vs[i].q_row0 = (long long)b * L.slots[level - 1];
+    vs[i].tok_off = (long long)b * c->md.max_seq + ctx[b];
+    vs[i].t = c->buf_len[b] - ctx[b];
+    vs[i].serial = ser[i]; vs[i].seq = b; vs[i].level = level;
+  }
+  HSD_CUDA_OK(cudaMemcpyAsync(devp, host, act.size() * sizeof(VerifySeq), cudaMemcpyHostToDevice, c->stream));
+  std::vector<std::vector<int32_t>> drafts(c->trace ? act.size() : 0);
+  for (size_t i = 0; i < drafts.size(); ++i) HSD_TRY(fetch_tokens(c, act[i], ctx[act[i]], c->buf_len[act[i]] - ctx[act[i]], drafts[i]));
+  HSD_TRY(launch_verify(c->ws + L.logits[level], c->ws + L.logits[level - 1], c->dev<int>(L.tokens), c->md.dtype, c->md.V,
+                        (int)act.size(), t_max, (const VerifySeq *)devp, 0, 0, 0, c->ws + L.vscratch, c->seed, nullptr,
+                        c->dev<int>(L.n_acc), 1, c->stream));
+  HSD_CUDA_OK(cudaMemcpyAsync(c->n_acc_host, c->dev<int>(L.n_acc), act.size() * 4, cudaMemcpyDeviceToHost, c->stream));
+  HSD_TRY(sync_stream(c));
+  hsd_level_stats &st = c->stats[level];
+  for (size_t i = 0; i < act.size(); ++i) {
+    int b = act[i], t = c->buf_len[b] - ctx[b], n = c->n_acc_host[i];
+    if (n < 0 || n > t) return HSD_E_CUDA;
+    // rollback / commit: the buffer keeps x_1..x_n and m; the position of m (and everything the
+    // rejected drafts wrote) is valid in no layer group
+    c->buf_len[b] = ctx[b] + n + 1;
+    for (int g = 0; g < c->n_levels; ++g) c->len_g[b][g] = std::min(c->len_g[b][g], ctx[b] + n);
+    trim_pages(c, b, c->buf_len[b]);
+    st.calls++;
+    st.drafted += t;
+    st.tested += std::min(n + 1, t);
+    st.accepted += n;
+    st.emitted += n + 1;
+    if (c->trace) {
+      HSD_TRY(fetch_tokens(c, b, ctx[b] + n, 1, drafts[i]));          // the final token m
+      HSD_TRY(trace_write(c, level, b, ser[i], ctx[b], t, n, work[i].end - work[i].start, t + 1,
+                          (long long)b * L.slots[level] + count[b], drafts[i]));
+    }
+    count[b] += n + 1;
+  }
+  return HSD_OK;
+}
+
+int run_level(hsd_ctx *c, int level, const std::vector<int> &act) {
+  if (act.empty()) return HSD_OK;
+  if (level == 0) return run_level0(c, act);
+  const int K = c->n_levels - 1;
+  std::vector<int> ctx(c->max_batch, 0), count(c->max_batch, 0);
+  if (level == K) {
+    for (int b : act) ctx[b] = c->buf_len[b];
+    HSD_TRY(run_level(c, level - 1, act));
+    return run_verify(c, level, act, ctx, count);
+  }
+  for (;;) {
+    std::vector<int> need;
+    for (int b : act)
+      if (count[b] < c->T[level]) need.push_back(b);
+    if (need.empty()) break;
+    for (int b : need) ctx[b] = c->buf_len[b];
+    HSD_TRY(run_level(c, level - 1, need));
+    HSD_TRY(run_verify(c, level, need, ctx, count));
+  }
+  return HSD_OK;
+}
+
+int prefill(hsd_ctx *c, int batch, int prompt_len) {
+  // the target runs over prompt positions [0, P-1); the last prompt token stays unprocessed and is
+  // every level's first catch-up row
+  const int K = c->n_levels - 1;
+  int end = prompt_len - 1;
+  std::vector<int> done(batch, 0);
+  for (;;) {
+    std::vector<SeqWork> work;
+    int budget = kPrefillRows;
+    for (int b = 0; b < batch && budget > 0; ++b) {
+      if (done[b] >= end) continue;
+      int rows = std::min(budget, end - done[b]);
+      work.push_back({b, done[b], done[b] + rows, -1, 0});
+      done[b] += rows;
+      budget -= rows;
+    }
+    if (work.empty()) break;
+    HSD_TRY(forward(c, K, work));
+  }
+  return HSD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t hsd_workspace_bytes(const hsd_model_desc *model, const int32_t *exit_layers, int n_levels, const int32_t *T) {
+  if (!valid_model(model, exit_layers, n_levels, T)) return 0;
+  return make_layout(model, n_levels, T).total;
+}
+
+int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_levels, const int32_t *T, void *workspace,
+               size_t workspace_bytes, hsd_ctx **out) {
+  if (!out) return HSD_E_INVALID_ARG;
+  *out = nullptr;
+  if (!valid_model(model, exit_layers, n_levels, T) || !workspace) return HSD_E_INVALID_ARG;
+  if (!model->embed || !model->final_norm || !model->lm_head || !model->layer_weights) return HSD_E_INVALID_ARG;
+  for (int i = 0; i < model->n_layers * 9; ++i)
+    if (!model->layer_weights[i]) return HSD_E_INVALID_ARG;
+  if (((uintptr_t)workspace & 255) != 0) return HSD_E_INVALID_ARG;
+  if (model->head_dim != 32 && model->head_dim != 64 && model->head_dim != 128) return HSD_E_UNSUPPORTED;
+  if (model->n_q_heads / model->n_kv_heads > 8) return HSD_E_UNSUPPORTED;
+  const int vec = model->dtype == HSD_BF16 ? 8 : 4;
+  if (model->d_model % vec || model->d_ff % vec || (model->n_q_heads * model->head_dim) % vec) return HSD_E_UNSUPPORTED;
+  Layout lay = make_layout(model, n_levels, T);
+  if (workspace_bytes < lay.total) return HSD_E_WORKSPACE_TOO_SMALL;
+  hsd_ctx *c = new (std::nothrow) hsd_ctx();
+  if (!c) return HSD_E_INVALID_ARG;
+  c->md = ModelDims{model->n_layers, model->d_model, model->n_q_heads, model->n_kv_heads, model->head_dim, model->d_ff,
+                    model->vocab, model->dtype, model->rms_eps, model->rope_theta, model->max_seq,
+                    model->page_size ? model->page_size : 16, lay.pages_per_seq};
+  c->n_levels = n_levels;
+  c->max_batch = model->max_batch;
+  c->exits.assign(exit_layers, exit_layers + n_levels);
+  if (n_levels > 1) c->T.assign(T, T + n_levels - 1);
+  c->lay = lay;
+  c->ws = (char *)workspace;
+  c->embed = model->embed; c->final_norm = model->final_norm; c->lm_head = model->lm_head;
+  c->lw.assign(model->layer_weights, model->layer_weights + (size_t)model->n_layers * 9);
+  c->ring_host = nullptr; c->n_acc_host = nullptr; c->page_table_host = nullptr;
+  c->trace = nullptr; c->trace_logit_calls = 0; c->trace_records = 0;
+  c->ring_next = 0; c->ring_in_flight = 0; c->timers_used = 0; c->timers_ok = true; c->stream = nullptr; c->seed = 0;
+  bool ok = cudaMallocHost(&c->ring_host, lay.ring_slot * kRingSlots) == cudaSuccess &&
+            cudaMallocHost(&c->n_acc_host, (size_t)c->max_batch * 4) == cudaSuccess &&
+            cudaMallocHost(&c->page_table_host, (size_t)c->max_batch * lay.pages_per_seq * 4) == cudaSuccess;
+  for (int i = 0; i < kTimerPairs; ++i) { c->timers[i].a = nullptr; c->timers[i].b = nullptr; }
+  for (int i = 0; ok && i < kTimerPairs; ++i)
+    c->timers_ok = c->timers_ok && cudaEventCreate(&c->timers[i].a) == cudaSuccess && cudaEventCreate(&c->timers[i].b) == cudaSuccess;
+  if (ok) {
+    // rotary tables: angles in double, rounded to fp32
+    const int half = c->md.hd / 2;
+    std::vector<float> cs((size_t)c->md.max_seq * half), sn((size_t)c->md.max_seq * half);
+    for (int p = 0; p < c->md.max_seq; ++p)
+      for (int k = 0; k < half; ++k) {
+        double ang = (double)p * pow((double)c->md.theta, -2.0 * k / (double)c->md.hd);
+        cs[(size_t)p * half + k] = (float)cos(ang);
+        sn[(size_t)p * half + k] = (float)sin(ang);
+      }
+    ok = cudaMemcpy(c->ws + lay.cos_tab, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess &&
+         cudaMemcpy(c->ws + lay.sin_tab, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
+  }
+  if (!ok) {
+    hsd_destroy(c);
+    return HSD_E_CUDA;
+  }
+  c->stats.assign(n_levels, hsd_level_stats{});
+  *out = c;
+  return HSD_OK;
+}
+
+int hsd_generate(hsd_ctx *c, const int32_t *prompt_ids, int batch, int prompt_len, int n_new, uint64_t seed, void *stream,
+                 int32_t *out_tokens, hsd_level_stats *stats, double *timing_ms) {
+  if (!c || !prompt_ids || !out_tokens || batch < 1 || batch > c->max_batch || prompt_len < 1 || n_new < 1)
+    return HSD_E_INVALID_ARG;
+  int sumT = 0;
+  for (int t : c->T) sumT += t;
+  if ((long long)prompt_len + n_new + sumT + c->n_levels + 1 > c->md.max_seq) return HSD_E_INVALID_ARG;
+  c->stream = (cudaStream_t)stream;
+  c->seed = seed;
+  c->stats.assign(c->n_levels, hsd_level_stats{});
+  c->buf_len.assign(c->max_batch, 0);
+  c->len_g.assign(c->max_batch, std::vector<int>(c->n_levels, 0));
+  c->serial.assign(c->max_batch, std::vector<uint32_t>(c->n_levels, 0));
+  c->n_pages_of.assign(c->max_batch, 0);
+  c->pt_dirty.assign(c->max_batch, 0);
+  c->free_pages.clear();
+  for (int p = c->lay.n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
+  c->trace_records = 0;
+  cudaEvent_t e0 = nullptr, e1 = nullptr, e2 = nullptr;
+  bool ev = cudaEventCreate(&e0) == cudaSuccess && cudaEventCreate(&e1) == cudaSuccess && cudaEventCreate(&e2) == cudaSuccess;
+  int st = HSD_OK;
+  auto body = [&]() -> int {
+    if (ev) cudaEventRecord(e0, c->stream);
+    HSD_CUDA_OK(cudaMemcpy2DAsync(c->dev<int>(c->lay.tokens), (size_t)c->md.max_seq * 4, prompt_ids, (size_t)prompt_len * 4,
+                                  (size_t)prompt_len * 4, batch, cudaMemcpyDeviceToDevice, c->stream));
+    for (int b = 0; b < batch; ++b) c->buf_len[b] = prompt_len;
+    HSD_TRY(prefill(c, batch, prompt_len));
+    if (ev) cudaEventRecord(e1, c->stream);
+    const int K = c->n_levels - 1;
+    for (;;) {
+      std::vector<int> act;
+      for (int b = 0; b < batch; ++b)
+        if (c->buf_len[b] - prompt_len < n_new) act.push_back(b);
+      if (act.empty()) break;
+      HSD_TRY(run_level(c, K, act));
+    }
+    HSD_CUDA_OK(cudaMemcpy2DAsync(out_tokens, (size_t)n_new * 4, c->dev<int>(c->lay.tokens) + prompt_len,
+                                  (size_t)c->md.max_seq * 4, (size_t)n_new * 4, batch, cudaMemcpyDeviceToDevice, c->stream));
+    if (ev) cudaEventRecord(e2, c->stream);
+    return sync_stream(c);
+  };
+  st = body();
+  if (st != HSD_OK) cudaStreamSynchronize(c->stream);
+  if (st == HSD_OK && timing_ms) {
+    float a = 0.f, b = 0.f;
+    if (ev) { cudaEventElapsedTime(&a, e0, e1); cudaEventElapsedTime(&b, e1, e2); }
+    timing_ms[0] = a; timing_ms[1] = b;
+  }
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  if (e2) cudaEventDestroy(e2);
+  if (st == HSD_OK && stats)
+    for (int i = 0; i < c->n_levels; ++i) stats[i] = c->stats[i];
+  if (c->trace) fflush(c->trace);
+  return st;
+}
+
+int hsd_set_trace(hsd_ctx *c, const char *path, int logit_calls) {
+  if (!c) return HSD_E_INVALID_ARG;
+  if (c->trace) { fclose(c->trace); c->trace = nullptr; }
+  if (!path) return HSD_OK;
+  c->trace = fopen(path, "wb");
+  if (!c->trace) return HSD_E_IO;
+  c->trace_logit_calls = logit_calls < 0 ? 0 : logit_calls;
+  c->trace_records = 0;
+  return HSD_OK;
+}
+
+void hsd_destroy(hsd_ctx *c) {
+  if (!c) return;
+  if (c->trace) fclose(c->trace);
+  if (c->ring_host) cudaFreeHost(c->ring_host);
+  if (c->n_acc_host) cudaFreeHost(c->n_acc_host);
+  if (c->page_table_host) cudaFreeHost(c->page_table_host);
+  for (int i = 0; i < kTimerPairs; ++i) {
+    if (c->timers[i].a) cudaEventDestroy(c->timers[i].a);
+    if (c->timers[i].b) cudaEventDestroy(c->timers[i].b);
+  }
+  delete c;
+}
+
+}  // extern "C"

@@ -27,7 +27,7 @@ struct RowBatch {
   const long long *lrow_dst;  // [L] destination row in the level's logits buffer
 };
 
-constexpr int kAttnRows = 16;        // rows of one sequence handled by one attention block
+constexpr int kAttnRows = 8;         // rows of one sequence handled by one attention block
 constexpr int kAttnKeyTile = 32;
 constexpr int kGemmRowTile = 16;     // rows per weight stream in the SIMT GEMM
 

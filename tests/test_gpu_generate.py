@@ -1,0 +1,191 @@
+"""End-to-end parity of hsd_generate with the oracle: token streams, per-level counters, logits."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import philox, sampling
+from oracle.hsd import HSD, SpecDecisions
+from oracle.transformer import Transformer
+from paper_2510_19705_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+STAT_KEYS = ("calls", "drafted", "tested", "accepted", "emitted")
+
+
+def _setup(name, lib, max_batch=1, T=None, exits=None):
+    wl = inputs.WORKLOADS[name]
+    cfg = wl["model"]
+    w_cpu = inputs.make_weights(cfg, wl["weight_seed"])
+    w_gpu = {k: (v.cuda() if k != "layers" else [{n: t.cuda() for n, t in l.items()} for l in v]) for k, v in w_cpu.items()}
+    exits = exits or wl["exits"]
+    T = wl["T"] if T is None else T
+    max_seq = wl["prompt"] + wl["n_new"] + sum(T) + len(exits) + 8
+    eng = lib.Hsd(cfg, w_gpu, exits, T, max_batch=max_batch, max_seq=max_seq, page_size=wl["page"])
+    oracle_model = Transformer(cfg, inputs.weights_to_numpy(w_cpu), exits)
+    prompts = inputs.make_prompts(cfg["vocab"], max_batch, wl["prompt"], wl["prompt_seed"])
+    return wl, cfg, eng, oracle_model, prompts, T
+
+
+def _oracle_run(model, T, prompt, n_new, seed, seq=0):
+    model.reset()
+    run = HSD(model, T, SpecDecisions(seed, seq))
+    toks = run.generate(prompt, n_new)
+    return np.asarray(toks, dtype=np.int32), run
+
+
+def _check_stats(gpu_stats, run):
+    for lvl, st in enumerate(run.stats):
+        for k in STAT_KEYS:
+            assert gpu_stats[lvl][k] == getattr(st, k), (lvl, k, gpu_stats[lvl], st.as_tuple())
+
+
+def test_tiny_fp32_streams_match_oracle_bit_exact(lib):
+    wl, cfg, eng, om, prompts, T = _setup("tiny3", lib)
+    p_gpu = prompts.cuda()
+    for seed in range(4):
+        toks, stats, _ = eng.generate(p_gpu, wl["n_new"], seed)
+        want, run = _oracle_run(om, T, prompts[0].tolist(), wl["n_new"], seed)
+        assert np.array_equal(toks[0].cpu().numpy(), want), seed
+        _check_stats(stats, run)
+        for s in stats[1:]:
+            assert s["calls"] <= s["emitted"] <= s["drafted"] + s["calls"]      # 1 .. t+1 tokens per round
+
+
+def test_tiny_fp32_logits_within_tolerance_and_trace_matches(lib, tmp_path):
+    wl, cfg, eng, om, prompts, T = _setup("tiny3", lib)
+    path = str(tmp_path / "trace.bin")
+    eng.set_trace(path, logit_calls=10 ** 6)
+    toks, stats, _ = eng.generate(prompts.cuda(), 24, 3)
+    eng.set_trace(None)
+    recs = lib.read_trace(path)
+    want, run = _oracle_run(om, T, prompts[0].tolist(), 24, 3)
+    assert np.array_equal(toks[0].cpu().numpy(), want)
+    assert len(recs) == len(run.trace)
+    for rec, orc in zip(recs, run.trace):
+        lvl, serial, ctx_len, t, n, otoks = orc
+        assert (rec["level"], rec["serial"], rec["ctx_len"]) == (lvl, serial, ctx_len)
+        if lvl == 0:
+            assert rec["tokens"].tolist() == list(otoks)
+        else:
+            assert (rec["t"], rec["n"]) == (t, n) and rec["tokens"][-1] == otoks[-1]
+    # logits of every verification against the oracle's own forward (fp32: 1e-5 absolute)
+    om.reset()
+    full = prompts[0].tolist() + want.tolist()
+    worst = 0.0
+    for rec in recs:
+        if rec["level"] == 0:
+            continue
+        drafts = rec["tokens"][:-1].tolist()
+        context = _context_of(recs, rec, prompts[0].tolist())
+        om.rows(rec["level"], context, drafts)
+        worst = max(worst, float(np.abs(om.last_logits64 - rec["logits"]).max()))
+    assert worst < 1e-5, worst
+
+
+def _context_of(recs, rec, prompt):
+    """Rebuild the token buffer at the time of `rec` by replaying the log up to it."""
+    buf = list(prompt)
+    for r in recs:
+        if r is rec:
+            break
+        if r["level"] == 0:
+            buf = buf[:r["ctx_len"]] + r["tokens"].tolist()
+        else:
+            buf = buf[:r["ctx_len"] + r["n"]] + [int(r["tokens"][-1])]
+    return buf if rec is None else buf[:rec["ctx_len"]]
+
+
+def test_degenerate_hierarchies(lib):
+    # one level = ancestral sampling from the target; two levels = single-draft speculative decoding
+    wl, cfg, eng, om, prompts, _ = _setup("tiny3", lib, T=(), exits=(4,))
+    toks, stats, _ = eng.generate(prompts.cuda(), 20, 9)
+    ctx = prompts[0].tolist()
+    om.reset()
+    for i in range(20):
+        row = om.rows(0, ctx, [])[0]
+        tok = sampling.categorical(row, philox.uniform24(9, 0, i, 0, philox.PURPOSE_DRAFT, 0))
+        assert tok == int(toks[0, i])
+        ctx.append(tok)
+    assert stats[0]["emitted"] == 20
+    wl, cfg, eng2, om2, prompts, T2 = _setup("tiny3", lib, T=(4,), exits=(2, 4))
+    toks, stats, _ = eng2.generate(prompts.cuda(), 40, 1)
+    want, run = _oracle_run(om2, T2, prompts[0].tolist(), 40, 1)
+    assert np.array_equal(toks[0].cpu().numpy(), want)
+    _check_stats(stats, run)
+
+
+def test_batch_sequences_equal_their_single_runs(lib):
+    # sequences are independent: sequence b of a batch = the same prompt run alone with the same seed
+    wl, cfg, eng, om, prompts, T = _setup("tiny3", lib, max_batch=3)
+    toks, stats, _ = eng.generate(prompts.cuda(), 32, 5)
+    for b in range(3):
+        want, _ = _oracle_run(om, T, prompts[b].tolist(), 32, 5, seq=b)
+        assert np.array_equal(toks[b].cpu().numpy(), want), b
+
+
+def test_page_size_does_not_change_the_stream(lib):
+    wl = inputs.WORKLOADS["tiny3"]
+    cfg = wl["model"]
+    w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
+    prompts = inputs.make_prompts(cfg["vocab"], 1, wl["prompt"], wl["prompt_seed"]).cuda()
+    outs = []
+    for page in (4, 16, 64):
+        eng = lib.Hsd(cfg, w, wl["exits"], wl["T"], max_batch=1, max_seq=128, page_size=page)
+        outs.append(eng.generate(prompts, 40, 2)[0].cpu())
+        eng.close()
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[1], outs[2])
+
+
+def test_mini_bf16_decisions_follow_the_oracle_on_the_same_logits(lib, tmp_path):
+    """bf16: the two forwards differ by rounding, so the stream is checked call by call: given the
+    library's own stored logits, the oracle's decision arithmetic must reproduce every token and accept
+    count; the logits themselves must match the oracle's forward within 2e-2."""
+    wl, cfg, eng, om, prompts, T = _setup("mini3", lib)
+    path = str(tmp_path / "trace.bin")
+    eng.set_trace(path, logit_calls=10 ** 6)
+    toks, stats, _ = eng.generate(prompts.cuda(), wl["n_new"], 0)
+    eng.set_trace(None)
+    recs = lib.read_trace(path)
+    prompt = prompts[0].tolist()
+    rows_of = {}                   # level -> logits rows of the level's current frame, by buffer position
+    worst = 0.0
+    n_checked = 0
+    for rec in recs:
+        lvl, ctx, serial = rec["level"], rec["ctx_len"], rec["serial"]
+        context = _context_of(recs, rec, prompt)
+        if lvl == 0:
+            buf = list(context)
+            for j, tok in enumerate(rec["tokens"].tolist()):
+                U = philox.uniform24(0, j, serial, 0, philox.PURPOSE_DRAFT, 0)
+                assert sampling.categorical(rec["logits"][j], U) == tok
+                rows_of[(0, len(buf))] = rec["logits"][j]
+                buf.append(tok)
+        else:
+            drafts = rec["tokens"][:-1].tolist()
+            dec = SpecDecisions(0, 0)
+            n = len(drafts)
+            for j, x in enumerate(drafts):
+                if not dec.accept(rec["logits"][j], rows_of[(lvl - 1, ctx + j)], x, j, serial, lvl):
+                    n = j
+                    break
+            assert n == rec["n"]
+            q = rows_of[(lvl - 1, ctx + n)] if n < len(drafts) else None
+            assert dec.final_sample(rec["logits"][n], q, serial, lvl) == int(rec["tokens"][-1])
+            for j in range(n + 1):
+                rows_of[(lvl, ctx + j)] = rec["logits"][j]
+        if n_checked < 40:           # forward parity on the first calls (the oracle is slow)
+            if lvl == 0:
+                for j in range(len(rec["tokens"])):
+                    om.rows(0, context + rec["tokens"][:j].tolist(), [])
+                    worst = max(worst, float(np.abs(om.last_logits64[0] - rec["logits"][j]).max()))
+            else:
+                om.rows(lvl, context, drafts)
+                worst = max(worst, float(np.abs(om.last_logits64 - rec["logits"]).max()))
+            n_checked += 1
+    assert n_checked >= 10 and worst < 2e-2, worst
+    # the emitted stream is what the log says
+    final = _context_of(recs, None, prompt)
+    assert final[len(prompt):len(prompt) + wl["n_new"]] == toks[0].cpu().tolist()
