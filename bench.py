@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Benchmark of the HSD hot path.
+
+Workload: the 8B-shape, 3-level hierarchy at batch 1 (Llama-style 32 layers, d=4096, 32 q / 8 kv heads,
+SwiGLU 14336, vocab 32000, bf16, early exits at layers 4 and 12, prompt 1024, 256 new tokens), random-init
+weights and uniform-random prompts.  A step is one hsd_generate call; `value` is generated tokens per
+second over the generation loop (prompt pass excluded, reported separately), inputs resident in HBM; `e2e`
+times the same call from pinned host memory (prompt upload, prompt pass, generation, token download).
+
+T is chosen as the contract asks: a short calibration run measures the per-level forward costs and
+acceptance rates, then the library's own search minimises the expected latency of Theorem 3.2.
+
+`--impl reference` times the CPU oracle (the only reference implementation there is) on a bounded sample of
+the same workload.  `--workload` selects a smaller shape for development runs.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "hsd_generated_tokens_per_s_b1"
+UNIT = "tokens/s"
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], 0, set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx = max(mx, float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": mx or None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def weight_bytes(cfg, n_layers):
+    es = 2 if cfg["dtype"] == "bf16" else 4
+    d, hd, ff, V = cfg["d_model"], cfg["head_dim"], cfg["d_ff"], cfg["vocab"]
+    per_layer = (cfg["n_q_heads"] * hd * d * 2 + cfg["n_kv_heads"] * hd * d * 2 + 3 * ff * d + 2 * d) * es
+    return n_layers * per_layer + (V * d + d) * es
+
+
+def pass_bytes(cfg, n_layers, ctx, rows, logit_rows):
+    """Algorithmic bytes of one level forward: weights once, KV read for the context, KV write and
+    embedding rows for the processed rows, logits written."""
+    es = 2 if cfg["dtype"] == "bf16" else 4
+    kv = 2 * cfg["n_kv_heads"] * cfg["head_dim"] * es
+    return (weight_bytes(cfg, n_layers) + n_layers * kv * (ctx + rows) + rows * cfg["d_model"] * es
+            + logit_rows * cfg["vocab"] * es)
+
+
+def to_cuda(w):
+    return {k: (v.cuda() if k != "layers" else [{n: t.cuda() for n, t in l.items()} for l in v]) for k, v in w.items()}
+
+
+def choose_T(binding, cfg, weights, wl, prompts, n_calib=64):
+    """Calibration run with T = (2, ..., 2), then the Theorem 3.2 search (monotone T, T_max 15)."""
+    exits = wl["exits"]
+    K = len(exits) - 1
+    T0 = [2] * K
+    eng = binding.Hsd(cfg, weights, exits, T0, max_batch=1, max_seq=wl["prompt"] + n_calib + 64, page_size=wl["page"])
+    eng.generate(prompts, 8, 12345)                      # warm-up
+    _, stats, _ = eng.generate(prompts, n_calib, 12345)
+    eng.close()
+    costs = [s["ms"] / max(1, s["forwards"]) for s in stats]
+    alphas = [min(0.999, max(0.001, stats[i]["accepted"] / max(1, stats[i]["tested"]))) for i in range(1, K + 1)]
+    T, lat = binding.hsd_search_T(costs, alphas, 15, True)
+    return list(T), costs, alphas, lat
+
+
+def run_ours(args):
+    from paper_2510_19705_b200 import binding, inputs
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    wl = inputs.WORKLOADS[args.workload]
+    cfg = wl["model"]
+    n_new, P = (args.n_new or wl["n_new"]), wl["prompt"]
+    # replicas only: each rank runs its own independent sequence (no data-path collective)
+    weights = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
+    prompts_host = inputs.make_prompts(cfg["vocab"], 1, P, wl["prompt_seed"] + rank).pin_memory()
+    prompts = prompts_host.cuda()
+    if wl["T"] is None:
+        T, costs, alphas, lat = choose_T(binding, cfg, weights, wl, prompts)
+        calib = {"costs_ms": [round(c, 4) for c in costs], "alphas": [round(a, 4) for a in alphas],
+                 "expected_ms_per_token": round(lat, 4)}
+    else:
+        T, calib = list(wl["T"]), None
+    eng = binding.Hsd(cfg, weights, wl["exits"], T, max_batch=1, max_seq=P + n_new + sum(T) + 16, page_size=wl["page"])
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            torch.distributed.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        eng.generate(prompts, n_new, 1000 + i)
+    barrier()
+    launches0 = binding.hsd_kernel_launches()
+    dec_ms = pre_ms = 0.0
+    agg = None
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local) as clk:
+        ev0.record()
+        for i in range(args.steps):
+            _, stats, (t_pre, t_dec) = eng.generate(prompts, n_new, i)
+            dec_ms += t_dec
+            pre_ms += t_pre
+            agg = stats if agg is None else [{k: a[k] + b[k] for k in a} for a, b in zip(agg, stats)]
+        ev1.record()
+        barrier()
+    launches = binding.hsd_kernel_launches() - launches0
+    step_ms = ev0.elapsed_time(ev1) / args.steps
+    # end to end through the public call, host buffers: prompt upload + prompt pass + generation + download
+    out_host = torch.empty(1, n_new, dtype=torch.int32).pin_memory()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e2e_steps = max(1, min(args.steps, 3))
+    for i in range(e2e_steps):
+        d_prompt = prompts_host.cuda(non_blocking=True)
+        toks, _, _ = eng.generate(d_prompt, n_new, i)
+        out_host.copy_(toks, non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    t = torch.tensor([dec_ms / args.steps, step_ms, e2e_s * 1e3, pre_ms / args.steps], device="cuda", dtype=torch.float64)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    dec_ms_step, step_ms, e2e_ms, pre_ms_step = t.tolist()
+    if rank != 0:
+        return
+    hbm_peak, peak_kind = peaks()
+    K = len(wl["exits"]) - 1
+    # dominant unit: the target level's verification forward (one pass streams every weight once)
+    tgt = agg[K]
+    tgt_ms = tgt["ms"] / max(1, tgt["forwards"])
+    mean_rows = tgt["rows"] / max(1, tgt["forwards"])
+    mean_ctx = P + n_new / 2.0
+    levels = []
+    for i, s in enumerate(agg):
+        ms = s["ms"] / max(1, s["forwards"])
+        rows = s["rows"] / max(1, s["forwards"])
+        b = pass_bytes(cfg, wl["exits"][i], mean_ctx, rows, rows if i == 0 else (s["drafted"] / max(1, s["calls"]) + 1))
+        levels.append({"level": i, "layers": wl["exits"][i], "forwards": s["forwards"], "ms_per_forward": round(ms, 4),
+                       "rows_per_forward": round(rows, 2), "gbs": round(b / ms / 1e6, 1) if ms > 0 else None,
+                       "accept_rate": round(s["accepted"] / s["tested"], 4) if s["tested"] else None})
+    tgt_bytes = pass_bytes(cfg, wl["exits"][K], mean_ctx, mean_rows, tgt["drafted"] / max(1, tgt["calls"]) + 1)
+    achieved = tgt_bytes / tgt_ms / 1e6 if tgt_ms > 0 else 0.0
+    line = {
+        "metric": METRIC, "value": round(world * n_new / (dec_ms_step / 1e3), 2), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dec_ms_step, 3), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
+        "config": {"workload": args.workload, "batch": 1, "prompt_len": P, "n_new": n_new, "exits": list(wl["exits"]),
+                   "T": T, "T_search": calib, "l2": "inputs larger than L2 (weights %.1f GB per target pass)"
+                   % (weight_bytes(cfg, cfg["n_layers"]) / 1e9), "replicas": "independent sequence per GPU"},
+        "prefill_ms": round(pre_ms_step, 3), "step_ms_with_prefill": round(step_ms, 3),
+        "e2e": {"value": round(world * n_new / (e2e_ms / 1e3), 2), "unit": UNIT, "h2d_bytes_per_step": P * 4,
+                "d2h_bytes_per_step": n_new * 4},
+        "gpu_launches": int(launches),
+        "clocks": clk.summary(),
+        "roofline": {"bound": "hbm", "kernel": "target-level verification forward (all kernels of one pass)",
+                     "achieved": round(achieved, 1), "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": round(achieved / hbm_peak, 4), "frac_of_8000": round(achieved / 8000.0, 4),
+                     "traffic": None, "ms_per_launch": round(tgt_ms, 4), "bytes_per_launch": int(tgt_bytes)},
+        "levels": levels,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        line["cpu_baseline"] = cpu_baseline(args.workload, T, weights)
+    print(json.dumps(line))
+
+
+def cpu_baseline(workload, T, weights=None, rounds=1, prompt_len=8):
+    """The oracle, as it stands, on a bounded sample: `rounds` top-level HSD rounds of the same model
+    after a short prompt."""
+    from paper_2510_19705_b200 import inputs
+    from oracle.hsd import HSD, SpecDecisions
+    from oracle.transformer import Transformer
+    wl = inputs.WORKLOADS[workload]
+    cfg = wl["model"]
+    if weights is None:
+        weights = inputs.make_weights(cfg, wl["weight_seed"], device="cuda" if torch.cuda.is_available() else "cpu")
+    w_np = inputs.weights_to_numpy(weights)
+    model = Transformer(cfg, w_np, wl["exits"])
+    prompt = inputs.make_prompts(cfg["vocab"], 1, prompt_len, wl["prompt_seed"])[0].tolist()
+    run = HSD(model, T, SpecDecisions(0))
+    t0 = time.perf_counter()
+    n = 0
+    out = []
+    for _ in range(rounds):
+        toks, _ = run.hsd(run.K, prompt + out)
+        out += toks
+        n += len(toks)
+    dt = time.perf_counter() - t0
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except AttributeError:
+        cores = os.cpu_count()
+    return {"value": round(n / dt, 4), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": "%d top-level HSD round(s) (%d tokens, %.1f s) of the %s model after a %d-token prompt, T=%s"
+                      % (rounds, n, dt, workload, prompt_len, list(T))}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2510_19705_b200 import inputs
+    wl = inputs.WORKLOADS[args.workload]
+    T = list(wl["T"]) if wl["T"] is not None else [2] * (len(wl["exits"]) - 1)
+    weights = inputs.make_weights(wl["model"], wl["weight_seed"], device="cuda" if torch.cuda.is_available() else "cpu")
+    vals = []
+    steps = max(1, min(args.steps, 2))
+    for i in range(min(args.warmup, 1) + steps):
+        cb = cpu_baseline(args.workload, T, weights)
+        vals.append(cb)
+    vals = vals[-steps:]
+    v = sum(c["value"] for c in vals) / len(vals)
+    cb = dict(vals[-1], value=round(v, 4))
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": round(v, 4), "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": None, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "batch": 1, "T": T, "note": "CPU oracle on a bounded sample of the workload"},
+        "cpu_baseline": cb, "e2e": {"value": round(v, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8b3")
+    ap.add_argument("--n-new", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -152,6 +152,39 @@ int hsd_set_trace(hsd_ctx *ctx, const char *path, int logit_calls);
 
 void hsd_destroy(hsd_ctx *ctx);
 
+/* ---------------------------------------------------------------------------------------
+ * Expected latency per token of the chain M_0..M_K (Theorem 3.2):
+ *   cost(0) = T_0 c_0;  cost(k) = gamma(alpha_{k-1,k}, T_{k-1}, T_k) (cost(k-1) + c_k), 0 < k < K;
+ *   L = (1 - a) / (1 - a^(T_{K-1}+1)) (cost(K-1) + c_K), a = alpha_{K-1,K}.
+ * gamma = expected draft/verify rounds until T_k tokens are collected under IID acceptance (the
+ * paper estimates it empirically; this is a renewal computation over the per-round yield).
+ *   costs host [n_levels], alphas host [n_levels-1] (alphas[i] = rate level i -> i+1), T host [n_levels-1].
+ * hsd_search_T minimises L over T in [1, T_max]^(n_levels-1); monotone != 0 keeps the search
+ * graph's constraint T_k >= T_{k-1} (Section 4.2, edge list).  Ties keep the lexicographically
+ * first T.  Host-only; Errors: INVALID_ARG. */
+int hsd_expected_latency(const double *costs, const double *alphas, int n_levels, const int32_t *T, double *out);
+int hsd_search_T(const double *costs, const double *alphas, int n_levels, int T_max, int monotone, int32_t *out_T,
+                 double *out_latency);
+
+/* ---------------------------------------------------------------------------------------
+ * One weight-streaming matrix product of the verifier forward in isolation (the contraction
+ * behind every projection of Algorithm 2's multi-row forward pass): out[r, n] = sum_k A[r, k] W[n, k],
+ * bf16 inputs, fp32 accumulation on the tensor cores, fp32 output.
+ *   A    device bf16 [R, K] row-major, 1 <= R <= 128, K a multiple of 64
+ *   W    device bf16 [N, K] row-major
+ *   out  device fp32 [R, N]
+ *   workspace  device, 256-byte aligned, >= hsd_gemm_workspace_bytes(R, N, K); ignored on entry
+ * Errors: INVALID_ARG, WORKSPACE_TOO_SMALL, UNSUPPORTED (no tensor-map support), CUDA,
+ * DEVICE_TIMEOUT is reported by hsd_gemm_status after synchronising. */
+size_t hsd_gemm_workspace_bytes(int R, int N, int K);
+int hsd_gemm_bf16(const void *A, int R, int K, const void *W, int N, float *out, void *workspace, size_t workspace_bytes,
+                  void *stream);
+/* Synchronises `stream` and returns DEVICE_TIMEOUT if a kernel using `workspace` gave up a bounded wait. */
+int hsd_gemm_status(void *workspace, void *stream);
+
+/* Number of CUDA kernels this library has launched in the calling process so far. */
+uint64_t hsd_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -138,6 +138,20 @@ def _declare_engine(lib):
     lib.hsd_set_trace.argtypes = [vp, c.c_char_p, i32]
     lib.hsd_destroy.restype = None
     lib.hsd_destroy.argtypes = [vp]
+    lib.hsd_expected_latency.restype = i32
+    lib.hsd_expected_latency.argtypes = [c.POINTER(c.c_double), c.POINTER(c.c_double), i32, c.POINTER(c.c_int32),
+                                         c.POINTER(c.c_double)]
+    lib.hsd_search_T.restype = i32
+    lib.hsd_search_T.argtypes = [c.POINTER(c.c_double), c.POINTER(c.c_double), i32, i32, i32, c.POINTER(c.c_int32),
+                                 c.POINTER(c.c_double)]
+    lib.hsd_kernel_launches.restype = c.c_uint64
+    lib.hsd_kernel_launches.argtypes = []
+    lib.hsd_gemm_workspace_bytes.restype = sz
+    lib.hsd_gemm_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.hsd_gemm_bf16.restype = i32
+    lib.hsd_gemm_bf16.argtypes = [vp, i32, i32, vp, i32, vp, vp, sz, vp]
+    lib.hsd_gemm_status.restype = i32
+    lib.hsd_gemm_status.argtypes = [vp, vp]
 
 
 class Hsd:
@@ -226,3 +240,59 @@ def read_trace(path):
             recs.append(dict(level=level, seq=seq, serial=serial, ctx_len=ctx_len, t=t, n=n, rows=rows,
                              tokens=toks, logits=logits))
     return recs
+
+
+def hsd_expected_latency(costs, alphas, T):
+    """Theorem 3.2 for the chain with costs c_0..c_K, alphas[i] = rate level i -> i+1, parameters T."""
+    lib = library()
+    _declare_engine(lib)
+    n = len(costs)
+    out = ctypes.c_double()
+    _check(lib.hsd_expected_latency((ctypes.c_double * n)(*costs), (ctypes.c_double * max(1, n - 1))(*(alphas or [0])), n,
+                                    (ctypes.c_int32 * max(1, n - 1))(*(T or [1])), ctypes.byref(out)))
+    return out.value
+
+
+def hsd_search_T(costs, alphas, T_max=15, monotone=True):
+    """argmin over T in [1, T_max]^K of the expected latency -> (T tuple, latency)."""
+    lib = library()
+    _declare_engine(lib)
+    n = len(costs)
+    out_T = (ctypes.c_int32 * max(1, n - 1))()
+    out = ctypes.c_double()
+    _check(lib.hsd_search_T((ctypes.c_double * n)(*costs), (ctypes.c_double * max(1, n - 1))(*(alphas or [0])), n, T_max,
+                            1 if monotone else 0, out_T, ctypes.byref(out)))
+    return tuple(out_T[i] for i in range(n - 1)), out.value
+
+
+def hsd_kernel_launches():
+    lib = library()
+    _declare_engine(lib)
+    return int(lib.hsd_kernel_launches())
+
+
+def hsd_gemm_workspace_bytes(R, N, K):
+    lib = library()
+    _declare_engine(lib)
+    return int(lib.hsd_gemm_workspace_bytes(R, N, K))
+
+
+def hsd_gemm_bf16(A, W, out=None, workspace=None, check=True):
+    """A bf16 [R, K], W bf16 [N, K] (CUDA) -> fp32 [R, N] = A @ W^T on the tensor cores."""
+    lib = library()
+    _declare_engine(lib)
+    R, K = A.shape
+    N = W.shape[0]
+    need = hsd_gemm_workspace_bytes(R, N, K)
+    if need == 0:
+        raise HsdError("hsd_gemm_bf16: unsupported shape R=%d N=%d K=%d" % (R, N, K))
+    if workspace is None:
+        workspace = torch.empty(need + 256, dtype=torch.uint8, device=A.device)
+    base = (workspace.data_ptr() + 255) // 256 * 256
+    if out is None:
+        out = torch.empty(R, N, dtype=torch.float32, device=A.device)
+    _check(lib.hsd_gemm_bf16(_dev(A), R, K, _dev(W), N, _dev(out), ctypes.c_void_p(base),
+                             workspace.numel() - (base - workspace.data_ptr()), _stream()))
+    if check:
+        _check(lib.hsd_gemm_status(ctypes.c_void_p(base), _stream()))
+    return out

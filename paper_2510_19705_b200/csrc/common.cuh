@@ -14,6 +14,10 @@ typedef unsigned int u32;
     if (e__ != cudaSuccess) return HSD_E_CUDA;    \
   } while (0)
 
+// Kernel launches issued by this library (reported by hsd_kernel_launches()).
+extern unsigned long long g_hsd_launches;
+static inline void hsd_count_launches(int n) { g_hsd_launches += (unsigned long long)n; }
+
 static inline int hsd_launch_status() {
   return cudaGetLastError() == cudaSuccess ? HSD_OK : HSD_E_CUDA;
 }

@@ -8,6 +8,7 @@
 #include <vector>
 
 #include "forward.cuh"
+#include "gemm_tc.cuh"
 #include "sampling_api.cuh"
 
 using namespace hsd;
@@ -21,13 +22,22 @@ constexpr int kMaxSplits = 64;
 constexpr int kPrefillRows = 128;
 constexpr uint32_t kTraceMagic = 0x48534454u;
 
+constexpr size_t kTcCtrlBytes = 16384 + 256;    // status word (first 256 bytes) + per-tile counters
+
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+int device_sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+      sms < 1)
+    return 148;
+  return sms;
+}
 size_t elem_size(int dtype) { return dtype == HSD_BF16 ? 2 : 4; }
 
 // Workspace layout, shared by hsd_workspace_bytes and hsd_create.
 struct Layout {
   size_t tokens, cos_tab, sin_tab, page_table, k_pool, v_pool, pool_layer_stride, x, h, qkv, q, att, act, partials, hf,
-      vscratch, n_acc, ring, total;
+      vscratch, n_acc, ring, tc_scratch, tc_pieces_bytes, total;
   std::vector<size_t> logits;
   std::vector<int> slots;
   int max_rows, pages_per_seq, n_pages, partial_rows;
@@ -98,6 +108,23 @@ Layout make_layout(const hsd_model_desc *m, int n_levels, const int32_t *T) {
   L.n_acc = take((size_t)B * 4);
   L.ring_slot = align_up((size_t)L.max_rows * 40 + (size_t)B * 96 + 1024, 256);
   L.ring = take(L.ring_slot * kRingSlots);
+  // tensor-core GEMM scratch: [status word | per-tile counters (16 KiB)] + split pieces (largest plan)
+  L.tc_pieces_bytes = 0;
+  if (m->dtype == HSD_BF16) {
+    const int sms = device_sm_count();
+    const int npads[4] = {16, 32, 64, 128};
+    const int shapes[5][4] = {{nq * hd, nkv * hd, nkv * hd, d}, {d, 0, 0, nq * hd}, {m->d_ff, m->d_ff, 0, d},
+                              {d, 0, 0, m->d_ff}, {m->vocab, 0, 0, d}};
+    const int modes[5] = {GEMM_STORE_F32, GEMM_ADD_F32, GEMM_SWIGLU_T, GEMM_ADD_F32, GEMM_STORE_T_SCATTER};
+    for (int g = 0; g < 5; ++g)
+      for (int np : npads) {
+        if (shapes[g][3] % kTcBlockK) continue;
+        int nsegs = shapes[g][2] ? 3 : (shapes[g][1] ? 2 : 1);
+        TcGemmPlan pl = tc_plan(shapes[g], nsegs, modes[g], shapes[g][3], np, sms);
+        L.tc_pieces_bytes = std::max(L.tc_pieces_bytes, pl.scratch_bytes);
+      }
+  }
+  L.tc_scratch = take(kTcCtrlBytes + L.tc_pieces_bytes);
   L.total = off;
   return L;
 }
@@ -142,6 +169,12 @@ struct hsd_ctx {
   int trace_logit_calls, trace_records;
   cudaStream_t stream;
   uint64_t seed;
+  // tensor-core GEMM state (bf16 models)
+  bool use_tc;
+  int sm_count;
+  std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + 1]: wq wk wv wo wg wu wd per layer, then lm_head
+  CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
+  int *status_host;
 
   template <typename U> U *dev(size_t off) const { return reinterpret_cast<U *>(ws + off); }
 };
@@ -149,7 +182,11 @@ struct hsd_ctx {
 namespace {
 
 int sync_stream(hsd_ctx *c) {
+  if (c->use_tc &&
+      cudaMemcpyAsync(c->status_host, c->ws + c->lay.tc_scratch, 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
+    return HSD_E_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return HSD_E_CUDA;
+  if (c->use_tc && *c->status_host != 0) return HSD_E_DEVICE_TIMEOUT;
   c->ring_in_flight = 0;
   for (int i = 0; i < c->timers_used; ++i) {
     float ms = 0.f;
@@ -204,6 +241,40 @@ int upload_page_tables(hsd_ctx *c) {
     HSD_CUDA_OK(cudaMemcpyAsync(c->dev<int>(c->lay.page_table) + off, c->page_table_host + off,
                                 (size_t)c->n_pages_of[b] * 4, cudaMemcpyHostToDevice, c->stream));
     c->pt_dirty[b] = 0;
+  }
+  return HSD_OK;
+}
+
+// Matrix product of the forward pass: tensor cores for bf16 models, CUDA cores otherwise.
+// abuf names the activation buffer A lives in (0 = h, 1 = att, 2 = act, 3 = hf); wmap0 the index of
+// the first segment's tensor map.
+int gemm(hsd_ctx *c, int abuf, const void *A, int R, int K, const GemmSegs &segs, int wmap0, int mode, float *out_f32,
+         void *out_t, const long long *dst) {
+  if (!c->use_tc) return launch_gemm_simt(c->md, A, R, K, segs, mode, out_f32, out_t, dst, c->stream);
+  TcGemmArgs a;
+  int total = 0;
+  for (int i = 0; i < 3; ++i) {
+    a.seg_n[i] = i < segs.count ? segs.n[i] : 0;
+    if (i < segs.count) a.w[i] = c->wmaps[wmap0 + i];
+    total += a.seg_n[i];
+  }
+  a.n_segs = segs.count;
+  a.K = K;
+  a.mode = mode;
+  a.out_f32 = out_f32;
+  a.out_bf16 = (__nv_bfloat16 *)out_t;
+  a.dst = dst;
+  a.ldo = (mode == GEMM_SWIGLU_T) ? segs.n[0] : total;
+  a.status = (int *)(c->ws + c->lay.tc_scratch);
+  a.counters = (int *)(c->ws + c->lay.tc_scratch + 256);
+  a.pieces = (float *)(c->ws + c->lay.tc_scratch + kTcCtrlBytes);
+  for (int r0 = 0; r0 < R; r0 += 128) {
+    a.R = std::min(128, R - r0);
+    a.row0 = r0;
+    int np = tc_npad(a.R);
+    a.a = c->amaps[abuf][np == 16 ? 0 : np == 32 ? 1 : np == 64 ? 2 : 3];
+    int st = launch_gemm_tc(a, c->sm_count, c->stream);
+    if (st) return st;
   }
   return HSD_OK;
 }
@@ -295,23 +366,23 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     void *kp = c->ws + L.k_pool + L.pool_layer_stride * l, *vp = c->ws + L.v_pool + L.pool_layer_stride * l;
     HSD_TRY(launch_rmsnorm(md, x, w[0], nullptr, R, h, s));
     GemmSegs qkv_segs = {{w[1], w[2], w[3]}, {md.nq * md.hd, md.nkv * md.hd, md.nkv * md.hd}, 3};
-    HSD_TRY(launch_gemm_simt(md, h, R, md.d, qkv_segs, GEMM_STORE_F32, qkv, nullptr, nullptr, s));
+    HSD_TRY(gemm(c, 0, h, R, md.d, qkv_segs, l * 7 + 0, GEMM_STORE_F32, qkv, nullptr, nullptr));
     HSD_TRY(launch_rope_kv(md, qkv, rb, c->dev<float>(L.cos_tab), c->dev<float>(L.sin_tab), pt, kp, vp, q, s));
     HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(L.partials), keys_per_split, n_splits, att, s));
     GemmSegs o_segs = {{w[4], nullptr, nullptr}, {md.d, 0, 0}, 1};
-    HSD_TRY(launch_gemm_simt(md, att, R, md.nq * md.hd, o_segs, GEMM_ADD_F32, x, nullptr, nullptr, s));
+    HSD_TRY(gemm(c, 1, att, R, md.nq * md.hd, o_segs, l * 7 + 3, GEMM_ADD_F32, x, nullptr, nullptr));
     HSD_TRY(launch_rmsnorm(md, x, w[5], nullptr, R, h, s));
     GemmSegs gu_segs = {{w[6], w[7], nullptr}, {md.ff, md.ff, 0}, 2};
-    HSD_TRY(launch_gemm_simt(md, h, R, md.d, gu_segs, GEMM_SWIGLU_T, nullptr, act, nullptr, s));
+    HSD_TRY(gemm(c, 0, h, R, md.d, gu_segs, l * 7 + 4, GEMM_SWIGLU_T, nullptr, act, nullptr));
     GemmSegs d_segs = {{w[8], nullptr, nullptr}, {md.d, 0, 0}, 1};
-    HSD_TRY(launch_gemm_simt(md, act, R, md.ff, d_segs, GEMM_ADD_F32, x, nullptr, nullptr, s));
+    HSD_TRY(gemm(c, 2, act, R, md.ff, d_segs, l * 7 + 6, GEMM_ADD_F32, x, nullptr, nullptr));
   }
   if (n_logit > 0) {
     void *hf = c->dev<void>(L.hf);
     HSD_TRY(launch_rmsnorm(md, x, c->final_norm, rb.lrow_src, n_logit, hf, s));
     GemmSegs lm_segs = {{c->lm_head, nullptr, nullptr}, {md.V, 0, 0}, 1};
-    HSD_TRY(launch_gemm_simt(md, hf, n_logit, md.d, lm_segs, GEMM_STORE_T_SCATTER, nullptr, c->ws + L.logits[level],
-                             rb.lrow_dst, s));
+    HSD_TRY(gemm(c, 3, hf, n_logit, md.d, lm_segs, md.n_layers * 7, GEMM_STORE_T_SCATTER, nullptr, c->ws + L.logits[level],
+                 rb.lrow_dst));
   }
   if (tp) cudaEventRecord(tp->b, s);
   c->stats[level].forwards++;
@@ -541,7 +612,8 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
   c->ws = (char *)workspace;
   c->embed = model->embed; c->final_norm = model->final_norm; c->lm_head = model->lm_head;
   c->lw.assign(model->layer_weights, model->layer_weights + (size_t)model->n_layers * 9);
-  c->ring_host = nullptr; c->n_acc_host = nullptr; c->page_table_host = nullptr;
+  c->ring_host = nullptr; c->n_acc_host = nullptr; c->page_table_host = nullptr; c->status_host = nullptr;
+  c->use_tc = false; c->sm_count = 148;
   c->trace = nullptr; c->trace_logit_calls = 0; c->trace_records = 0;
   c->ring_next = 0; c->ring_in_flight = 0; c->timers_used = 0; c->timers_ok = true; c->stream = nullptr; c->seed = 0;
   bool ok = cudaMallocHost(&c->ring_host, lay.ring_slot * kRingSlots) == cudaSuccess &&
@@ -568,6 +640,37 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
     return HSD_E_CUDA;
   }
   c->stats.assign(n_levels, hsd_level_stats{});
+  // tensor-core path: bf16 model whose contraction sizes are multiples of the 64-element k-block
+  c->sm_count = device_sm_count();
+  c->use_tc = model->dtype == HSD_BF16 && model->d_model % kTcBlockK == 0 && model->d_ff % kTcBlockK == 0 &&
+              (model->n_q_heads * model->head_dim) % kTcBlockK == 0 && tc_init() == HSD_OK;
+  if (c->use_tc) {
+    const ModelDims &md = c->md;
+    int st = HSD_OK;
+    c->wmaps.resize((size_t)md.n_layers * 7 + 1);
+    const long long rows7[7] = {(long long)md.nq * md.hd, (long long)md.nkv * md.hd, (long long)md.nkv * md.hd, md.d, md.ff, md.ff, md.d};
+    const long long cols7[7] = {md.d, md.d, md.d, (long long)md.nq * md.hd, md.d, md.d, md.ff};
+    const int widx[7] = {1, 2, 3, 4, 6, 7, 8};
+    for (int l = 0; l < md.n_layers && !st; ++l)
+      for (int k = 0; k < 7 && !st; ++k)
+        st = tc_make_map(&c->wmaps[(size_t)l * 7 + k], c->lw[(size_t)l * 9 + widx[k]], rows7[k], cols7[k], kTcBoxRows);
+    if (!st) st = tc_make_map(&c->wmaps[(size_t)md.n_layers * 7], c->lm_head, md.V, md.d, kTcBoxRows);
+    const size_t abuf_off[4] = {lay.h, lay.att, lay.act, lay.hf};
+    const long long acols[4] = {md.d, (long long)md.nq * md.hd, md.ff, md.d};
+    int max_logit_rows = 0;
+    for (int i = 0; i < n_levels; ++i) max_logit_rows = std::max(max_logit_rows, c->max_batch * lay.slots[i]);
+    const long long arows[4] = {lay.max_rows, lay.max_rows, lay.max_rows, max_logit_rows};
+    const int npads[4] = {16, 32, 64, 128};
+    for (int b = 0; b < 4 && !st; ++b)
+      for (int p = 0; p < 4 && !st; ++p) st = tc_make_map(&c->amaps[b][p], c->ws + abuf_off[b], arows[b], acols[b], npads[p]);
+    if (!st && cudaMemset(c->ws + lay.tc_scratch, 0, kTcCtrlBytes) != cudaSuccess) st = HSD_E_CUDA;
+    if (!st && cudaMallocHost(&c->status_host, 4) != cudaSuccess) st = HSD_E_CUDA;
+    if (st) {
+      hsd_destroy(c);
+      return st;
+    }
+    *c->status_host = 0;
+  }
   *out = c;
   return HSD_OK;
 }
@@ -599,6 +702,8 @@ int hsd_generate(hsd_ctx *c, const int32_t *prompt_ids, int batch, int prompt_le
                                   (size_t)prompt_len * 4, batch, cudaMemcpyDeviceToDevice, c->stream));
     for (int b = 0; b < batch; ++b) c->buf_len[b] = prompt_len;
     HSD_TRY(prefill(c, batch, prompt_len));
+    HSD_TRY(sync_stream(c));
+    c->stats.assign(c->n_levels, hsd_level_stats{});      // level counters cover the generation loop only
     if (ev) cudaEventRecord(e1, c->stream);
     const int K = c->n_levels - 1;
     for (;;) {
@@ -640,12 +745,49 @@ int hsd_set_trace(hsd_ctx *c, const char *path, int logit_calls) {
   return HSD_OK;
 }
 
+size_t hsd_gemm_workspace_bytes(int R, int N, int K) {
+  if (R < 1 || R > 128 || N < 1 || K < kTcBlockK || K % kTcBlockK) return 0;
+  int seg[3] = {N, 0, 0};
+  return kTcCtrlBytes + tc_plan(seg, 1, GEMM_STORE_F32, K, tc_npad(R), device_sm_count()).scratch_bytes;
+}
+
+int hsd_gemm_bf16(const void *A, int R, int K, const void *W, int N, float *out, void *workspace, size_t workspace_bytes,
+                  void *stream) {
+  if (!A || !W || !out || !workspace || ((uintptr_t)workspace & 255)) return HSD_E_INVALID_ARG;
+  size_t need = hsd_gemm_workspace_bytes(R, N, K);
+  if (need == 0) return HSD_E_INVALID_ARG;
+  if (workspace_bytes < need) return HSD_E_WORKSPACE_TOO_SMALL;
+  int st = tc_init();
+  if (st) return st;
+  TcGemmArgs a;
+  st = tc_make_map(&a.w[0], W, N, K, kTcBoxRows);
+  if (!st) st = tc_make_map(&a.a, A, R, K, tc_npad(R));
+  if (st) return st;
+  a.seg_n[0] = N; a.seg_n[1] = a.seg_n[2] = 0; a.n_segs = 1;
+  a.K = K; a.R = R; a.row0 = 0; a.mode = GEMM_STORE_F32;
+  a.out_f32 = out; a.out_bf16 = nullptr; a.dst = nullptr; a.ldo = N;
+  a.status = (int *)workspace;
+  a.counters = (int *)((char *)workspace + 256);
+  a.pieces = (float *)((char *)workspace + kTcCtrlBytes);
+  HSD_CUDA_OK(cudaMemsetAsync(workspace, 0, kTcCtrlBytes, (cudaStream_t)stream));
+  return launch_gemm_tc(a, device_sm_count(), (cudaStream_t)stream);
+}
+
+int hsd_gemm_status(void *workspace, void *stream) {
+  if (!workspace) return HSD_E_INVALID_ARG;
+  int flag = 0;
+  if (cudaMemcpyAsync(&flag, workspace, 4, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess) return HSD_E_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return HSD_E_CUDA;
+  return flag ? HSD_E_DEVICE_TIMEOUT : HSD_OK;
+}
+
 void hsd_destroy(hsd_ctx *c) {
   if (!c) return;
   if (c->trace) fclose(c->trace);
   if (c->ring_host) cudaFreeHost(c->ring_host);
   if (c->n_acc_host) cudaFreeHost(c->n_acc_host);
   if (c->page_table_host) cudaFreeHost(c->page_table_host);
+  if (c->status_host) cudaFreeHost(c->status_host);
   for (int i = 0; i < kTimerPairs; ++i) {
     if (c->timers[i].a) cudaEventDestroy(c->timers[i].a);
     if (c->timers[i].b) cudaEventDestroy(c->timers[i].b);

@@ -159,8 +159,10 @@ static void gemm_simt_launch(const T *A, int R, int K, const GemmSegs &segs, flo
                              int n_total, cudaStream_t s) {
   constexpr int CPW = 2;
   int grid = ceil_div(n_total, kGemmWarps * CPW);
-  for (int r0 = 0; r0 < R; r0 += RT)
+  for (int r0 = 0; r0 < R; r0 += RT) {
     gemm_simt_kernel<T, RT, CPW, MODE><<<grid, kGemmWarps * 32, 0, s>>>(A, R, r0, K, segs, out_f32, out_t, dst, n_total);
+    hsd_count_launches(1);
+  }
 }
 
 template <typename T, int MODE>
@@ -365,6 +367,7 @@ static int attention_t(const ModelDims &md, const void *q, const RowBatch &rb, c
                                                            md.pages_per_seq, keys_per_split, n_splits, rsqrtf((float)HD));
   if (cudaGetLastError() != cudaSuccess) return HSD_E_CUDA;
   attn_combine_kernel<T, HD><<<rb.R * md.nq, HD, 0, s>>>(partials, rb.row_pos, md.nq, keys_per_split, n_splits, (T *)att_out);
+  hsd_count_launches(2);
   return hsd_launch_status();
 }
 
@@ -375,6 +378,7 @@ int launch_embed(const ModelDims &md, const void *embed, const int *tokens, cons
     embed_kernel<__nv_bfloat16><<<rb.R, 256, 0, s>>>((const __nv_bfloat16 *)embed, tokens, rb.row_seq, rb.row_pos, md.d, md.max_seq, x);
   else
     embed_kernel<float><<<rb.R, 256, 0, s>>>((const float *)embed, tokens, rb.row_seq, rb.row_pos, md.d, md.max_seq, x);
+  hsd_count_launches(1);
   return hsd_launch_status();
 }
 
@@ -384,6 +388,7 @@ int launch_rmsnorm(const ModelDims &md, const float *x, const void *gain, const 
     rmsnorm_kernel<__nv_bfloat16><<<rows, 256, 0, s>>>(x, (const __nv_bfloat16 *)gain, src, md.d, md.eps, (__nv_bfloat16 *)out);
   else
     rmsnorm_kernel<float><<<rows, 256, 0, s>>>(x, (const float *)gain, src, md.d, md.eps, (float *)out);
+  hsd_count_launches(1);
   return hsd_launch_status();
 }
 
@@ -406,6 +411,7 @@ int launch_rope_kv(const ModelDims &md, const float *qkv, const RowBatch &rb, co
   else
     rope_kv_kernel<float><<<grid, threads, 0, s>>>(qkv, rb.row_seq, rb.row_pos, cos_tab, sin_tab, page_table, (float *)k_pool,
                                                   (float *)v_pool, (float *)q_out, md.nq, md.nkv, md.hd, md.page, md.pages_per_seq);
+  hsd_count_launches(1);
   return hsd_launch_status();
 }
 

@@ -140,6 +140,7 @@ template <typename T>
 static int launch_draft_sample_t(const void *logits, int V, const SampleRow *desc, int n_rows, int regular_rows,
                                  u32 regular_serial, u64 seed, int32_t *out, cudaStream_t s) {
   draft_sample_kernel<T><<<n_rows, kSampleThreads, 0, s>>>((const T *)logits, V, desc, regular_rows, regular_serial, seed, out);
+  hsd_count_launches(1);
   return hsd_launch_status();
 }
 
@@ -162,6 +163,7 @@ static int launch_verify_t(const void *p, const void *q, int32_t *tokens, int V,
   decide_kernel<T><<<batch, kSampleThreads, 0, s>>>((const T *)p, (const T *)q, tokens, V, t_max, desc, regular_t,
                                                    regular_serial, regular_level, stats, seed, out_tokens, out_n,
                                                    write_in_place);
+  hsd_count_launches(2);
   return hsd_launch_status();
 }
 
@@ -178,7 +180,11 @@ int launch_verify(const void *p, const void *q, int32_t *tokens, int dtype, int 
 }  // namespace hsd
 
 // ------------------------------------------------------------------------------ C ABI
+unsigned long long g_hsd_launches = 0;
+
 extern "C" {
+
+uint64_t hsd_kernel_launches(void) { return g_hsd_launches; }
 
 const char *hsd_strerror(int status) {
   switch (status) {
