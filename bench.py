@@ -138,7 +138,9 @@ def run_ours(args):
     weights = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
     prompts_host = inputs.make_prompts(cfg["vocab"], 1, P, wl["prompt_seed"] + rank).pin_memory()
     prompts = prompts_host.cuda()
-    if wl["T"] is None:
+    if args.T:
+        T, calib = [int(v) for v in args.T.split(",")], None
+    elif wl["T"] is None:
         T, costs, alphas, lat = choose_T(binding, cfg, weights, wl, prompts)
         calib = {"costs_ms": [round(c, 4) for c in costs], "alphas": [round(a, 4) for a in alphas],
                  "expected_ms_per_token": round(lat, 4)}
@@ -291,6 +293,7 @@ def main():
     ap.add_argument("--workload", default="8b3")
     ap.add_argument("--n-new", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--T", default="", help="fix T (comma separated) instead of calibrating / using the workload's")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
