@@ -40,7 +40,8 @@ enum {
   HSD_E_CUDA = -4,
   HSD_E_DEVICE_TIMEOUT = -5,
   HSD_E_UNSUPPORTED = -6,
-  HSD_E_IO = -7
+  HSD_E_IO = -7,
+  HSD_E_TOO_LARGE = -8
 };
 enum { HSD_F32 = 0, HSD_BF16 = 1 };
 
@@ -80,6 +81,31 @@ int hsd_verify_level(int level, const void *target_logits, const void *draft_log
                      uint64_t seed, uint64_t call_serial, void *workspace, size_t workspace_bytes,
                      void *stream, int32_t *out_tokens, int32_t *out_n_accepted);
 
+/* ---------------------------------------------------------------------------------------
+ * hsd_verify_level without a workspace argument and without any allocation.  (The paper has no
+ * counterpart: this entry point exists for integration reasons only.)
+ *
+ * Who needs it: callers that get device buffers handed to them but cannot obtain more -- an
+ * inference-server plugin or a custom op that receives only its input and output tensors, code
+ * running under an allocator it must not re-enter, or a latency-critical thread for which an
+ * allocating call (which may synchronise the whole device) is off limits.  hsd_verify_level
+ * makes such callers find scratch memory somewhere; this variant brings its own.
+ *
+ * Same arguments, outputs and results as hsd_verify_level.  The row statistics live in a fixed
+ * 64 KiB device array inside the library image (every GPU that loads the library holds it until
+ * the process exits), which bounds the call: batch * (2 t + 1) <= 4096, else HSD_E_TOO_LARGE.
+ * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls share the one array and it keeps whatever the last call left in it.  Nothing in
+ *     it has to start at zero (each call overwrites every entry before reading it), but two
+ *     calls that overlap on the GPU -- different streams, or different host threads -- race on it.
+ *     Serialise such calls (one stream, or an event between them).
+ * Errors: INVALID_ARG, TOO_LARGE, CUDA. */
+int hsd_verify_level_static(int level, const void *target_logits, const void *draft_logits,
+                            const int32_t *draft_tokens, int batch, int t, int vocab, int dtype,
+                            uint64_t seed, uint64_t call_serial, void *stream, int32_t *out_tokens,
+                            int32_t *out_n_accepted);
 
 /* ---------------------------------------------------------------------------------------
  * The hierarchy: models M_0..M_K as early exits of one decoder-only transformer (Section 5.1:

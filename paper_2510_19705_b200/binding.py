@@ -43,6 +43,8 @@ def _declare(lib):
     lib.hsd_verify_workspace_bytes.argtypes = [i32, i32]
     lib.hsd_verify_level.restype = i32
     lib.hsd_verify_level.argtypes = [i32, vp, vp, vp, i32, i32, i32, i32, u64, u64, vp, sz, vp, vp, vp]
+    lib.hsd_verify_level_static.restype = i32
+    lib.hsd_verify_level_static.argtypes = [i32, vp, vp, vp, i32, i32, i32, i32, u64, u64, vp, vp, vp]
 
 
 def _check(status):
@@ -99,6 +101,21 @@ def hsd_verify_level(level, target_logits, draft_logits, draft_tokens, seed, cal
                                       _dev(draft_tokens) if t > 0 else None, batch, t, vocab,
                                       _dtype_code(target_logits), seed, call_serial, _dev(workspace),
                                       workspace.numel(), _stream(), _dev(out_tokens), _dev(out_n_accepted)))
+    return out_tokens, out_n_accepted
+
+
+def hsd_verify_level_static(level, target_logits, draft_logits, draft_tokens, seed, call_serial, out_tokens,
+                            out_n_accepted):
+    """hsd_verify_level for callers that cannot allocate: the library's built-in scratch is used and
+    the caller supplies the outputs (out_tokens int32 [batch, t+1], out_n_accepted int32 [batch]).
+    This wrapper allocates nothing either.  Limit: batch * (2 t + 1) <= 4096.  Calls must not
+    overlap on the GPU (they share the scratch)."""
+    batch, tp1, vocab = target_logits.shape
+    t = tp1 - 1
+    _check(library().hsd_verify_level_static(level, _dev(target_logits), _dev(draft_logits) if t > 0 else None,
+                                             _dev(draft_tokens) if t > 0 else None, batch, t, vocab,
+                                             _dtype_code(target_logits), seed, call_serial, _stream(),
+                                             _dev(out_tokens), _dev(out_n_accepted)))
     return out_tokens, out_n_accepted
 
 

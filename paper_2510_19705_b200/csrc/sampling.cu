@@ -177,6 +177,27 @@ int launch_verify(const void *p, const void *q, int32_t *tokens, int dtype, int 
                                                     regular_level, scratch, seed, out_tokens, out_n, write_in_place, s);
 }
 
+// ------------------------------------------------------------------------------ static scratch
+// Scratch for hsd_verify_level_static: lives in the library image, so every GPU that loads the
+// library holds these bytes until the process exits.  One RowStat per logits row of a call.
+constexpr int kStaticStatRows = 4096;                       // 64 KiB
+static __device__ __align__(256) unsigned char g_static_verify_scratch[kStaticStatRows * sizeof(RowStat)];
+
+// In host code the array's name is only a stand-in for the symbol, not a device address: the
+// address has to be asked for, once per device, with that device current.
+static void *g_static_scratch_ptr[64] = {nullptr};
+static int static_scratch_address(void **out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HSD_E_CUDA;
+  if (!g_static_scratch_ptr[dev]) {
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_verify_scratch) != cudaSuccess || !p) return HSD_E_CUDA;
+    g_static_scratch_ptr[dev] = p;
+  }
+  *out = g_static_scratch_ptr[dev];
+  return HSD_OK;
+}
+
 }  // namespace hsd
 
 // ------------------------------------------------------------------------------ C ABI
@@ -196,6 +217,7 @@ const char *hsd_strerror(int status) {
     case HSD_E_DEVICE_TIMEOUT: return "device-side wait timed out";
     case HSD_E_UNSUPPORTED: return "unsupported configuration";
     case HSD_E_IO: return "I/O error";
+    case HSD_E_TOO_LARGE: return "request exceeds the built-in scratch capacity";
     default: return "unknown status";
   }
 }
@@ -226,6 +248,25 @@ int hsd_verify_level(int level, const void *target_logits, const void *draft_log
   if (workspace_bytes < hsd::verify_scratch_bytes(batch, t)) return HSD_E_WORKSPACE_TOO_SMALL;
   return hsd::launch_verify(target_logits, draft_logits, const_cast<int32_t *>(draft_tokens), dtype, vocab, batch, t,
                             nullptr, t, (u32)call_serial, (u32)level, workspace, seed, out_tokens, out_n_accepted, 0,
+                            (cudaStream_t)stream);
+}
+
+int hsd_verify_level_static(int level, const void *target_logits, const void *draft_logits, const int32_t *draft_tokens,
+                            int batch, int t, int vocab, int dtype, uint64_t seed, uint64_t call_serial, void *stream,
+                            int32_t *out_tokens, int32_t *out_n_accepted) {
+  if (!target_logits || !out_tokens || !out_n_accepted) return HSD_E_INVALID_ARG;
+  if (batch <= 0 || t < 0 || vocab <= 0 || level < 0 || level > 255) return HSD_E_INVALID_ARG;
+  if (t > 0 && (!draft_logits || !draft_tokens)) return HSD_E_INVALID_ARG;
+  if (t >= hsd::kSampleThreads || batch > 65535) return HSD_E_INVALID_ARG;
+  if (dtype != HSD_F32 && dtype != HSD_BF16) return HSD_E_INVALID_ARG;
+  if ((long long)batch * (2 * t + 1) > hsd::kStaticStatRows) return HSD_E_TOO_LARGE;
+  void *scratch = nullptr;
+  int st = hsd::static_scratch_address(&scratch);          // first call on this device looks the symbol up
+  if (st) return st;
+  // every RowStat the decision reads is written by the statistics kernel of the same call first,
+  // so nothing left over from an earlier call needs clearing
+  return hsd::launch_verify(target_logits, draft_logits, const_cast<int32_t *>(draft_tokens), dtype, vocab, batch, t,
+                            nullptr, t, (u32)call_serial, (u32)level, scratch, seed, out_tokens, out_n_accepted, 0,
                             (cudaStream_t)stream);
 }
 
