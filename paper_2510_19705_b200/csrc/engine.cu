@@ -2,12 +2,14 @@
 // independent sequences), the per-level verification step (multi-row forward -> acceptance /
 // resample -> KV rollback), KV paging, workspace carving, statistics and the decision log.
 #include <stdio.h>
+#include <stdlib.h>
 #include <math.h>
 #include <algorithm>
 #include <new>
 #include <vector>
 
 #include "forward.cuh"
+#include "fwd_persist.cuh"
 #include "gemm_tc.cuh"
 #include "sampling_api.cuh"
 
@@ -37,7 +39,7 @@ size_t elem_size(int dtype) { return dtype == HSD_BF16 ? 2 : 4; }
 // Workspace layout, shared by hsd_workspace_bytes and hsd_create.
 struct Layout {
   size_t tokens, cos_tab, sin_tab, page_table, k_pool, v_pool, pool_layer_stride, x, h, qkv, q, att, act, partials, hf,
-      vscratch, n_acc, ring, tc_scratch, tc_pieces_bytes, total;
+      vscratch, n_acc, ring, tc_scratch, tc_pieces_bytes, wmaps_dev, layers_dev, attn_counters, grid_counter, prof, total;
   std::vector<size_t> logits;
   std::vector<int> slots;
   int max_rows, pages_per_seq, n_pages, partial_rows;
@@ -125,6 +127,11 @@ Layout make_layout(const hsd_model_desc *m, int n_levels, const int32_t *T) {
       }
   }
   L.tc_scratch = take(kTcCtrlBytes + L.tc_pieces_bytes);
+  L.wmaps_dev = take(((size_t)m->n_layers * 7 + 1) * sizeof(CUtensorMap));
+  L.layers_dev = take((size_t)m->n_layers * sizeof(FwdLayerDev));
+  L.attn_counters = take(16384);
+  L.grid_counter = take(256);
+  L.prof = take((size_t)device_sm_count() * kFwdProfEvents * 8);
   L.total = off;
   return L;
 }
@@ -170,7 +177,7 @@ struct hsd_ctx {
   cudaStream_t stream;
   uint64_t seed;
   // tensor-core GEMM state (bf16 models)
-  bool use_tc;
+  bool use_tc, use_persist;
   int sm_count;
   std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + 1]: wq wk wv wo wg wu wd per layer, then lm_head
   CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
@@ -285,11 +292,12 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   const ModelDims &md = c->md;
   const Layout &L = c->lay;
   int R = 0, n_attn = 0, n_logit = 0, max_kv = 0;
+  const int arows = c->use_persist ? fwd_attn_rows(md.nq / md.nkv, md.hd) : kAttnRows;   // rows per attention item
   for (const SeqWork &w : work) {
     int rows = w.end - w.start;
     if (rows <= 0 || w.start < 0 || w.end > md.max_seq) return HSD_E_INVALID_ARG;
     R += rows;
-    n_attn += (rows + kAttnRows - 1) / kAttnRows;
+    n_attn += (rows + arows - 1) / arows;
     if (w.logit_first >= 0) {
       if (w.logit_first < w.start || w.logit_first >= w.end) return HSD_E_INVALID_ARG;
       n_logit += w.end - w.logit_first;
@@ -313,8 +321,8 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   long long *ldst = (long long *)(host + o_dst);
   int r = 0, ia = 0, il = 0;
   for (const SeqWork &w : work) {
-    for (int p0 = w.start; p0 < w.end; p0 += kAttnRows) {
-      int rows = std::min(kAttnRows, w.end - p0);
+    for (int p0 = w.start; p0 < w.end; p0 += arows) {
+      int rows = std::min(arows, w.end - p0);
       attn[ia++] = make_int4(r + (p0 - w.start), rows, w.b, p0);
     }
     for (int p = w.start; p < w.end; ++p, ++r) {
@@ -343,7 +351,8 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   rb.lrow_dst = (const long long *)(devp + o_dst);
 
   // attention split: enough blocks to fill the GPU, never more partial rows than the buffer holds
-  int n_splits = std::max(1, std::min(kMaxSplits, kAttnBlocksTarget / std::max(1, n_attn * md.nkv)));
+  const int blocks_target = c->use_persist ? c->sm_count : kAttnBlocksTarget;
+  int n_splits = std::max(1, std::min(kMaxSplits, blocks_target / std::max(1, n_attn * md.nkv)));
   int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, kAttnKeyTile);
   n_splits = (max_kv + keys_per_split - 1) / keys_per_split;
   if ((size_t)R * n_splits > (size_t)L.partial_rows) return HSD_E_INVALID_ARG;
@@ -355,6 +364,60 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     cudaEventRecord(tp->a, c->stream);
   }
   cudaStream_t s = c->stream;
+  if (c->use_persist && R <= 128 && n_logit <= 128) {
+    // one cooperative launch runs the whole pass
+    FwdArgs a;
+    a.d = md.d; a.nq = md.nq; a.nkv = md.nkv; a.hd = md.hd; a.ff = md.ff; a.V = md.V;
+    a.n_run = c->exits[level]; a.lm_map = md.n_layers * 7; a.max_seq = md.max_seq; a.page = md.page;
+    a.pages_per_seq = md.pages_per_seq; a.eps = md.eps;
+    a.wmaps = c->dev<CUtensorMap>(L.wmaps_dev);
+    a.layers = c->dev<FwdLayerDev>(L.layers_dev);
+    a.embed = (const __nv_bfloat16 *)c->embed; a.final_norm = (const __nv_bfloat16 *)c->final_norm;
+    a.cos_tab = c->dev<float>(L.cos_tab); a.sin_tab = c->dev<float>(L.sin_tab);
+    a.R = R; a.L = n_logit; a.n_attn = n_attn; a.attn_rows = arows; a.n_splits = n_splits; a.keys_per_split = keys_per_split;
+    a.tokens = c->dev<int>(L.tokens); a.page_table = c->dev<int>(L.page_table);
+    a.row_seq = rb.row_seq; a.row_pos = rb.row_pos; a.lrow_src = rb.lrow_src; a.attn_items = rb.attn; a.lrow_dst = rb.lrow_dst;
+    a.x = c->dev<float>(L.x);
+    a.h = c->dev<__nv_bfloat16>(L.h); a.q = c->dev<__nv_bfloat16>(L.q); a.att = c->dev<__nv_bfloat16>(L.att);
+    a.act = c->dev<__nv_bfloat16>(L.act); a.hf = c->dev<__nv_bfloat16>(L.hf);
+    a.logits = (__nv_bfloat16 *)(c->ws + L.logits[level]);
+    a.attn_partials = c->dev<float>(L.partials); a.attn_counters = c->dev<int>(L.attn_counters);
+    a.pieces = (float *)(c->ws + L.tc_scratch + kTcCtrlBytes); a.tile_counters = (int *)(c->ws + L.tc_scratch + 256);
+    a.grid_counter = c->dev<unsigned>(L.grid_counter); a.status = (int *)(c->ws + L.tc_scratch);
+    const int np = tc_npad(std::max(R, n_logit));
+    const int pi = np == 16 ? 0 : np == 32 ? 1 : np == 64 ? 2 : 3;
+    for (int b = 0; b < 4; ++b) a.amap[b] = c->amaps[b][pi];
+    // debugging aid: HSD_PROFILE=<file> dumps the barrier timeline of the latest top-level pass
+    const char *prof_path = getenv("HSD_PROFILE");
+    const bool prof = prof_path && level == c->n_levels - 1 && n_logit > 0;
+    a.prof = prof ? c->dev<unsigned long long>(L.prof) : nullptr;
+    if (prof) HSD_CUDA_OK(cudaMemsetAsync(a.prof, 0, (size_t)c->sm_count * kFwdProfEvents * 8, s));
+    HSD_CUDA_OK(cudaMemsetAsync(a.grid_counter, 0, 4, s));
+    int stp = launch_forward_persistent(a, np, c->sm_count, s);
+    if (stp) return stp;
+    if (prof) {
+      std::vector<unsigned long long> ev((size_t)c->sm_count * kFwdProfEvents);
+      if (cudaMemcpyAsync(ev.data(), a.prof, ev.size() * 8, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
+          cudaStreamSynchronize(s) == cudaSuccess) {
+        FILE *f = fopen(prof_path, "w");
+        if (f) {
+          fprintf(f, "%d %d %d %d\n", c->sm_count, kFwdProfEvents, a.n_run, R);
+          for (int b = 0; b < c->sm_count; ++b) {
+            for (int e = 0; e < kFwdProfEvents && (e < 2 || ev[(size_t)b * kFwdProfEvents + e]); ++e)
+              fprintf(f, "%llu ", ev[(size_t)b * kFwdProfEvents + e]);
+            fprintf(f, "\n");
+          }
+          fclose(f);
+        }
+      }
+    }
+    if (tp) cudaEventRecord(tp->b, s);
+    c->stats[level].forwards++;
+    c->stats[level].rows += R;
+    for (const SeqWork &w : work)
+      for (int g = 0; g <= level; ++g) c->len_g[w.b][g] = w.end;
+    return HSD_OK;
+  }
   float *x = c->dev<float>(L.x);
   void *h = c->dev<void>(L.h), *q = c->dev<void>(L.q), *att = c->dev<void>(L.att), *act = c->dev<void>(L.act);
   float *qkv = c->dev<float>(L.qkv);
@@ -613,7 +676,7 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
   c->embed = model->embed; c->final_norm = model->final_norm; c->lm_head = model->lm_head;
   c->lw.assign(model->layer_weights, model->layer_weights + (size_t)model->n_layers * 9);
   c->ring_host = nullptr; c->n_acc_host = nullptr; c->page_table_host = nullptr; c->status_host = nullptr;
-  c->use_tc = false; c->sm_count = 148;
+  c->use_tc = false; c->use_persist = false; c->sm_count = 148;
   c->trace = nullptr; c->trace_logit_calls = 0; c->trace_records = 0;
   c->ring_next = 0; c->ring_in_flight = 0; c->timers_used = 0; c->timers_ok = true; c->stream = nullptr; c->seed = 0;
   bool ok = cudaMallocHost(&c->ring_host, lay.ring_slot * kRingSlots) == cudaSuccess &&
@@ -664,6 +727,25 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
     for (int b = 0; b < 4 && !st; ++b)
       for (int p = 0; p < 4 && !st; ++p) st = tc_make_map(&c->amaps[b][p], c->ws + abuf_off[b], arows[b], acols[b], npads[p]);
     if (!st && cudaMemset(c->ws + lay.tc_scratch, 0, kTcCtrlBytes) != cudaSuccess) st = HSD_E_CUDA;
+    // tables of the persistent forward: tensor maps and per-layer pointers in device memory
+    if (!st) {
+      std::vector<FwdLayerDev> ld(md.n_layers);
+      for (int l = 0; l < md.n_layers; ++l) {
+        ld[l].attn_norm = (const __nv_bfloat16 *)c->lw[(size_t)l * 9 + 0];
+        ld[l].mlp_norm = (const __nv_bfloat16 *)c->lw[(size_t)l * 9 + 5];
+        ld[l].k_pool = (__nv_bfloat16 *)(c->ws + lay.k_pool + lay.pool_layer_stride * l);
+        ld[l].v_pool = (__nv_bfloat16 *)(c->ws + lay.v_pool + lay.pool_layer_stride * l);
+      }
+      if (cudaMemcpy(c->ws + lay.wmaps_dev, c->wmaps.data(), c->wmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemcpy(c->ws + lay.layers_dev, ld.data(), ld.size() * sizeof(FwdLayerDev), cudaMemcpyHostToDevice) != cudaSuccess ||
+          cudaMemset(c->ws + lay.attn_counters, 0, 16384) != cudaSuccess || cudaMemset(c->ws + lay.grid_counter, 0, 256) != cudaSuccess)
+        st = HSD_E_CUDA;
+      int coop = 0, dev = 0;
+      cudaGetDevice(&dev);
+      cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+      c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 &&
+                       getenv("HSD_NO_PERSIST") == nullptr;
+    }
     if (!st && cudaMallocHost(&c->status_host, 4) != cudaSuccess) st = HSD_E_CUDA;
     if (st) {
       hsd_destroy(c);

@@ -1,0 +1,53 @@
+// Persistent single-launch verifier forward (bf16 models): one cooperative kernel, one CTA per SM,
+// runs every layer of a level's forward pass.  The TMA weight stream never stops at a GEMM
+// boundary: the producer keeps filling the shared-memory ring with the next projection's weight
+// tiles while the other warps go through a grid barrier and the small phases (RMSNorm, attention).
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+
+namespace hsd {
+
+struct FwdLayerDev {
+  const __nv_bfloat16 *attn_norm, *mlp_norm;
+  __nv_bfloat16 *k_pool, *v_pool;
+};
+
+struct FwdArgs {
+  // geometry
+  int d, nq, nkv, hd, ff, V, n_run, lm_map, max_seq, page, pages_per_seq;
+  float eps;
+  // immutable inputs
+  const CUtensorMap *wmaps;        // global memory: 7 per layer (wq wk wv wo wg wu wd), then the output head
+  const FwdLayerDev *layers;       // global memory [n_layers]
+  const __nv_bfloat16 *embed, *final_norm;
+  const float *cos_tab, *sin_tab;
+  // this call
+  int R, L, n_attn, attn_rows, n_splits, keys_per_split;
+  const int *tokens, *page_table, *row_seq, *row_pos, *lrow_src;
+  const int4 *attn_items;          // (first packed row, rows, sequence, position of first row)
+  const long long *lrow_dst;
+  // buffers
+  float *x;
+  __nv_bfloat16 *h, *q, *att, *act, *hf, *logits;
+  float *attn_partials;
+  int *attn_counters;              // zero on entry, zero on exit
+  float *pieces;
+  int *tile_counters;              // zero on entry, zero on exit
+  unsigned *grid_counter;          // zero on entry
+  int *status;                     // set non-zero when a bounded wait gave up
+  unsigned long long *prof;        // optional [gridDim][kFwdProfEvents]: barrier arrive / depart times (ns)
+  CUtensorMap amap[4];             // activations h, att, act, hf; box rows = row padding of this launch
+};
+
+constexpr int kFwdThreads = 384;
+constexpr int kFwdProfEvents = 1024;
+// rows of one sequence per attention work item for a given GQA group and head size
+inline int fwd_attn_rows(int group, int hd) {
+  int r = 4096 / (group * hd);
+  return r < 1 ? 1 : (r > 8 ? 8 : r);
+}
+bool fwd_persist_supported(int hd, int group);
+int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaStream_t s);
+
+}  // namespace hsd
