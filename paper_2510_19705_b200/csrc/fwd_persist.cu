@@ -8,7 +8,8 @@
 // with a grid barrier between phases.  The weight producer is not tied to the barriers: weights are
 // read-only, so it runs ahead into the next GEMM as far as the ring allows; the activation producer
 // waits for the barrier that completes its operand.  GEMM work is split evenly over the CTAs in
-// (tile, k-block) units; tiles cut by a split are finished by the last arriver in fixed piece order.
+// (tile, k-block) units; each segment's partial sums go to a piece buffer and the following phase
+// (the next RMSNorm for the residual projections, a short finish phase otherwise) adds them up.
 // Every wait (mbarrier, grid barrier) is bounded by wall time and raises a status word.
 #include "fwd_persist.cuh"
 #include "forward.cuh"
@@ -89,12 +90,47 @@ __device__ __forceinline__ Tile tile_of(const Gemm &g, int tile) {
   t.seg = 0; t.row0 = 0; t.col0 = 0;
   return t;
 }
-__device__ __forceinline__ long long cta_begin(long long U, int G, int c) { return (U * c) / G; }
-__device__ __forceinline__ int unit_owner(long long U, int G, long long u) {
-  int c = (int)((u * G) / U);
+// Unit arithmetic in 32 bits (the launcher checks n_tiles * KB * grid < 2^31).
+__device__ __forceinline__ int cta_begin(int U, int G, int c) { return (int)(((unsigned)U * (unsigned)c) / (unsigned)G); }
+__device__ __forceinline__ int unit_owner(int U, int G, int u) {
+  int c = (int)(((unsigned)u * (unsigned)G) / (unsigned)U);
   while (c + 1 < G && cta_begin(U, G, c + 1) <= u) ++c;
   while (c > 0 && cta_begin(U, G, c) > u) --c;
   return c;
+}
+// Work of one CTA in one GEMM, a segment (tile, k-block range) at a time.  One SM can pull only its
+// share of HBM bandwidth, so every GEMM is split evenly over all CTAs in (tile, k-block) units;
+// each segment's partial sums go to a piece buffer and the next phase adds the pieces of a tile in
+// fixed piece order (bit-reproducible; no CTA waits for another inside a GEMM).
+struct Seg { int tile, kb0, kb1; };
+struct SegIter { int cur, end; };
+struct SplitGeom { int U, Gp, pieces_max; };
+__device__ __forceinline__ SplitGeom split_geom(const Gemm &g, int G) {
+  SplitGeom sg;
+  sg.U = g.n_tiles * g.KB;
+  sg.Gp = min(G, sg.U);
+  const int per = sg.U / sg.Gp;
+  sg.pieces_max = (g.KB + per - 1) / per + 1;
+  return sg;
+}
+__device__ __forceinline__ SegIter seg_begin(const Gemm &g, int G, int c) {
+  SegIter it;
+  const SplitGeom sg = split_geom(g, G);
+  it.cur = c < sg.Gp ? cta_begin(sg.U, sg.Gp, c) : 0;
+  it.end = c < sg.Gp ? cta_begin(sg.U, sg.Gp, c + 1) : 0;
+  return it;
+}
+__device__ __forceinline__ bool seg_next(const Gemm &g, SegIter &it, Seg &s) {
+  if (it.cur >= it.end) return false;
+  s.tile = it.cur / g.KB; s.kb0 = it.cur % g.KB;
+  s.kb1 = min(g.KB, s.kb0 + (it.end - it.cur));
+  it.cur += s.kb1 - s.kb0;
+  return true;
+}
+// Pieces of a tile: they belong to consecutive CTAs first_owner .. first_owner + n - 1.
+__device__ __forceinline__ void tile_pieces(const Gemm &g, const SplitGeom &geo, int tile, int &first_owner, int &n) {
+  first_owner = unit_owner(geo.U, geo.Gp, tile * g.KB);
+  n = unit_owner(geo.U, geo.Gp, tile * g.KB + g.KB - 1) - first_owner + 1;
 }
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
@@ -104,12 +140,6 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
   return v;
 }
 __device__ __forceinline__ float bf(const __nv_bfloat16 v) { return __bfloat162float(v); }
-// Ask for one weight box to be brought into L2 (no shared-memory destination, nothing to wait for).
-__device__ __forceinline__ void tma_prefetch_l2(const CUtensorMap *map, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y)
-               : "memory");
-}
 
 // Grid-wide barrier of the worker threads.  `epoch` counts barriers; the counter only grows.
 // If ready_bar != 0 the spinning thread then releases the activation producer for the next GEMM.
@@ -151,12 +181,21 @@ __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, 
 }
 
 // ------------------------------------------------------------------------------ RMSNorm phase
-// One row per CTA turn, held in registers (all loads issued before the first use).  src_embed: rows
-// come from the embedding table (and are copied to x).  Requires d % 4 == 0 and d <= 8192.
+// One row per CTA turn, held in registers (all loads issued before their first use).
+//   src_embed: the row comes from the embedding table (and is copied to x).
+//   pend:      the residual-add projection that ran just before; its split pieces are added to the
+//              row in fixed piece order (x <- x + p_0 + p_1 + ...) and x is written back.
+// Requires d % 4 == 0 and d <= 4096.
+template <int NPAD>
 __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const int *row_list, bool src_embed,
-                                           const __nv_bfloat16 *gain, __nv_bfloat16 *dst, float *red, int wt) {
-  constexpr int MAXV = 8;                                  // float4 slots per thread
+                                           const Gemm *pend, const __nv_bfloat16 *gain, __nv_bfloat16 *dst, float *red,
+                                           int wt) {
+  constexpr int MAXV = 4;                                  // float4 slots per thread
+  constexpr int PB = 8;                                    // pieces loaded at a time per slot
   const int d = a.d, nvec = d >> 2;
+  SplitGeom geo;
+  geo.U = 1; geo.Gp = 1; geo.pieces_max = 1;
+  if (pend) geo = split_geom(*pend, gridDim.x);
   for (int i = blockIdx.x; i < n_rows; i += gridDim.x) {
     const int row = row_list ? row_list[i] : i;
     float *xrow = a.x + (size_t)row * d;
@@ -186,6 +225,42 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
       const int iv = wt + 256 * j;
       graw[j] = iv < nvec ? __ldg(reinterpret_cast<const uint2 *>(gain) + iv) : make_uint2(0u, 0u);
     }
+    if (pend) {
+#pragma unroll
+      for (int j0 = 0; j0 < MAXV; j0 += 2) {               // two slots at a time: all their loads in flight together
+        int np[2];
+        const float *base[2];
+#pragma unroll
+        for (int jj = 0; jj < 2; ++jj) {
+          const int iv = wt + 256 * (j0 + jj);
+          np[jj] = 0;
+          base[jj] = a.pieces;
+          if (iv < nvec) {
+            const int k = iv << 2, tile = k >> 7, mm = k & 127;
+            int fo;
+            tile_pieces(*pend, geo, tile, fo, np[jj]);
+            base[jj] = a.pieces + ((size_t)tile * geo.pieces_max * NPAD + row) * kTcBlockM + mm;
+          }
+        }
+        for (int p0 = 0; p0 < max(np[0], np[1]); p0 += PB) {
+          float4 t[2][PB];
+#pragma unroll
+          for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+            for (int pp = 0; pp < PB; ++pp)
+              t[jj][pp] = (p0 + pp < np[jj])
+                              ? __ldcg(reinterpret_cast<const float4 *>(base[jj] + (size_t)(p0 + pp) * NPAD * kTcBlockM))
+                              : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int jj = 0; jj < 2; ++jj)
+#pragma unroll
+            for (int pp = 0; pp < PB; ++pp) {
+              v[j0 + jj].x += t[jj][pp].x; v[j0 + jj].y += t[jj][pp].y;
+              v[j0 + jj].z += t[jj][pp].z; v[j0 + jj].w += t[jj][pp].w;
+            }
+        }
+      }
+    }
     float ss = 0.f;
 #pragma unroll
     for (int j = 0; j < MAXV; ++j) ss += v[j].x * v[j].x + v[j].y * v[j].y + v[j].z * v[j].z + v[j].w * v[j].w;
@@ -201,7 +276,7 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
     for (int j = 0; j < MAXV; ++j) {
       const int iv = wt + 256 * j;
       if (iv < nvec) {
-        if (src_embed) reinterpret_cast<float4 *>(xrow)[iv] = v[j];
+        if (src_embed || pend) reinterpret_cast<float4 *>(xrow)[iv] = v[j];
         const float g0 = __uint_as_float(graw[j].x << 16), g1 = __uint_as_float(graw[j].x & 0xFFFF0000u);
         const float g2 = __uint_as_float(graw[j].y << 16), g3 = __uint_as_float(graw[j].y & 0xFFFF0000u);
         __nv_bfloat162 lo = __floats2bfloat162_rn(v[j].x * inv * g0, v[j].y * inv * g1);
@@ -357,17 +432,7 @@ __device__ __forceinline__ void final_store(const FwdArgs &a, const Gemm &g, con
                                             int c0, const float *v, float *staging) {
   const int rows = g.rows;
   if (g.mode == MODE_ADD) {
-    const int n = ti.row0 + m;
-    if (n < g.seg_n[0]) {
-#pragma unroll
-      for (int i = 0; i < CH; ++i) {
-        const int r = c0 + i;
-        if (r < rows) {
-          float *px = a.x + (size_t)r * g.seg_n[0] + n;
-          *px = __ldcg(px) + v[i];
-        }
-      }
-    }
+    // residual-add projections never get here: their pieces are summed by the next norm phase
   } else if (g.mode == MODE_LOGITS) {
     const int n = ti.row0 + m;
     if (n < g.seg_n[0]) {
@@ -441,7 +506,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   volatile int *last_flag = reinterpret_cast<volatile int *>(ctl + 2);
   volatile int *wait_ok = reinterpret_cast<volatile int *>(ctl + 4);   // [2]
   float *red = reinterpret_cast<float *>(ctl + 8);                      // [8]
-  volatile long long *w_issued = reinterpret_cast<volatile long long *>(ctl + 16);   // weight tiles sent to the ring
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -458,7 +522,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); mbar_init(ready_bar(b), 1); }
     *abort_flag = 0;
     *last_flag = 0;
-    *w_issued = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
@@ -474,15 +537,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       bool ok = true;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
-        const long long U = (long long)g.n_tiles * g.KB;
-        const int Gp = (int)min((long long)G, U);               // CTAs that take part in this phase
-        const long long u0 = c < Gp ? cta_begin(U, Gp, c) : 0, u1 = c < Gp ? cta_begin(U, Gp, c + 1) : 0;
-        for (long long u = u0; u < u1 && ok;) {
-          const int tile = (int)(u / g.KB), kb0 = (int)(u % g.KB);
-          const int kb1 = (int)min((long long)g.KB, kb0 + (u1 - u));
-          const Tile ti = tile_of(g, tile);
+        SegIter it = seg_begin(g, G, c);
+        Seg sg;
+        while (ok && seg_next(g, it, sg)) {
+          const Tile ti = tile_of(g, sg.tile);
           const bool second = (g.mode == MODE_SWIGLU) || (ti.row0 + kTcBoxRows < g.seg_n[ti.seg]);
-          for (int kb = kb0; kb < kb1; ++kb, ++issued) {
+          for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++issued) {
             const int s = (int)(issued % STAGES);
             const uint32_t ph = (uint32_t)((issued / STAGES) & 1);
             if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -495,9 +555,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
               tma_load_2d(dst, g.w[ti.seg], kb * kTcBlockK, ti.row0, full_bar(s));
               if (second) tma_load_2d(dst + kBoxBytes, g.w[ti.seg], kb * kTcBlockK, ti.row0 + kTcBoxRows, full_bar(s));
             }
-            *w_issued = issued + 1;
           }
-          u += kb1 - kb0;
         }
       }
       if (!ok) {
@@ -517,19 +575,19 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       bool ok = true;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
-        const long long U = (long long)g.n_tiles * g.KB;
-        const int Gp = (int)min((long long)G, U);               // CTAs that take part in this phase
-        const long long u0 = c < Gp ? cta_begin(U, Gp, c) : 0, u1 = c < Gp ? cta_begin(U, Gp, c + 1) : 0;
         // the operand of phase p is complete once the workers have passed the barrier before it
         if (!mbar_wait(ready_bar(p & 1), (uint32_t)((p >> 1) & 1), abort_flag)) { ok = false; break; }
-        for (long long u = u0; u < u1 && ok; ++u, ++issued) {
-          const int kb = (int)(u % g.KB);
-          const int s = (int)(issued % STAGES);
-          const uint32_t ph = (uint32_t)((issued / STAGES) & 1);
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-          const uint32_t dst = smem_u32(ring + (size_t)s * Cfg::kStageBytes) + kWBytes;
-          mbar_expect_tx(full_bar(s), NPAD * kTcBlockK * 2);
-          tma_load_2d(dst, g.amap, kb * kTcBlockK, 0, full_bar(s));
+        SegIter it = seg_begin(g, G, c);
+        Seg sg;
+        while (ok && seg_next(g, it, sg)) {
+          for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++issued) {
+            const int s = (int)(issued % STAGES);
+            const uint32_t ph = (uint32_t)((issued / STAGES) & 1);
+            if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t dst = smem_u32(ring + (size_t)s * Cfg::kStageBytes) + kWBytes;
+            mbar_expect_tx(full_bar(s), NPAD * kTcBlockK * 2);
+            tma_load_2d(dst, g.amap, kb * kTcBlockK, 0, full_bar(s));
+          }
         }
       }
       if (!ok) atomicExch(a.status, 1);
@@ -543,12 +601,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       bool ok = true;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
-        const long long U = (long long)g.n_tiles * g.KB;
-        const int Gp = (int)min((long long)G, U);               // CTAs that take part in this phase
-        const long long u0 = c < Gp ? cta_begin(U, Gp, c) : 0, u1 = c < Gp ? cta_begin(U, Gp, c + 1) : 0;
-        for (long long u = u0; u < u1 && ok; ++seg_idx) {
-          const int kb0 = (int)(u % g.KB);
-          const int kb1 = (int)min((long long)g.KB, kb0 + (u1 - u));
+        SegIter it = seg_begin(g, G, c);
+        Seg sg;
+        for (; ok && seg_next(g, it, sg); ++seg_idx) {
+          const int kb0 = sg.kb0, kb1 = sg.kb1;
           const int ab = seg_idx & 1;
           if (!mbar_wait(acce_bar(ab), (uint32_t)(((seg_idx >> 1) & 1) ^ 1), abort_flag)) { ok = false; break; }
           tc_fence_after();
@@ -565,48 +621,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
             umma_commit(empty_bar(s));
           }
           if (ok) umma_commit(accf_bar(ab));
-          u += kb1 - kb0;
         }
       }
       if (!ok) atomicExch(a.status, 1);
-    }
-  } else if (warp == 3) {
-    // ------------------------------------------------------------ L2 prefetch stream
-    // Walks the same weight-tile sequence as the producer, kLookahead tiles further on, and only
-    // asks L2 to fetch them: when the ring is full (the consumers sit in a barrier or a small
-    // phase) HBM keeps streaming the next projection's weights into L2.
-    if (lane == 0) {
-      constexpr long long kLookahead = 28;
-      long long j = 0;
-      bool ok = true;
-      for (int p = 0; p < n_phases && ok; ++p) {
-        const Gemm g = make_gemm(a, p);
-        const long long U = (long long)g.n_tiles * g.KB;
-        const int Gp = (int)min((long long)G, U);
-        const long long u0 = c < Gp ? cta_begin(U, Gp, c) : 0, u1 = c < Gp ? cta_begin(U, Gp, c + 1) : 0;
-        for (long long u = u0; u < u1 && ok; ++u, ++j) {
-          if (j < STAGES) continue;                                  // the ring itself covers the first tiles
-          unsigned long long t0 = 0;
-          for (uint32_t it = 0; j >= *w_issued + kLookahead; ++it) {
-            __nanosleep(100);
-            if ((it & 63u) == 63u) {
-              if (t0 == 0) t0 = globaltimer_ns();
-              if (*abort_flag || globaltimer_ns() - t0 > 2 * kWaitLimitNs) { ok = false; break; }
-            }
-          }
-          if (!ok) break;
-          if (j < *w_issued) continue;                               // the producer already overtook this tile
-          const int tile = (int)(u / g.KB), kb = (int)(u % g.KB);
-          const Tile ti = tile_of(g, tile);
-          if (g.mode == MODE_SWIGLU) {
-            tma_prefetch_l2(g.w[0], kb * kTcBlockK, ti.row0);
-            tma_prefetch_l2(g.w[1], kb * kTcBlockK, ti.row0);
-          } else {
-            tma_prefetch_l2(g.w[ti.seg], kb * kTcBlockK, ti.row0);
-            if (ti.row0 + kTcBoxRows < g.seg_n[ti.seg]) tma_prefetch_l2(g.w[ti.seg], kb * kTcBlockK, ti.row0 + kTcBoxRows);
-          }
-        }
-      }
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------ workers (+ epilogue: warps 4..7)
@@ -622,94 +639,78 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     // GEMM phase p, epilogue side.  Group-uniform: a give-up is decided by one thread and shared.
     auto epilogue = [&](int p) {
       const Gemm g = make_gemm(a, p);
-      const long long U = (long long)g.n_tiles * g.KB;
-      const int Gp = (int)min((long long)G, U);
-      const long long u0 = c < Gp ? cta_begin(U, Gp, c) : 0, u1 = c < Gp ? cta_begin(U, Gp, c + 1) : 0;
-      const long long per = U / Gp;
-      const int pieces_max = (int)((g.KB + per - 1) / per) + 1;
-      const int layer = p >> 2;
-      for (long long u = u0; u < u1; ++seg_idx) {
-        const int tile = (int)(u / g.KB), kb0 = (int)(u % g.KB);
-        const int kb1 = (int)min((long long)g.KB, kb0 + (u1 - u));
+      const SplitGeom geo = split_geom(g, G);
+      SegIter it = seg_begin(g, G, c);
+      Seg sg;
+      for (; seg_next(g, it, sg); ++seg_idx) {
         const int ab = seg_idx & 1;
         if (et == 0) wait_ok[seg_idx & 1] = mbar_wait(accf_bar(ab), (uint32_t)((seg_idx >> 1) & 1), abort_flag) ? 1 : 0;
         epi_sync();
         if (!wait_ok[seg_idx & 1]) return;
         tc_fence_after();
-        const Tile ti = tile_of(g, tile);
-        const bool whole = (kb0 == 0 && kb1 == g.KB);
         const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * NPAD);
-        if (whole) {
+        // this CTA's piece of the tile; the next phase sums the pieces
+        const int piece = c - unit_owner(geo.U, geo.Gp, sg.tile * g.KB);
+        float *mine = a.pieces + ((size_t)sg.tile * geo.pieces_max + piece) * NPAD * kTcBlockM;
 #pragma unroll 1
-          for (int c0 = 0; c0 < NPAD; c0 += CH) {
-            float v[CH];
+        for (int c0 = 0; c0 < NPAD; c0 += CH) {
+          float v[CH];
 #pragma unroll
-            for (int j = 0; j < CH / 16; ++j) tmem_ld16(tbase + c0 + j * 16, v + j * 16);
-            tmem_ld_wait();
-            if (c0 + CH >= NPAD) {                 // accumulator fully read: hand it back to the MMA warp
-              tc_fence_before();
-              __syncwarp();
-              if (lane == 0) mbar_arrive(acce_bar(ab));
-            }
-            if (c0 < g.rows) final_store<CH>(a, g, ti, layer, m, et, c0, v, staging);
+          for (int j = 0; j < CH / 16; ++j) tmem_ld16(tbase + c0 + j * 16, v + j * 16);
+          tmem_ld_wait();
+          if (c0 + CH >= NPAD) {                   // accumulator fully read: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acce_bar(ab));
           }
-        } else {
-          const int first_owner = unit_owner(U, Gp, (long long)tile * g.KB);
-          const int last_owner = unit_owner(U, Gp, (long long)tile * g.KB + g.KB - 1);
-          const int n_pieces = last_owner - first_owner + 1, piece = c - first_owner;
-          float *mine = a.pieces + ((size_t)tile * pieces_max + piece) * NPAD * kTcBlockM;
-#pragma unroll 1
-          for (int c0 = 0; c0 < NPAD; c0 += CH) {
-            float v[CH];
+          if (c0 < g.rows) {
 #pragma unroll
-            for (int j = 0; j < CH / 16; ++j) tmem_ld16(tbase + c0 + j * 16, v + j * 16);
-            tmem_ld_wait();
-            if (c0 < g.rows) {
-#pragma unroll
-              for (int i = 0; i < CH; ++i) mine[(c0 + i) * kTcBlockM + m] = v[i];
-            }
-          }
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(acce_bar(ab));
-          __threadfence();
-          epi_sync();
-          if (et == 0) {
-            int prev = atomicAdd(&a.tile_counters[tile], 1);
-            int last = (prev == n_pieces - 1);
-            if (last) a.tile_counters[tile] = 0;
-            *last_flag = last;
-            __threadfence();
-          }
-          epi_sync();
-          const bool finish = (*last_flag != 0);
-          epi_sync();                               // last_flag may be rewritten by the next tile
-          if (finish) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < NPAD && c0 < g.rows; c0 += CH) {
-              float v[CH];
-#pragma unroll
-              for (int i = 0; i < CH; ++i) v[i] = 0.f;
-              for (int pc = 0; pc < n_pieces; ++pc) {
-                const float *src = a.pieces + ((size_t)tile * pieces_max + pc) * NPAD * kTcBlockM;
-#pragma unroll
-                for (int i = 0; i < CH; ++i) v[i] += __ldcg(src + (c0 + i) * kTcBlockM + m);
-              }
-              final_store<CH>(a, g, ti, layer, m, et, c0, v, staging);
-            }
+            for (int i = 0; i < CH; ++i)
+              if (c0 + i < g.rows) mine[(c0 + i) * kTcBlockM + m] = v[i];
           }
         }
-        u += kb1 - kb0;
+      }
+    };
+
+    // Finish phase of GEMM p (QKV, gate/up, output head): tiles round-robin over the CTAs; the pieces of
+    // a tile are added in piece order and the result goes through the projection's own epilogue.
+    auto finish = [&](int p) {
+      const Gemm g = make_gemm(a, p);
+      const SplitGeom geo = split_geom(g, G);
+      const int layer = p >> 2;
+      for (int tile = c; tile < g.n_tiles; tile += G) {
+        const Tile ti = tile_of(g, tile);
+        int fo, n_pieces;
+        tile_pieces(g, geo, tile, fo, n_pieces);
+        const float *base = a.pieces + (size_t)tile * geo.pieces_max * NPAD * kTcBlockM + m;
+#pragma unroll 1
+        for (int c0 = 0; c0 < NPAD && c0 < g.rows; c0 += CH) {
+          float v[CH];
+#pragma unroll
+          for (int i = 0; i < CH; ++i) v[i] = 0.f;
+          for (int pc = 0; pc < n_pieces; ++pc) {
+            float t[CH];
+#pragma unroll
+            for (int i = 0; i < CH; ++i)
+              t[i] = (c0 + i < g.rows) ? __ldcg(base + ((size_t)pc * NPAD + c0 + i) * kTcBlockM) : 0.f;
+#pragma unroll
+            for (int i = 0; i < CH; ++i) v[i] += t[i];
+          }
+          final_store<CH>(a, g, ti, layer, m, et, c0, v, staging);
+        }
       }
     };
 
     // ---- phase program
     if (a.prof && wt == 0) a.prof[(size_t)blockIdx.x * kFwdProfEvents] = globaltimer_ns();
-    norm_phase(a, a.R, nullptr, true, a.layers[0].attn_norm, a.h, red, wt);
+    norm_phase<NPAD>(a, a.R, nullptr, true, nullptr, a.layers[0].attn_norm, a.h, red, wt);
     alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar(0));
     for (int l = 0; l < a.n_run && alive; ++l) {
       const int p = 4 * l;
-      if (is_epi) epilogue(p);                                            // QKV + rope + KV append
+      if (is_epi) epilogue(p);                                            // QKV pieces
+      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
+      if (!alive) break;
+      if (is_epi) finish(p);                                              // sum, rope, q / KV append
       alive = grid_barrier(a, epoch, abort_flag, wt, 0);
       if (!alive) break;
       attn_phase<HD>(a, l, scratch, last_flag, wt);
@@ -718,22 +719,33 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       if (is_epi) epilogue(p + 1);                                        // O projection into the residual
       alive = grid_barrier(a, epoch, abort_flag, wt, 0);
       if (!alive) break;
-      norm_phase(a, a.R, nullptr, false, a.layers[l].mlp_norm, a.h, red, wt);
+      {
+        const Gemm pend = make_gemm(a, p + 1);
+        norm_phase<NPAD>(a, a.R, nullptr, false, &pend, a.layers[l].mlp_norm, a.h, red, wt);
+      }
       alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 2) & 1));
       if (!alive) break;
-      if (is_epi) epilogue(p + 2);                                        // gate / up + SwiGLU
+      if (is_epi) epilogue(p + 2);                                        // gate / up pieces
+      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
+      if (!alive) break;
+      if (is_epi) finish(p + 2);                                          // sum, SwiGLU
       alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 3) & 1));
       if (!alive) break;
       if (is_epi) epilogue(p + 3);                                        // down projection into the residual
       if (l + 1 < a.n_run || a.L > 0) {
         alive = grid_barrier(a, epoch, abort_flag, wt, 0);
         if (!alive) break;
-        if (l + 1 < a.n_run) norm_phase(a, a.R, nullptr, false, a.layers[l + 1].attn_norm, a.h, red, wt);
-        else norm_phase(a, a.L, a.lrow_src, false, a.final_norm, a.hf, red, wt);
+        const Gemm pend = make_gemm(a, p + 3);
+        if (l + 1 < a.n_run) norm_phase<NPAD>(a, a.R, nullptr, false, &pend, a.layers[l + 1].attn_norm, a.h, red, wt);
+        else norm_phase<NPAD>(a, a.L, a.lrow_src, false, &pend, a.final_norm, a.hf, red, wt);
         alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 4) & 1));
       }
     }
-    if (alive && a.L > 0 && is_epi) epilogue(4 * a.n_run);                // output head
+    if (alive && a.L > 0) {                                               // output head
+      if (is_epi) epilogue(4 * a.n_run);
+      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
+      if (alive && is_epi) finish(4 * a.n_run);
+    }
   }
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
@@ -777,6 +789,11 @@ bool fwd_persist_supported(int hd, int group) {
 
 int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaStream_t s) {
   if (args.R < 1 || args.R > npad || args.L > npad) return HSD_E_INVALID_ARG;
+  {  // unit arithmetic on the device is 32-bit
+    long long tiles = std::max<long long>((args.V + 127) / 128, (args.ff + 63) / 64);
+    long long kb = std::max(args.ff, std::max(args.d, args.nq * args.hd)) / kTcBlockK;
+    if (tiles * kb * sm_count >= (1ll << 31)) return HSD_E_UNSUPPORTED;
+  }
   switch (args.hd) {
     case 128: return launch_hd<128>(args, npad, sm_count, s);
     case 64: return launch_hd<64>(args, npad, sm_count, s);
