@@ -352,7 +352,8 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
 
   // attention split: enough blocks to fill the GPU, never more partial rows than the buffer holds
   const int blocks_target = c->use_persist ? c->sm_count : kAttnBlocksTarget;
-  int n_splits = std::max(1, std::min(kMaxSplits, blocks_target / std::max(1, n_attn * md.nkv)));
+  const int max_splits = c->use_persist ? 20 : kMaxSplits;      // the persistent merge phase takes <= 20 splits
+  int n_splits = std::max(1, std::min(max_splits, blocks_target / std::max(1, n_attn * md.nkv)));
   int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, kAttnKeyTile);
   n_splits = (max_kv + keys_per_split - 1) / keys_per_split;
   if ((size_t)R * n_splits > (size_t)L.partial_rows) return HSD_E_INVALID_ARG;
@@ -369,6 +370,8 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     FwdArgs a;
     a.d = md.d; a.nq = md.nq; a.nkv = md.nkv; a.hd = md.hd; a.ff = md.ff; a.V = md.V;
     a.n_run = c->exits[level]; a.lm_map = md.n_layers * 7; a.max_seq = md.max_seq; a.page = md.page;
+    a.page_shift = 0;
+    while ((1 << a.page_shift) < md.page) ++a.page_shift;
     a.pages_per_seq = md.pages_per_seq; a.eps = md.eps;
     a.wmaps = c->dev<CUtensorMap>(L.wmaps_dev);
     a.layers = c->dev<FwdLayerDev>(L.layers_dev);
@@ -403,7 +406,7 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
         if (f) {
           fprintf(f, "%d %d %d %d\n", c->sm_count, kFwdProfEvents, a.n_run, R);
           for (int b = 0; b < c->sm_count; ++b) {
-            for (int e = 0; e < kFwdProfEvents && (e < 2 || ev[(size_t)b * kFwdProfEvents + e]); ++e)
+            for (int e = 0; e < kFwdProfEvents; ++e)
               fprintf(f, "%llu ", ev[(size_t)b * kFwdProfEvents + e]);
             fprintf(f, "\n");
           }
@@ -743,7 +746,7 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
       int coop = 0, dev = 0;
       cudaGetDevice(&dev);
       cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-      c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 &&
+      c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 && md.n_layers <= 64 && (md.page & (md.page - 1)) == 0 &&
                        getenv("HSD_NO_PERSIST") == nullptr;
     }
     if (!st && cudaMallocHost(&c->status_host, 4) != cudaSuccess) st = HSD_E_CUDA;

@@ -23,16 +23,21 @@ using namespace ptx;
 
 constexpr int kWBytes = kTcBlockM * kTcBlockK * 2;     // 16 KiB weight tile
 constexpr int kBoxBytes = kTcBoxRows * kTcBlockK * 2;  // 8 KiB TMA box
-constexpr int kScratchBytes = 34 * 1024;               // union: epilogue staging / attention tiles
-constexpr int kCtrlBytes = 1024;
+constexpr int kScratchBytes = 60 * 1024;               // union: epilogue staging / attention tiles
+constexpr int kCtrlBytes = 4096;                       // barriers, flags, page-id cache, per-row info
 constexpr int kSmemTotal = 232448;
 constexpr int kKeyTile = 32;
+constexpr int kMaxLayersSh = 64;                       // layers whose pointer table fits the control area
 
 enum { MODE_QKV = 0, MODE_ADD = 1, MODE_SWIGLU = 2, MODE_LOGITS = 3 };
 
 template <int NPAD> struct PCfg {
   static constexpr int kStageBytes = kWBytes + NPAD * kTcBlockK * 2;
-  static constexpr int kStages = (kSmemTotal - 1024 - kCtrlBytes - kScratchBytes) / kStageBytes;
+#ifndef HSD_STAGE_CAP
+#define HSD_STAGE_CAP 64
+#endif
+  static constexpr int kStagesFit = (kSmemTotal - 1024 - kCtrlBytes - kScratchBytes) / kStageBytes;
+  static constexpr int kStages = kStagesFit < HSD_STAGE_CAP ? kStagesFit : HSD_STAGE_CAP;
   static constexpr int kSmemBytes = kStages * kStageBytes + kScratchBytes + kCtrlBytes + 1024;
   static constexpr int kTmemCols = (2 * NPAD < 32) ? 32 : 2 * NPAD;
   static constexpr int kChunk = NPAD < 32 ? NPAD : 32;      // accumulator columns handled at a time
@@ -104,20 +109,39 @@ __device__ __forceinline__ int unit_owner(int U, int G, int u) {
 // fixed piece order (bit-reproducible; no CTA waits for another inside a GEMM).
 struct Seg { int tile, kb0, kb1; };
 struct SegIter { int cur, end; };
-struct SplitGeom { int U, Gp, pieces_max; };
+// regular: every tile is cut into `parts` equal k-ranges (GEMMs with few tiles: at most 4 pieces per
+// tile, so the consumer can fetch all of them in one batch); otherwise the (tile, k-block) units are
+// dealt out evenly (tiles >= CTAs / 2: a tile then spans at most 3 CTAs).
+struct SplitGeom { int U, Gp, pieces_max, parts; };
 __device__ __forceinline__ SplitGeom split_geom(const Gemm &g, int G) {
   SplitGeom sg;
   sg.U = g.n_tiles * g.KB;
-  sg.Gp = min(G, sg.U);
-  const int per = sg.U / sg.Gp;
-  sg.pieces_max = (g.KB + per - 1) / per + 1;
+  if (g.n_tiles * 2 <= G) {
+    sg.parts = min(min(4, G / g.n_tiles), g.KB);
+    sg.Gp = g.n_tiles * sg.parts;
+    sg.pieces_max = sg.parts;
+  } else {
+    sg.parts = 0;
+    sg.Gp = min(G, sg.U);
+    const int per = sg.U / sg.Gp;
+    sg.pieces_max = (g.KB + per - 1) / per + 1;
+  }
   return sg;
 }
 __device__ __forceinline__ SegIter seg_begin(const Gemm &g, int G, int c) {
   SegIter it;
   const SplitGeom sg = split_geom(g, G);
-  it.cur = c < sg.Gp ? cta_begin(sg.U, sg.Gp, c) : 0;
-  it.end = c < sg.Gp ? cta_begin(sg.U, sg.Gp, c + 1) : 0;
+  it.cur = it.end = 0;
+  if (c < sg.Gp) {
+    if (sg.parts) {
+      const int tile = c / sg.parts, part = c % sg.parts;
+      it.cur = tile * g.KB + cta_begin(g.KB, sg.parts, part);
+      it.end = tile * g.KB + cta_begin(g.KB, sg.parts, part + 1);
+    } else {
+      it.cur = cta_begin(sg.U, sg.Gp, c);
+      it.end = cta_begin(sg.U, sg.Gp, c + 1);
+    }
+  }
   return it;
 }
 __device__ __forceinline__ bool seg_next(const Gemm &g, SegIter &it, Seg &s) {
@@ -129,11 +153,14 @@ __device__ __forceinline__ bool seg_next(const Gemm &g, SegIter &it, Seg &s) {
 }
 // Pieces of a tile: they belong to consecutive CTAs first_owner .. first_owner + n - 1.
 __device__ __forceinline__ void tile_pieces(const Gemm &g, const SplitGeom &geo, int tile, int &first_owner, int &n) {
+  if (geo.parts) { first_owner = tile * geo.parts; n = geo.parts; return; }
   first_owner = unit_owner(geo.U, geo.Gp, tile * g.KB);
   n = unit_owner(geo.U, geo.Gp, tile * g.KB + g.KB - 1) - first_owner + 1;
 }
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+// barrier of one 128-thread worker group (id 1 = warps 4..7, the epilogue group; id 3 = warps 8..11)
+__device__ __forceinline__ void group_sync(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -141,11 +168,18 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
 }
 __device__ __forceinline__ float bf(const __nv_bfloat16 v) { return __bfloat162float(v); }
 
+// Debug timeline: CTA 0's first worker thread stamps slot 960 + k (only when profiling is on).
+__device__ __forceinline__ void prof_mark(const FwdArgs &a, int wt, int k) {
+  if (a.prof && wt == 0 && blockIdx.x == 0) a.prof[960 + k] = globaltimer_ns();
+}
+
 // Grid-wide barrier of the worker threads.  `epoch` counts barriers; the counter only grows.
 // If ready_bar != 0 the spinning thread then releases the activation producer for the next GEMM.
 __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, volatile int *abort_flag, int wt,
                                              uint32_t ready_bar) {
+  prof_mark(a, wt, 10);
   __threadfence();
+  prof_mark(a, wt, 11);
   worker_sync();
   ++epoch;
   if (*abort_flag) return false;
@@ -191,7 +225,7 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
                                            const Gemm *pend, const __nv_bfloat16 *gain, __nv_bfloat16 *dst, float *red,
                                            int wt) {
   constexpr int MAXV = 4;                                  // float4 slots per thread
-  constexpr int PB = 8;                                    // pieces loaded at a time per slot
+  constexpr int PB = 4;                                    // pieces loaded at a time per slot
   const int d = a.d, nvec = d >> 2;
   SplitGeom geo;
   geo.U = 1; geo.Gp = 1; geo.pieces_max = 1;
@@ -226,39 +260,38 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
       graw[j] = iv < nvec ? __ldg(reinterpret_cast<const uint2 *>(gain) + iv) : make_uint2(0u, 0u);
     }
     if (pend) {
+      // every piece of every slot in one batch of loads (a tile of these projections has <= 4 pieces)
+      int np[MAXV];
+      const float *base[MAXV];
+      int np_max = 0;
 #pragma unroll
-      for (int j0 = 0; j0 < MAXV; j0 += 2) {               // two slots at a time: all their loads in flight together
-        int np[2];
-        const float *base[2];
+      for (int j = 0; j < MAXV; ++j) {
+        const int iv = wt + 256 * j;
+        np[j] = 0;
+        base[j] = a.pieces;
+        if (iv < nvec) {
+          const int k = iv << 2, tile = k >> 7, mm = k & 127;
+          int fo;
+          tile_pieces(*pend, geo, tile, fo, np[j]);
+          base[j] = a.pieces + ((size_t)tile * geo.pieces_max * NPAD + row) * kTcBlockM + mm;
+        }
+        np_max = max(np_max, np[j]);
+      }
+      for (int p0 = 0; p0 < np_max; p0 += PB) {
+        float4 t[MAXV][PB];
 #pragma unroll
-        for (int jj = 0; jj < 2; ++jj) {
-          const int iv = wt + 256 * (j0 + jj);
-          np[jj] = 0;
-          base[jj] = a.pieces;
-          if (iv < nvec) {
-            const int k = iv << 2, tile = k >> 7, mm = k & 127;
-            int fo;
-            tile_pieces(*pend, geo, tile, fo, np[jj]);
-            base[jj] = a.pieces + ((size_t)tile * geo.pieces_max * NPAD + row) * kTcBlockM + mm;
+        for (int j = 0; j < MAXV; ++j)
+#pragma unroll
+          for (int pp = 0; pp < PB; ++pp)
+            t[j][pp] = (p0 + pp < np[j])
+                           ? __ldcg(reinterpret_cast<const float4 *>(base[j] + (size_t)(p0 + pp) * NPAD * kTcBlockM))
+                           : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < MAXV; ++j)
+#pragma unroll
+          for (int pp = 0; pp < PB; ++pp) {
+            v[j].x += t[j][pp].x; v[j].y += t[j][pp].y; v[j].z += t[j][pp].z; v[j].w += t[j][pp].w;
           }
-        }
-        for (int p0 = 0; p0 < max(np[0], np[1]); p0 += PB) {
-          float4 t[2][PB];
-#pragma unroll
-          for (int jj = 0; jj < 2; ++jj)
-#pragma unroll
-            for (int pp = 0; pp < PB; ++pp)
-              t[jj][pp] = (p0 + pp < np[jj])
-                              ? __ldcg(reinterpret_cast<const float4 *>(base[jj] + (size_t)(p0 + pp) * NPAD * kTcBlockM))
-                              : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-          for (int jj = 0; jj < 2; ++jj)
-#pragma unroll
-            for (int pp = 0; pp < PB; ++pp) {
-              v[j0 + jj].x += t[jj][pp].x; v[j0 + jj].y += t[jj][pp].y;
-              v[j0 + jj].z += t[jj][pp].z; v[j0 + jj].w += t[jj][pp].w;
-            }
-        }
       }
     }
     float ss = 0.f;
@@ -290,38 +323,51 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
   }
 }
 
-// ------------------------------------------------------------------------------ attention phase
-// Work item = (attention item, KV head, key split); online softmax per query; the last split of an
-// (item, head) to finish merges the partials and writes the attention output.
+// ------------------------------------------------------------------------------ attention phases
+// Under the weight stream every dependent global round trip costs microseconds, so the attention is
+// two phases of one load batch each.  Phase A: work item = (attention item, KV head, key split); the
+// q rows and a tile of up to kAttnTile keys (K and V) arrive together through cp.async, scores /
+// softmax / P.V run out of shared memory, the partial (o, m, l) goes to global memory.  Phase B
+// (after a grid barrier): one (row, head) per 128 threads merges the partials of its splits.
+constexpr int kAttnTile = 80;                          // keys per tile (three 32-key sub-tiles, the last partial)
+constexpr int kAttnPStride = 96;
+constexpr int kRopeCacheRows = 16;                     // rows whose cos / sin values are kept in shared memory
+constexpr int kAttnMaxSplits = 20;
+
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() {
+  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+__device__ __forceinline__ float bf_lo(unsigned w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf_hi(unsigned w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+struct PageCache { int tag_item, tag_tile; int pg[128]; };
+
 template <int HD>
-__device__ __forceinline__ void attn_phase(const FwdArgs &a, int layer, uint8_t *scratch, volatile int *flag, int wt) {
-  constexpr int DPL = HD / 32;
+__device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt) {
+  constexpr int CPR = HD / 8;                      // 16-byte chunks per row
+  constexpr int SWZ = CPR >= 8 ? 7 : CPR - 1;      // chunk swizzle mask (bank-conflict-free 16-byte reads)
+  constexpr int DPL = HD / 32;                     // output dims per lane
   const int group = a.nq / a.nkv;
   const int warp = wt >> 5, lane = wt & 31;
-  float *shQ = reinterpret_cast<float *>(scratch);                                        // [attn_rows*group][HD]
-  __nv_bfloat16 *shK = reinterpret_cast<__nv_bfloat16 *>(scratch + 16384);                // [32][HD+2]
-  __nv_bfloat16 *shV = shK + kKeyTile * (HD + 2);                                         // [32][HD]
-  float *shP = reinterpret_cast<float *>(shV + kKeyTile * HD);                            // [8][32]
-  const __nv_bfloat16 *kpool = a.layers[layer].k_pool, *vpool = a.layers[layer].v_pool;
+  __nv_bfloat16 *shK = reinterpret_cast<__nv_bfloat16 *>(scratch);             // [kAttnTile][HD], chunk-swizzled
+  __nv_bfloat16 *shV = shK + kAttnTile * HD;                                   // [kAttnTile][HD]
+  __nv_bfloat16 *shQ = shV + kAttnTile * HD;                                   // [<= 32][HD]
+  float *shP = reinterpret_cast<float *>(shQ + 32 * HD);                       // [8 warps][kAttnTile]
+  const __nv_bfloat16 *kpool = lay.k_pool, *vpool = lay.v_pool;
   const float scale = rsqrtf((float)HD);
   const int n_work = a.n_attn * a.nkv * a.n_splits;
   for (int wi = blockIdx.x; wi < n_work; wi += gridDim.x) {
+    prof_mark(a, wt, 4);
     const int split = wi % a.n_splits, kvh = (wi / a.n_splits) % a.nkv, ai = wi / (a.n_splits * a.nkv);
     const int4 it = a.attn_items[ai];
     const int row0 = it.x, nrows = it.y, seq = it.z, pos0 = it.w;
     const int kv_len = pos0 + nrows;
     const int key_lo = split * a.keys_per_split, key_hi = min(kv_len, key_lo + a.keys_per_split);
     if (key_lo >= kv_len) continue;                              // uniform over the CTA
-    const int ns_item = (kv_len + a.keys_per_split - 1) / a.keys_per_split;
     const int nqv = nrows * group;
-    worker_sync();
-    // (bf16 has no __ldcg overload: read the 16-bit pattern through L2 and widen)
-    for (int i = wt; i < nqv * HD; i += 256) {
-      int qi = i / HD, dd = i % HD;
-      int r = qi / group, g = qi % group;
-      unsigned short bits = __ldcg(reinterpret_cast<const unsigned short *>(a.q) + ((size_t)(row0 + r) * a.nq + kvh * group + g) * HD + dd);
-      shQ[i] = __uint_as_float((unsigned)bits << 16);
-    }
     float m_run[4], l_run[4], o_run[4][DPL];                     // <= 32 queries over 8 warps
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -329,107 +375,174 @@ __device__ __forceinline__ void attn_phase(const FwdArgs &a, int layer, uint8_t 
 #pragma unroll
       for (int e = 0; e < DPL; ++e) o_run[i][e] = 0.f;
     }
-    for (int kt = key_lo; kt < key_hi; kt += kKeyTile) {
-      worker_sync();
-      for (int i = wt; i < kKeyTile * (HD / 2); i += 256) {
-        int kk = i / (HD / 2), w2 = i % (HD / 2);
-        int key = kt + kk;
-        unsigned kb2 = 0u, vb2 = 0u;
-        if (key < key_hi) {
-          int pg = a.page_table[(size_t)seq * a.pages_per_seq + key / a.page];
-          size_t off = (((size_t)pg * a.nkv + kvh) * a.page + (key % a.page)) * HD + 2 * w2;
-          kb2 = __ldcg(reinterpret_cast<const unsigned *>(kpool + off));
-          vb2 = __ldcg(reinterpret_cast<const unsigned *>(vpool + off));
-        }
-        *reinterpret_cast<unsigned *>(shK + kk * (HD + 2) + 2 * w2) = kb2;
-        *reinterpret_cast<unsigned *>(shV + kk * HD + 2 * w2) = vb2;
+    for (int kt = key_lo, tile = 0; kt < key_hi; kt += kAttnTile, ++tile) {
+      const int nk = min(kAttnTile, key_hi - kt);
+      const int pi0 = kt >> a.page_shift, n_pg = ((kt + nk - 1) >> a.page_shift) - pi0 + 1;
+      worker_sync();                                             // previous tile / item fully consumed
+      if (!(pc->tag_item == wi && pc->tag_tile == tile)) {       // page ids of this tile (kept across layers)
+        if (wt < n_pg) pc->pg[wt] = a.page_table[(size_t)seq * a.pages_per_seq + pi0 + wt];
+        worker_sync();
+        if (wt == 0 && wi == (int)blockIdx.x && tile == 0) { pc->tag_item = wi; pc->tag_tile = 0; }
+        else if (wt == 0) { pc->tag_item = -1; }
       }
+      if (tile == 0)
+        for (int i = wt; i < nqv * CPR; i += 256) {
+          const int qi = i / CPR, ch = i % CPR;
+          const int r = qi / group, g = qi % group;
+          cp_async16(shQ + qi * HD + ch * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + g) * HD + ch * 8);
+        }
+      for (int i = wt; i < nk * CPR; i += 256) {
+        const int kk = i / CPR, ch = i % CPR;
+        const int key = kt + kk;
+        const int pg = pc->pg[(key >> a.page_shift) - pi0];
+        const size_t off = ((((size_t)pg * a.nkv + kvh) << a.page_shift) + (key & (a.page - 1))) * HD + ch * 8;
+        cp_async16(shK + kk * HD + ((ch ^ (kk & SWZ)) * 8), kpool + off);
+        cp_async16(shV + kk * HD + ch * 8, vpool + off);
+      }
+      prof_mark(a, wt, 5);
+      cp_async_wait_all();
       worker_sync();
+      prof_mark(a, wt, 6);
       int qslot = 0;
       for (int qi = warp; qi < nqv; qi += 8, ++qslot) {
         const int qpos = pos0 + qi / group;
-        const int key = kt + lane;
-        const float *qv = shQ + qi * HD;
-        const __nv_bfloat16 *kr = shK + lane * (HD + 2);
-        float sc = 0.f;
-#pragma unroll 8
-        for (int dd = 0; dd < HD; dd += 2) {
-          unsigned kk2 = *reinterpret_cast<const unsigned *>(kr + dd);
-          sc = fmaf(qv[dd], __uint_as_float(kk2 << 16), sc);
-          sc = fmaf(qv[dd + 1], __uint_as_float(kk2 & 0xFFFF0000u), sc);
+        const uint4 *q4 = reinterpret_cast<const uint4 *>(shQ + qi * HD);
+        float sc[3];
+        float mx = -INFINITY;
+        {
+          // three 32-key sub-tiles at once, two accumulators each: six independent FMA chains
+          float acc[3][2];
+          const __nv_bfloat16 *krow[3];
+          int ksw[3];
+#pragma unroll
+          for (int j = 0; j < 3; ++j) {
+            const int kk = j * 32 + lane;
+            const int kr = kk < nk ? kk : nk - 1;                 // clamp: rows past the tile hold nothing
+            krow[j] = shK + kr * HD;
+            ksw[j] = kr & SWZ;
+            acc[j][0] = acc[j][1] = 0.f;
+          }
+#pragma unroll
+          for (int ch = 0; ch < CPR; ++ch) {
+            const uint4 qv = q4[ch];
+            const float q0 = bf_lo(qv.x), q1 = bf_hi(qv.x), q2 = bf_lo(qv.y), q3 = bf_hi(qv.y);
+            const float q4f = bf_lo(qv.z), q5 = bf_hi(qv.z), q6 = bf_lo(qv.w), q7 = bf_hi(qv.w);
+#pragma unroll
+            for (int j = 0; j < 3; ++j) {
+              if (j * 32 < nk) {
+                const uint4 kv = *reinterpret_cast<const uint4 *>(krow[j] + ((ch ^ ksw[j]) * 8));
+                acc[j][0] = fmaf(q0, bf_lo(kv.x), acc[j][0]); acc[j][1] = fmaf(q1, bf_hi(kv.x), acc[j][1]);
+                acc[j][0] = fmaf(q2, bf_lo(kv.y), acc[j][0]); acc[j][1] = fmaf(q3, bf_hi(kv.y), acc[j][1]);
+                acc[j][0] = fmaf(q4f, bf_lo(kv.z), acc[j][0]); acc[j][1] = fmaf(q5, bf_hi(kv.z), acc[j][1]);
+                acc[j][0] = fmaf(q6, bf_lo(kv.w), acc[j][0]); acc[j][1] = fmaf(q7, bf_hi(kv.w), acc[j][1]);
+              }
+            }
+          }
+#pragma unroll
+          for (int j = 0; j < 3; ++j) {
+            const int kk = j * 32 + lane;
+            float v = (acc[j][0] + acc[j][1]) * scale;
+            if (kk >= nk || kt + kk > qpos) v = -INFINITY;
+            sc[j] = v;
+            mx = fmaxf(mx, v);
+          }
         }
-        sc *= scale;
-        if (key >= key_hi || key > qpos) sc = -INFINITY;
-        float mx = sc;
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
         const float m_new = fmaxf(m_run[qslot], mx);
-        float p = 0.f, corr = 1.f;
-        if (m_new > -INFINITY) {
-          p = __expf(sc - m_new);
-          corr = __expf(m_run[qslot] - m_new);
+        float corr = 1.f, ps = 0.f;
+        if (m_new > -INFINITY) corr = __expf(m_run[qslot] - m_new);
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {
+          const float p = (m_new > -INFINITY) ? __expf(sc[j] - m_new) : 0.f;
+          ps += p;
+          shP[warp * kAttnPStride + j * 32 + lane] = p;
         }
-        float ps = p;
         for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xFFFFFFFFu, ps, o);
         l_run[qslot] = l_run[qslot] * corr + ps;
         m_run[qslot] = m_new;
-        shP[warp * kKeyTile + lane] = p;
         __syncwarp();
 #pragma unroll
         for (int e = 0; e < DPL; ++e) o_run[qslot][e] *= corr;
-        for (int kk = 0; kk < kKeyTile; ++kk) {
-          const float pk = shP[warp * kKeyTile + kk];
+        {
+          float oe[2][DPL];
 #pragma unroll
-          for (int e = 0; e < DPL; ++e) o_run[qslot][e] = fmaf(pk, bf(shV[kk * HD + lane + 32 * e]), o_run[qslot][e]);
+          for (int e = 0; e < DPL; ++e) oe[0][e] = oe[1][e] = 0.f;
+          const float *pw = shP + warp * kAttnPStride;
+          const int nk2 = (nk + 1) & ~1;                         // P is zero past nk (masked scores)
+#pragma unroll 4
+          for (int kk = 0; kk < nk2; kk += 2) {
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+              const float pk = pw[kk + u];
+              const __nv_bfloat16 *vr = shV + min(kk + u, nk - 1) * HD + lane * DPL;   // odd tail: P is 0, row must be valid
+              if (DPL == 4) {
+                const uint2 vv = *reinterpret_cast<const uint2 *>(vr);
+                oe[u][0] = fmaf(pk, bf_lo(vv.x), oe[u][0]);
+                oe[u][1] = fmaf(pk, bf_hi(vv.x), oe[u][1]);
+                oe[u][2] = fmaf(pk, bf_lo(vv.y), oe[u][2]);
+                oe[u][3] = fmaf(pk, bf_hi(vv.y), oe[u][3]);
+              } else {
+#pragma unroll
+                for (int e = 0; e < DPL; ++e) oe[u][e] = fmaf(pk, bf(vr[e]), oe[u][e]);
+              }
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < DPL; ++e) o_run[qslot][e] += oe[0][e] + oe[1][e];
         }
         __syncwarp();
       }
     }
-    {
-      int qslot = 0;
-      for (int qi = warp; qi < nqv; qi += 8, ++qslot) {
-        int r = row0 + qi / group, h = kvh * group + qi % group;
-        float *dst = a.attn_partials + (((size_t)r * a.nq + h) * a.n_splits + split) * (HD + 2);
+    prof_mark(a, wt, 7);
+    int qslot = 0;
+    for (int qi = warp; qi < nqv; qi += 8, ++qslot) {
+      const int r = row0 + qi / group, h = kvh * group + qi % group;
+      float *dst = a.attn_partials + (((size_t)r * a.nq + h) * a.n_splits + split) * (HD + 2);
 #pragma unroll
-        for (int e = 0; e < DPL; ++e) dst[lane + 32 * e] = o_run[qslot][e];
-        if (lane == 0) { dst[HD] = m_run[qslot]; dst[HD + 1] = l_run[qslot]; }
-      }
+      for (int e = 0; e < DPL; ++e) dst[lane * DPL + e] = o_run[qslot][e];
+      if (lane == 0) { dst[HD] = m_run[qslot]; dst[HD + 1] = l_run[qslot]; }
     }
-    __threadfence();
-    worker_sync();
-    if (wt == 0) {
-      int prev = atomicAdd(&a.attn_counters[ai * a.nkv + kvh], 1);
-      int last = (prev == ns_item - 1);
-      if (last) a.attn_counters[ai * a.nkv + kvh] = 0;
-      *flag = last;
-      __threadfence();
+  }
+}
+
+// Phase B: merge the split partials of one (row, head) per 128 threads; a single batch of loads.
+template <int HD>
+__device__ __forceinline__ void attn_merge_phase(const FwdArgs &a, const int *row_pos_sh, int wt) {
+  const int half = wt >> 7, dd = wt & 127;
+  const int n_items = a.R * a.nq;
+  for (int it = blockIdx.x * 2 + half; it < n_items; it += 2 * gridDim.x) {
+    if (dd >= HD) continue;
+    const int r = it / a.nq;
+    const int used = min(a.n_splits, row_pos_sh[r] / a.keys_per_split + 1);   // splits holding keys <= own position
+    const float *src = a.attn_partials + (size_t)it * a.n_splits * (HD + 2);
+    float ms[kAttnMaxSplits], ls[kAttnMaxSplits], os[kAttnMaxSplits];
+#pragma unroll
+    for (int s = 0; s < kAttnMaxSplits; ++s) {
+      const bool on = s < used;
+      ms[s] = on ? __ldcg(src + s * (HD + 2) + HD) : -INFINITY;
+      ls[s] = on ? __ldcg(src + s * (HD + 2) + HD + 1) : 0.f;
+      os[s] = on ? __ldcg(src + s * (HD + 2) + dd) : 0.f;
     }
-    worker_sync();
-    if (*flag) {
-      for (int i = wt; i < nqv * HD; i += 256) {
-        int qi = i / HD, dd = i % HD;
-        int r = row0 + qi / group, h = kvh * group + qi % group;
-        int used = min(ns_item, (pos0 + qi / group) / a.keys_per_split + 1);
-        const float *src = a.attn_partials + ((size_t)r * a.nq + h) * a.n_splits * (HD + 2);
-        float m = -INFINITY;
-        for (int s = 0; s < used; ++s) m = fmaxf(m, __ldcg(src + s * (HD + 2) + HD));
-        float l = 0.f, o = 0.f;
-        for (int s = 0; s < used; ++s) {
-          float ms = __ldcg(src + s * (HD + 2) + HD);
-          float w = (ms > -INFINITY) ? __expf(ms - m) : 0.f;
-          l += w * __ldcg(src + s * (HD + 2) + HD + 1);
-          o += w * __ldcg(src + s * (HD + 2) + dd);
-        }
-        a.att[((size_t)r * a.nq + h) * HD + dd] = __float2bfloat16_rn(o / l);
-      }
+    float m = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < kAttnMaxSplits; ++s) m = fmaxf(m, ms[s]);
+    float l = 0.f, o = 0.f;
+#pragma unroll
+    for (int s = 0; s < kAttnMaxSplits; ++s) {
+      const float w = (ms[s] > -INFINITY) ? __expf(ms[s] - m) : 0.f;
+      l += w * ls[s];
+      o += w * os[s];
     }
+    a.att[(size_t)it * HD + dd] = __float2bfloat16_rn(o / l);
   }
 }
 
 // ------------------------------------------------------------------------------ epilogue stores
 // v[i] = final value of output feature (tile row m) for token row c0 + i.
 template <int CH>
-__device__ __forceinline__ void final_store(const FwdArgs &a, const Gemm &g, const Tile &ti, int layer, int m, int et,
-                                            int c0, const float *v, float *staging) {
+__device__ __forceinline__ void final_store(const FwdArgs &a, const Gemm &g, const Tile &ti, const FwdLayerDev &lay, int m, int et,
+                                            int c0, const float *v, float *staging, const int *rpos, const int *rpg,
+                                            const float *cs, const float *sn, int bar_id) {
   const int rows = g.rows;
   if (g.mode == MODE_ADD) {
     // residual-add projections never get here: their pieces are summed by the next norm phase
@@ -445,7 +558,7 @@ __device__ __forceinline__ void final_store(const FwdArgs &a, const Gemm &g, con
   } else if (g.mode == MODE_SWIGLU) {
 #pragma unroll
     for (int i = 0; i < CH; ++i) staging[m * (CH + 1) + i] = v[i];
-    epi_sync();
+    group_sync(bar_id);
     for (int idx = et; idx < kTcBoxRows * CH; idx += 128) {
       const int cc = idx % kTcBoxRows, i = idx / kTcBoxRows;
       const int r = c0 + i, col = ti.row0 + cc;
@@ -454,11 +567,12 @@ __device__ __forceinline__ void final_store(const FwdArgs &a, const Gemm &g, con
         a.act[(size_t)r * a.ff + col] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * up);
       }
     }
-    epi_sync();
-  } else {   // MODE_QKV: rotary embedding on q and k, then q -> buffer, k / v -> their cache pages
+    group_sync(bar_id);
+  } else {   // MODE_QKV: rotary embedding on q and k (cos / sin preloaded by the caller), then q -> buffer,
+             // k / v -> their cache pages (row position and page id come from the per-launch row table)
 #pragma unroll
     for (int i = 0; i < CH; ++i) staging[m * (CH + 1) + i] = v[i];
-    epi_sync();
+    group_sync(bar_id);
     const int n = ti.row0 + m;
     if (n < g.seg_n[ti.seg]) {
       const int hd = a.hd, half = hd >> 1;
@@ -468,26 +582,137 @@ __device__ __forceinline__ void final_store(const FwdArgs &a, const Gemm &g, con
       for (int i = 0; i < CH; ++i) {
         const int r = c0 + i;
         if (r < rows) {
-          const int pos = a.row_pos[r];
           float out = v[i];
           if (ti.seg < 2) {
             const float pv = staging[mp * (CH + 1) + i];
-            const float cs = a.cos_tab[(size_t)pos * half + (dd % half)], sn = a.sin_tab[(size_t)pos * half + (dd % half)];
-            out = dd < half ? v[i] * cs - pv * sn : v[i] * cs + pv * sn;
+            out = dd < half ? v[i] * cs[i] - pv * sn[i] : v[i] * cs[i] + pv * sn[i];
           }
           if (ti.seg == 0) {
             a.q[(size_t)r * g.seg_n[0] + n] = __float2bfloat16_rn(out);
           } else {
-            const int pg = a.page_table[(size_t)a.row_seq[r] * a.pages_per_seq + pos / a.page];
-            const size_t off = (((size_t)pg * a.nkv + head) * a.page + (pos % a.page)) * hd + dd;
-            (ti.seg == 1 ? a.layers[layer].k_pool : a.layers[layer].v_pool)[off] = __float2bfloat16_rn(out);
+            const size_t off = (((size_t)rpg[r] * a.nkv + head) * a.page + (rpos[r] & (a.page - 1))) * hd + dd;
+            (ti.seg == 1 ? lay.k_pool : lay.v_pool)[off] = __float2bfloat16_rn(out);
           }
         }
       }
     }
-    epi_sync();
+    group_sync(bar_id);
   }
 }
+
+struct WorkerCtx {
+  uint32_t tmem_base, accf_bar0, acce_bar0;      // accumulator-full / -empty barrier b = base + 8 b
+  volatile int *abort_flag, *wait_ok;
+  float *staging;
+  const int *row_pos_sh, *row_pg_sh;
+  const FwdLayerDev *layers_sh;
+  const float *rope_cos_sh, *rope_sin_sh;
+  int wt, lane, q, G, c;
+  int seg_idx;
+};
+
+// GEMM phase p, epilogue side (warps 4..7): accumulator -> this CTA's piece of the tile.  Group-uniform:
+// a give-up is decided by one thread and shared. 
+
+template <int NPAD>
+__device__ __forceinline__ void gemm_epilogue(const FwdArgs &a, WorkerCtx &w, int p) {
+  constexpr int CH = PCfg<NPAD>::kChunk;
+  const int m = w.q * 32 + w.lane;
+
+    const Gemm g = make_gemm(a, p);
+    const SplitGeom geo = split_geom(g, w.G);
+    SegIter it = seg_begin(g, w.G, w.c);
+    Seg sg;
+    for (; seg_next(g, it, sg); ++w.seg_idx) {
+      const int ab = w.seg_idx & 1;
+      if (w.wt == 0) w.wait_ok[w.seg_idx & 1] = mbar_wait((w.accf_bar0 + 8u * ab), (uint32_t)((w.seg_idx >> 1) & 1), w.abort_flag) ? 1 : 0;
+      epi_sync();
+      if (!w.wait_ok[w.seg_idx & 1]) return;
+      tc_fence_after();
+      const uint32_t tbase = w.tmem_base + ((uint32_t)(w.q * 32) << 16) + (uint32_t)(ab * NPAD);
+      // this CTA's piece of the tile; the next phase sums the pieces
+      int fo, np_tile;
+      tile_pieces(g, geo, sg.tile, fo, np_tile);
+      const int piece = w.c - fo;
+      float *mine = a.pieces + ((size_t)sg.tile * geo.pieces_max + piece) * NPAD * kTcBlockM;
+#pragma unroll 1
+      for (int c0 = 0; c0 < NPAD; c0 += CH) {
+        float v[CH];
+#pragma unroll
+        for (int j = 0; j < CH / 16; ++j) tmem_ld16(tbase + c0 + j * 16, v + j * 16);
+        tmem_ld_wait();
+        if (c0 + CH >= NPAD) {                   // accumulator fully read: hand it back to the MMA warp
+          tc_fence_before();
+          __syncwarp();
+          if (w.lane == 0) mbar_arrive((w.acce_bar0 + 8u * ab));
+        }
+        if (c0 < g.rows) {
+#pragma unroll
+          for (int i = 0; i < CH; ++i)
+            if (c0 + i < g.rows) mine[(c0 + i) * kTcBlockM + m] = v[i];
+        }
+      }
+    }
+  }
+
+// Finish phase of GEMM p (QKV, gate/up, output head): tiles round-robin over the CTAs, two at a time
+// (one per 128-thread group); the pieces of a tile are added in piece order and the result goes
+// through the projection's own epilogue.  All loads of a chunk are issued before the first use.
+template <int NPAD>
+__device__ __forceinline__ void gemm_finish(const FwdArgs &a, WorkerCtx &w, int p) {
+  constexpr int CH = PCfg<NPAD>::kChunk;
+
+    constexpr int PBF = CH > 16 ? 2 : 4;
+    const Gemm g = make_gemm(a, p);
+    const SplitGeom geo = split_geom(g, w.G);
+    const int layer = p >> 2;
+    const int gidx = w.wt >> 7, gm = w.wt & 127;       // two groups of 128 threads, one tile each at a time
+    float *gstage = w.staging + gidx * (kTcBlockM * (CH + 1));
+    for (int tile = w.c + gidx * w.G; tile < g.n_tiles; tile += 2 * w.G) {
+      if (g.mode == MODE_QKV) prof_mark(a, w.wt, 0);
+      const Tile ti = tile_of(g, tile);
+      int fo, n_pieces;
+      tile_pieces(g, geo, tile, fo, n_pieces);
+      const float *base = a.pieces + (size_t)tile * geo.pieces_max * NPAD * kTcBlockM + gm;
+#pragma unroll 1
+      for (int c0 = 0; c0 < NPAD && c0 < g.rows; c0 += CH) {
+        float v[CH], cs[CH], sn[CH];
+#pragma unroll
+        for (int i = 0; i < CH; ++i) { v[i] = 0.f; cs[i] = 1.f; sn[i] = 0.f; }
+        if (g.mode == MODE_QKV && ti.seg < 2) {
+          const int half = a.hd >> 1, dh = ((ti.row0 + gm) % a.hd) % half;
+#pragma unroll
+          for (int i = 0; i < CH; ++i)
+            if (c0 + i < g.rows) {
+              if (a.R <= kRopeCacheRows) {
+                cs[i] = w.rope_cos_sh[(c0 + i) * half + dh];
+                sn[i] = w.rope_sin_sh[(c0 + i) * half + dh];
+              } else {
+                cs[i] = __ldg(a.cos_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
+                sn[i] = __ldg(a.sin_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
+              }
+            }
+        }
+        for (int p0 = 0; p0 < n_pieces; p0 += PBF) {
+          float t[PBF][CH];
+#pragma unroll
+          for (int pp = 0; pp < PBF; ++pp)
+#pragma unroll
+            for (int i = 0; i < CH; ++i)
+              t[pp][i] = (p0 + pp < n_pieces && c0 + i < g.rows)
+                             ? __ldcg(base + ((size_t)(p0 + pp) * NPAD + c0 + i) * kTcBlockM)
+                             : 0.f;
+#pragma unroll
+          for (int pp = 0; pp < PBF; ++pp)
+#pragma unroll
+            for (int i = 0; i < CH; ++i) v[i] += t[pp][i];
+        }
+        if (g.mode == MODE_QKV) prof_mark(a, w.wt, 1);
+        final_store<CH>(a, g, ti, w.layers_sh[layer < a.n_run ? layer : 0], gm, gm, c0, v, gstage, w.row_pos_sh, w.row_pg_sh, cs, sn, 1 + 2 * gidx);
+        if (g.mode == MODE_QKV) prof_mark(a, w.wt, 2);
+      }
+    }
+  }
 
 template <int NPAD, int HD>
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __grid_constant__ FwdArgs a) {
@@ -506,6 +731,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   volatile int *last_flag = reinterpret_cast<volatile int *>(ctl + 2);
   volatile int *wait_ok = reinterpret_cast<volatile int *>(ctl + 4);   // [2]
   float *red = reinterpret_cast<float *>(ctl + 8);                      // [8]
+  PageCache *pcache = reinterpret_cast<PageCache *>(ctl + 16);          // 130 words
+  int *row_pos_sh = reinterpret_cast<int *>(ctl + 160);                 // [128] position of each packed row
+  int *row_pg_sh = reinterpret_cast<int *>(ctl + 288);                  // [128] KV page holding that position
+  FwdLayerDev *layers_sh = reinterpret_cast<FwdLayerDev *>(ctl + 416);  // [<= kMaxLayersSh] pointer table
+  // cos / sin of the launch's rows (the tables are touched once per layer, so the weight stream would
+  // evict them from L2 between uses): [kRopeCacheRows][hd / 2] each, after the attention / staging area
+  float *rope_cos_sh = reinterpret_cast<float *>(scratch + kScratchBytes - 2 * kRopeCacheRows * (HD / 2) * 4);
+  float *rope_sin_sh = rope_cos_sh + kRopeCacheRows * (HD / 2);
   const uint32_t bar0 = smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
@@ -522,6 +755,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); mbar_init(ready_bar(b), 1); }
     *abort_flag = 0;
     *last_flag = 0;
+    pcache->tag_item = -1;
+    pcache->tag_tile = -1;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
@@ -629,80 +864,35 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     // ------------------------------------------------------------ workers (+ epilogue: warps 4..7)
     const int wt = threadIdx.x - 128;              // 0..255
     const bool is_epi = warp < 8;
-    const int et = wt;                             // 0..127 for the epilogue warps
     const int q = warp & 3, m = q * 32 + lane;
     float *staging = reinterpret_cast<float *>(scratch);
     unsigned epoch = 0;
     int seg_idx = 0;
     bool alive = true;
 
-    // GEMM phase p, epilogue side.  Group-uniform: a give-up is decided by one thread and shared.
-    auto epilogue = [&](int p) {
-      const Gemm g = make_gemm(a, p);
-      const SplitGeom geo = split_geom(g, G);
-      SegIter it = seg_begin(g, G, c);
-      Seg sg;
-      for (; seg_next(g, it, sg); ++seg_idx) {
-        const int ab = seg_idx & 1;
-        if (et == 0) wait_ok[seg_idx & 1] = mbar_wait(accf_bar(ab), (uint32_t)((seg_idx >> 1) & 1), abort_flag) ? 1 : 0;
-        epi_sync();
-        if (!wait_ok[seg_idx & 1]) return;
-        tc_fence_after();
-        const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * NPAD);
-        // this CTA's piece of the tile; the next phase sums the pieces
-        const int piece = c - unit_owner(geo.U, geo.Gp, sg.tile * g.KB);
-        float *mine = a.pieces + ((size_t)sg.tile * geo.pieces_max + piece) * NPAD * kTcBlockM;
-#pragma unroll 1
-        for (int c0 = 0; c0 < NPAD; c0 += CH) {
-          float v[CH];
-#pragma unroll
-          for (int j = 0; j < CH / 16; ++j) tmem_ld16(tbase + c0 + j * 16, v + j * 16);
-          tmem_ld_wait();
-          if (c0 + CH >= NPAD) {                   // accumulator fully read: hand it back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acce_bar(ab));
-          }
-          if (c0 < g.rows) {
-#pragma unroll
-            for (int i = 0; i < CH; ++i)
-              if (c0 + i < g.rows) mine[(c0 + i) * kTcBlockM + m] = v[i];
-          }
-        }
-      }
-    };
-
-    // Finish phase of GEMM p (QKV, gate/up, output head): tiles round-robin over the CTAs; the pieces of
-    // a tile are added in piece order and the result goes through the projection's own epilogue.
-    auto finish = [&](int p) {
-      const Gemm g = make_gemm(a, p);
-      const SplitGeom geo = split_geom(g, G);
-      const int layer = p >> 2;
-      for (int tile = c; tile < g.n_tiles; tile += G) {
-        const Tile ti = tile_of(g, tile);
-        int fo, n_pieces;
-        tile_pieces(g, geo, tile, fo, n_pieces);
-        const float *base = a.pieces + (size_t)tile * geo.pieces_max * NPAD * kTcBlockM + m;
-#pragma unroll 1
-        for (int c0 = 0; c0 < NPAD && c0 < g.rows; c0 += CH) {
-          float v[CH];
-#pragma unroll
-          for (int i = 0; i < CH; ++i) v[i] = 0.f;
-          for (int pc = 0; pc < n_pieces; ++pc) {
-            float t[CH];
-#pragma unroll
-            for (int i = 0; i < CH; ++i)
-              t[i] = (c0 + i < g.rows) ? __ldcg(base + ((size_t)pc * NPAD + c0 + i) * kTcBlockM) : 0.f;
-#pragma unroll
-            for (int i = 0; i < CH; ++i) v[i] += t[i];
-          }
-          final_store<CH>(a, g, ti, layer, m, et, c0, v, staging);
-        }
-      }
-    };
+    WorkerCtx w;
+    w.tmem_base = tmem_base; w.accf_bar0 = accf_bar(0); w.acce_bar0 = acce_bar(0);
+    w.abort_flag = abort_flag; w.wait_ok = wait_ok; w.staging = staging;
+    w.row_pos_sh = row_pos_sh; w.row_pg_sh = row_pg_sh; w.layers_sh = layers_sh;
+    w.rope_cos_sh = rope_cos_sh; w.rope_sin_sh = rope_sin_sh;
+    w.wt = wt; w.lane = lane; w.q = q; w.G = G; w.c = c; w.seg_idx = 0;
+    auto epilogue = [&](int p) { gemm_epilogue<NPAD>(a, w, p); };
+    auto finish = [&](int p) { gemm_finish<NPAD>(a, w, p); };
 
     // ---- phase program
     if (a.prof && wt == 0) a.prof[(size_t)blockIdx.x * kFwdProfEvents] = globaltimer_ns();
+    for (int l = wt; l < a.n_run; l += 256) layers_sh[l] = a.layers[l];
+    if (a.R <= kRopeCacheRows)
+      for (int i = wt; i < a.R * (HD / 2); i += 256) {
+        const int r = i / (HD / 2), k = i % (HD / 2);
+        rope_cos_sh[i] = a.cos_tab[(size_t)a.row_pos[r] * (HD / 2) + k];
+        rope_sin_sh[i] = a.sin_tab[(size_t)a.row_pos[r] * (HD / 2) + k];
+      }
+    for (int r = wt; r < a.R; r += 256) {             // per-row facts every layer needs, fetched once
+      const int pos = a.row_pos[r];
+      row_pos_sh[r] = pos;
+      row_pg_sh[r] = a.page_table[(size_t)a.row_seq[r] * a.pages_per_seq + pos / a.page];
+    }
     norm_phase<NPAD>(a, a.R, nullptr, true, nullptr, a.layers[0].attn_norm, a.h, red, wt);
     alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar(0));
     for (int l = 0; l < a.n_run && alive; ++l) {
@@ -710,10 +900,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       if (is_epi) epilogue(p);                                            // QKV pieces
       alive = grid_barrier(a, epoch, abort_flag, wt, 0);
       if (!alive) break;
-      if (is_epi) finish(p);                                              // sum, rope, q / KV append
+      finish(p);                                                          // sum, rope, q / KV append
       alive = grid_barrier(a, epoch, abort_flag, wt, 0);
       if (!alive) break;
-      attn_phase<HD>(a, l, scratch, last_flag, wt);
+      attn_tiles_phase<HD>(a, layers_sh[l], scratch, pcache, wt);
+      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
+      if (!alive) break;
+      attn_merge_phase<HD>(a, row_pos_sh, wt);
       alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 1) & 1));
       if (!alive) break;
       if (is_epi) epilogue(p + 1);                                        // O projection into the residual
@@ -721,14 +914,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       if (!alive) break;
       {
         const Gemm pend = make_gemm(a, p + 1);
-        norm_phase<NPAD>(a, a.R, nullptr, false, &pend, a.layers[l].mlp_norm, a.h, red, wt);
+        norm_phase<NPAD>(a, a.R, nullptr, false, &pend, layers_sh[l].mlp_norm, a.h, red, wt);
       }
       alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 2) & 1));
       if (!alive) break;
       if (is_epi) epilogue(p + 2);                                        // gate / up pieces
       alive = grid_barrier(a, epoch, abort_flag, wt, 0);
       if (!alive) break;
-      if (is_epi) finish(p + 2);                                          // sum, SwiGLU
+      finish(p + 2);                                                      // sum, SwiGLU
       alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 3) & 1));
       if (!alive) break;
       if (is_epi) epilogue(p + 3);                                        // down projection into the residual
@@ -736,7 +929,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         alive = grid_barrier(a, epoch, abort_flag, wt, 0);
         if (!alive) break;
         const Gemm pend = make_gemm(a, p + 3);
-        if (l + 1 < a.n_run) norm_phase<NPAD>(a, a.R, nullptr, false, &pend, a.layers[l + 1].attn_norm, a.h, red, wt);
+        if (l + 1 < a.n_run) norm_phase<NPAD>(a, a.R, nullptr, false, &pend, layers_sh[l + 1].attn_norm, a.h, red, wt);
         else norm_phase<NPAD>(a, a.L, a.lrow_src, false, &pend, a.final_norm, a.hf, red, wt);
         alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 4) & 1));
       }
@@ -744,7 +937,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     if (alive && a.L > 0) {                                               // output head
       if (is_epi) epilogue(4 * a.n_run);
       alive = grid_barrier(a, epoch, abort_flag, wt, 0);
-      if (alive && is_epi) finish(4 * a.n_run);
+      if (alive) finish(4 * a.n_run);
     }
   }
   // ------------------------------------------------------------------ teardown
@@ -789,6 +982,7 @@ bool fwd_persist_supported(int hd, int group) {
 
 int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaStream_t s) {
   if (args.R < 1 || args.R > npad || args.L > npad) return HSD_E_INVALID_ARG;
+  if (args.n_run > kMaxLayersSh) return HSD_E_UNSUPPORTED;
   {  // unit arithmetic on the device is 32-bit
     long long tiles = std::max<long long>((args.V + 127) / 128, (args.ff + 63) / 64);
     long long kb = std::max(args.ff, std::max(args.d, args.nq * args.hd)) / kTcBlockK;
