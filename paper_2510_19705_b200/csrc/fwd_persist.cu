@@ -422,7 +422,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
             ksw[j] = kr & SWZ;
             acc[j][0] = acc[j][1] = 0.f;
           }
-#pragma unroll
+#pragma unroll 2
           for (int ch = 0; ch < CPR; ++ch) {
             const uint4 qv = q4[ch];
             const float q0 = bf_lo(qv.x), q1 = bf_hi(qv.x), q2 = bf_lo(qv.y), q3 = bf_hi(qv.y);
@@ -491,6 +491,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
           for (int e = 0; e < DPL; ++e) o_run[qslot][e] += oe[0][e] + oe[1][e];
         }
         __syncwarp();
+        prof_mark(a, wt, 8 + (qslot > 0 ? 1 : 0));
       }
     }
     prof_mark(a, wt, 7);
@@ -660,59 +661,62 @@ __device__ __forceinline__ void gemm_epilogue(const FwdArgs &a, WorkerCtx &w, in
 // through the projection's own epilogue.  All loads of a chunk are issued before the first use.
 template <int NPAD>
 __device__ __forceinline__ void gemm_finish(const FwdArgs &a, WorkerCtx &w, int p) {
-  constexpr int CH = PCfg<NPAD>::kChunk;
-
-    constexpr int PBF = CH > 16 ? 2 : 4;
-    const Gemm g = make_gemm(a, p);
-    const SplitGeom geo = split_geom(g, w.G);
-    const int layer = p >> 2;
-    const int gidx = w.wt >> 7, gm = w.wt & 127;       // two groups of 128 threads, one tile each at a time
-    float *gstage = w.staging + gidx * (kTcBlockM * (CH + 1));
-    for (int tile = w.c + gidx * w.G; tile < g.n_tiles; tile += 2 * w.G) {
-      if (g.mode == MODE_QKV) prof_mark(a, w.wt, 0);
-      const Tile ti = tile_of(g, tile);
-      int fo, n_pieces;
-      tile_pieces(g, geo, tile, fo, n_pieces);
-      const float *base = a.pieces + (size_t)tile * geo.pieces_max * NPAD * kTcBlockM + gm;
+  constexpr int RG = 4;                          // token rows per load batch (decode passes have few rows)
+  constexpr int PBF = 4;                         // pieces per load batch
+  const Gemm g = make_gemm(a, p);
+  const SplitGeom geo = split_geom(g, w.G);
+  const int layer = p >> 2;
+  const int gidx = w.wt >> 7, gm = w.wt & 127;   // two groups of 128 threads, one tile each at a time
+  float *gstage = w.staging + gidx * (kTcBlockM * (RG + 1));
 #pragma unroll 1
-      for (int c0 = 0; c0 < NPAD && c0 < g.rows; c0 += CH) {
-        float v[CH], cs[CH], sn[CH];
+  for (int tile = w.c + gidx * w.G; tile < g.n_tiles; tile += 2 * w.G) {
+    if (g.mode == MODE_QKV) prof_mark(a, w.wt, 0);
+    const Tile ti = tile_of(g, tile);
+    int fo, n_pieces;
+    tile_pieces(g, geo, tile, fo, n_pieces);
+    const float *base = a.pieces + (size_t)tile * geo.pieces_max * NPAD * kTcBlockM + gm;
+    const int half = a.hd >> 1, dh = ((ti.row0 + gm) % a.hd) % half;
+    const bool rope = (g.mode == MODE_QKV && ti.seg < 2);
+#pragma unroll 1
+    for (int c0 = 0; c0 < g.rows; c0 += RG) {
+      float v[RG], cs[RG], sn[RG];
 #pragma unroll
-        for (int i = 0; i < CH; ++i) { v[i] = 0.f; cs[i] = 1.f; sn[i] = 0.f; }
-        if (g.mode == MODE_QKV && ti.seg < 2) {
-          const int half = a.hd >> 1, dh = ((ti.row0 + gm) % a.hd) % half;
+      for (int i = 0; i < RG; ++i) { v[i] = 0.f; cs[i] = 1.f; sn[i] = 0.f; }
+      if (rope) {
 #pragma unroll
-          for (int i = 0; i < CH; ++i)
-            if (c0 + i < g.rows) {
-              if (a.R <= kRopeCacheRows) {
-                cs[i] = w.rope_cos_sh[(c0 + i) * half + dh];
-                sn[i] = w.rope_sin_sh[(c0 + i) * half + dh];
-              } else {
-                cs[i] = __ldg(a.cos_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
-                sn[i] = __ldg(a.sin_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
-              }
+        for (int i = 0; i < RG; ++i)
+          if (c0 + i < g.rows) {
+            if (a.R <= kRopeCacheRows) {
+              cs[i] = w.rope_cos_sh[(c0 + i) * half + dh];
+              sn[i] = w.rope_sin_sh[(c0 + i) * half + dh];
+            } else {
+              cs[i] = __ldg(a.cos_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
+              sn[i] = __ldg(a.sin_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
             }
-        }
-        for (int p0 = 0; p0 < n_pieces; p0 += PBF) {
-          float t[PBF][CH];
-#pragma unroll
-          for (int pp = 0; pp < PBF; ++pp)
-#pragma unroll
-            for (int i = 0; i < CH; ++i)
-              t[pp][i] = (p0 + pp < n_pieces && c0 + i < g.rows)
-                             ? __ldcg(base + ((size_t)(p0 + pp) * NPAD + c0 + i) * kTcBlockM)
-                             : 0.f;
-#pragma unroll
-          for (int pp = 0; pp < PBF; ++pp)
-#pragma unroll
-            for (int i = 0; i < CH; ++i) v[i] += t[pp][i];
-        }
-        if (g.mode == MODE_QKV) prof_mark(a, w.wt, 1);
-        final_store<CH>(a, g, ti, w.layers_sh[layer < a.n_run ? layer : 0], gm, gm, c0, v, gstage, w.row_pos_sh, w.row_pg_sh, cs, sn, 1 + 2 * gidx);
-        if (g.mode == MODE_QKV) prof_mark(a, w.wt, 2);
+          }
       }
+#pragma unroll 1
+      for (int p0 = 0; p0 < n_pieces; p0 += PBF) {
+        float t[PBF][RG];
+#pragma unroll
+        for (int pp = 0; pp < PBF; ++pp)
+#pragma unroll
+          for (int i = 0; i < RG; ++i)
+            t[pp][i] = (p0 + pp < n_pieces && c0 + i < g.rows)
+                           ? __ldcg(base + ((size_t)(p0 + pp) * NPAD + c0 + i) * kTcBlockM)
+                           : 0.f;
+#pragma unroll
+        for (int pp = 0; pp < PBF; ++pp)
+#pragma unroll
+          for (int i = 0; i < RG; ++i) v[i] += t[pp][i];
+      }
+      if (g.mode == MODE_QKV) prof_mark(a, w.wt, 1);
+      final_store<RG>(a, g, ti, w.layers_sh[layer < a.n_run ? layer : 0], gm, gm, c0, v, gstage, w.row_pos_sh,
+                      w.row_pg_sh, cs, sn, 1 + 2 * gidx);
+      if (g.mode == MODE_QKV) prof_mark(a, w.wt, 2);
     }
   }
+}
 
 template <int NPAD, int HD>
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __grid_constant__ FwdArgs a) {
@@ -876,8 +880,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     w.row_pos_sh = row_pos_sh; w.row_pg_sh = row_pg_sh; w.layers_sh = layers_sh;
     w.rope_cos_sh = rope_cos_sh; w.rope_sin_sh = rope_sin_sh;
     w.wt = wt; w.lane = lane; w.q = q; w.G = G; w.c = c; w.seg_idx = 0;
-    auto epilogue = [&](int p) { gemm_epilogue<NPAD>(a, w, p); };
-    auto finish = [&](int p) { gemm_finish<NPAD>(a, w, p); };
 
     // ---- phase program
     if (a.prof && wt == 0) a.prof[(size_t)blockIdx.x * kFwdProfEvents] = globaltimer_ns();
@@ -893,51 +895,60 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       row_pos_sh[r] = pos;
       row_pg_sh[r] = a.page_table[(size_t)a.row_seq[r] * a.pages_per_seq + pos / a.page];
     }
-    norm_phase<NPAD>(a, a.R, nullptr, true, nullptr, a.layers[0].attn_norm, a.h, red, wt);
-    alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar(0));
-    for (int l = 0; l < a.n_run && alive; ++l) {
-      const int p = 4 * l;
-      if (is_epi) epilogue(p);                                            // QKV pieces
-      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
-      if (!alive) break;
-      finish(p);                                                          // sum, rope, q / KV append
-      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
-      if (!alive) break;
-      attn_tiles_phase<HD>(a, layers_sh[l], scratch, pcache, wt);
-      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
-      if (!alive) break;
-      attn_merge_phase<HD>(a, row_pos_sh, wt);
-      alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 1) & 1));
-      if (!alive) break;
-      if (is_epi) epilogue(p + 1);                                        // O projection into the residual
-      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
-      if (!alive) break;
-      {
-        const Gemm pend = make_gemm(a, p + 1);
-        norm_phase<NPAD>(a, a.R, nullptr, false, &pend, layers_sh[l].mlp_norm, a.h, red, wt);
+    // One step loop, one call site per phase body: the whole per-layer program has to stay resident in
+    // the instruction cache (every phase runs once per layer, so code that does not fit is fetched
+    // cold through the saturated memory system every single time).
+    //   t = 0                embed + norm                                  -> ready(QKV 0)
+    //   t = 1 + 10 l + s     s: 0 QKV pieces | 1 QKV finish | 2 attention tiles | 3 attention merge -> ready(O)
+    //                           4 O pieces | 5 norm (+O pieces) -> ready(gate/up) | 6 gate/up pieces
+    //                           7 gate/up finish -> ready(down) | 8 down pieces | 9 norm (+down pieces) -> ready(next)
+    //   t = 1 + 10 n, + 1    output-head pieces | output-head finish
+    const int n_steps = 1 + 10 * a.n_run + (a.L > 0 ? 2 : 0);
+    enum { K_EPI, K_FIN, K_ATTN_A, K_ATTN_B, K_NORM, K_NONE };
+#pragma unroll 1
+    for (int t = 0; t < n_steps && alive; ++t) {
+      int kind, gp = 0, ready = -1, l = 0;
+      bool barrier = true;
+      if (t == 0) { kind = K_NORM; ready = 0; }
+      else if (t > 10 * a.n_run) { gp = 4 * a.n_run; kind = (t == 1 + 10 * a.n_run) ? K_EPI : K_FIN; barrier = (kind == K_EPI); }
+      else {
+        l = (t - 1) / 10;
+        const int sstep = (t - 1) % 10, p = 4 * l;
+        switch (sstep) {
+          case 0: kind = K_EPI; gp = p; break;
+          case 1: kind = K_FIN; gp = p; break;
+          case 2: kind = K_ATTN_A; break;
+          case 3: kind = K_ATTN_B; ready = p + 1; break;
+          case 4: kind = K_EPI; gp = p + 1; break;
+          case 5: kind = K_NORM; gp = p + 1; ready = p + 2; break;
+          case 6: kind = K_EPI; gp = p + 2; break;
+          case 7: kind = K_FIN; gp = p + 2; ready = p + 3; break;
+          case 8: kind = K_EPI; gp = p + 3; barrier = (l + 1 < a.n_run || a.L > 0); break;
+          default:
+            kind = (l + 1 < a.n_run || a.L > 0) ? K_NORM : K_NONE; gp = p + 3; ready = p + 4;
+            barrier = (kind == K_NORM);
+            break;
+        }
       }
-      alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 2) & 1));
-      if (!alive) break;
-      if (is_epi) epilogue(p + 2);                                        // gate / up pieces
-      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
-      if (!alive) break;
-      finish(p + 2);                                                      // sum, SwiGLU
-      alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 3) & 1));
-      if (!alive) break;
-      if (is_epi) epilogue(p + 3);                                        // down projection into the residual
-      if (l + 1 < a.n_run || a.L > 0) {
-        alive = grid_barrier(a, epoch, abort_flag, wt, 0);
-        if (!alive) break;
-        const Gemm pend = make_gemm(a, p + 3);
-        if (l + 1 < a.n_run) norm_phase<NPAD>(a, a.R, nullptr, false, &pend, layers_sh[l + 1].attn_norm, a.h, red, wt);
-        else norm_phase<NPAD>(a, a.L, a.lrow_src, false, &pend, a.final_norm, a.hf, red, wt);
-        alive = grid_barrier(a, epoch, abort_flag, wt, ready_bar((p + 4) & 1));
+      switch (kind) {
+        case K_EPI: if (is_epi) gemm_epilogue<NPAD>(a, w, gp); break;
+        case K_FIN: gemm_finish<NPAD>(a, w, gp); break;
+        case K_ATTN_A: attn_tiles_phase<HD>(a, layers_sh[l], scratch, pcache, wt); break;
+        case K_ATTN_B: attn_merge_phase<HD>(a, row_pos_sh, wt); break;
+        case K_NORM: {
+          const bool first = (t == 0);
+          const bool last = !first && (((t - 1) % 10) == 9) && (l + 1 >= a.n_run);      // final norm over the logit rows
+          const bool mid = !first && (((t - 1) % 10) == 5);
+          const Gemm pend = make_gemm(a, first ? 0 : gp);
+          const __nv_bfloat16 *gain = first ? a.layers[0].attn_norm
+                                            : (last ? a.final_norm : (mid ? layers_sh[l].mlp_norm : layers_sh[l + 1].attn_norm));
+          norm_phase<NPAD>(a, last ? a.L : a.R, last ? a.lrow_src : nullptr, first, first ? nullptr : &pend, gain,
+                           last ? a.hf : a.h, red, wt);
+          break;
+        }
+        default: break;
       }
-    }
-    if (alive && a.L > 0) {                                               // output head
-      if (is_epi) epilogue(4 * a.n_run);
-      alive = grid_barrier(a, epoch, abort_flag, wt, 0);
-      if (alive) finish(4 * a.n_run);
+      if (barrier) alive = grid_barrier(a, epoch, abort_flag, wt, ready >= 0 ? ready_bar(ready & 1) : 0u);
     }
   }
   // ------------------------------------------------------------------ teardown
