@@ -354,7 +354,7 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   const int blocks_target = c->use_persist ? c->sm_count : kAttnBlocksTarget;
   const int max_splits = c->use_persist ? 20 : kMaxSplits;      // the persistent merge phase takes <= 20 splits
   int n_splits = std::max(1, std::min(max_splits, blocks_target / std::max(1, n_attn * md.nkv)));
-  int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, kAttnKeyTile);
+  int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, c->use_persist ? 16 : kAttnKeyTile);
   n_splits = (max_kv + keys_per_split - 1) / keys_per_split;
   if ((size_t)R * n_splits > (size_t)L.partial_rows) return HSD_E_INVALID_ARG;
 

@@ -23,7 +23,7 @@ using namespace ptx;
 
 constexpr int kWBytes = kTcBlockM * kTcBlockK * 2;     // 16 KiB weight tile
 constexpr int kBoxBytes = kTcBoxRows * kTcBlockK * 2;  // 8 KiB TMA box
-constexpr int kScratchBytes = 60 * 1024;               // union: epilogue staging / attention tiles
+constexpr int kScratchBytes = 78 * 1024;               // union: epilogue staging / attention tiles, + rope cache
 constexpr int kCtrlBytes = 4096;                       // barriers, flags, page-id cache, per-row info
 constexpr int kSmemTotal = 232448;
 constexpr int kKeyTile = 32;
@@ -345,20 +345,36 @@ __device__ __forceinline__ float bf_hi(unsigned w) { return __uint_as_float(w & 
 
 struct PageCache { int tag_item, tag_tile; int pg[128]; };
 
+__device__ __forceinline__ void mma_bf16_16x8x16(float *c, const unsigned *a, unsigned b0, unsigned b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x2_trans(unsigned &r0, unsigned &r1, const void *row_ptr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(smem_u32(row_ptr)));
+}
+
+// Phase A on the (legacy) tensor path: S = Q K^T and O += P V with mma.sync m16n8k16, fp32 softmax in
+// between.  Shared memory: K, V, Q as bf16 rows padded by 16 bytes (conflict-free fragment loads),
+// S as fp32 [32][84] with P (bf16) written in place over each S row, running (m, l, corr) per query.
 template <int HD>
 __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt) {
   constexpr int CPR = HD / 8;                      // 16-byte chunks per row
-  constexpr int SWZ = CPR >= 8 ? 7 : CPR - 1;      // chunk swizzle mask (bank-conflict-free 16-byte reads)
-  constexpr int DPL = HD / 32;                     // output dims per lane
+  constexpr int RS = HD + 8;                       // padded row stride (bf16 elements)
+  constexpr int SS = 84;                           // S row stride (floats)
+  constexpr int KST = HD / 16;                     // k-steps of Q K^T
+  constexpr int NTW = (HD / 8 + 7) / 8;            // output n-tiles (8 dims) per warp
   const int group = a.nq / a.nkv;
-  const int warp = wt >> 5, lane = wt & 31;
-  __nv_bfloat16 *shK = reinterpret_cast<__nv_bfloat16 *>(scratch);             // [kAttnTile][HD], chunk-swizzled
-  __nv_bfloat16 *shV = shK + kAttnTile * HD;                                   // [kAttnTile][HD]
-  __nv_bfloat16 *shQ = shV + kAttnTile * HD;                                   // [<= 32][HD]
-  float *shP = reinterpret_cast<float *>(shQ + 32 * HD);                       // [8 warps][kAttnTile]
+  const int warp = wt >> 5, lane = wt & 31, g = lane >> 2, t = lane & 3;
+  __nv_bfloat16 *shK = reinterpret_cast<__nv_bfloat16 *>(scratch);             // [kAttnTile][RS]
+  __nv_bfloat16 *shV = shK + kAttnTile * RS;                                   // [kAttnTile][RS]
+  __nv_bfloat16 *shQ = shV + kAttnTile * RS;                                   // [32][RS]
+  float *shS = reinterpret_cast<float *>(shQ + 32 * RS);                       // [32][SS]; P in place
+  float *shM = shS + 32 * SS, *shL = shM + 32, *shC = shL + 32;                // running max, sum, correction
   const __nv_bfloat16 *kpool = lay.k_pool, *vpool = lay.v_pool;
   const float scale = rsqrtf((float)HD);
   const int n_work = a.n_attn * a.nkv * a.n_splits;
+#pragma unroll 1
   for (int wi = blockIdx.x; wi < n_work; wi += gridDim.x) {
     prof_mark(a, wt, 4);
     const int split = wi % a.n_splits, kvh = (wi / a.n_splits) % a.nkv, ai = wi / (a.n_splits * a.nkv);
@@ -367,14 +383,15 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
     const int kv_len = pos0 + nrows;
     const int key_lo = split * a.keys_per_split, key_hi = min(kv_len, key_lo + a.keys_per_split);
     if (key_lo >= kv_len) continue;                              // uniform over the CTA
-    const int nqv = nrows * group;
-    float m_run[4], l_run[4], o_run[4][DPL];                     // <= 32 queries over 8 warps
+    const int nqv = nrows * group, n_mt = (nqv + 15) >> 4;
+    float o[2][NTW][4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      m_run[i] = -INFINITY; l_run[i] = 0.f;
+    for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-      for (int e = 0; e < DPL; ++e) o_run[i][e] = 0.f;
-    }
+      for (int n = 0; n < NTW; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) o[mt][n][e] = 0.f;
+#pragma unroll 1
     for (int kt = key_lo, tile = 0; kt < key_hi; kt += kAttnTile, ++tile) {
       const int nk = min(kAttnTile, key_hi - kt);
       const int pi0 = kt >> a.page_shift, n_pg = ((kt + nk - 1) >> a.page_shift) - pi0 + 1;
@@ -382,126 +399,146 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
       if (!(pc->tag_item == wi && pc->tag_tile == tile)) {       // page ids of this tile (kept across layers)
         if (wt < n_pg) pc->pg[wt] = a.page_table[(size_t)seq * a.pages_per_seq + pi0 + wt];
         worker_sync();
-        if (wt == 0 && wi == (int)blockIdx.x && tile == 0) { pc->tag_item = wi; pc->tag_tile = 0; }
-        else if (wt == 0) { pc->tag_item = -1; }
+        if (wt == 0) pc->tag_item = (wi == (int)blockIdx.x && tile == 0) ? wi : -1, pc->tag_tile = 0;
       }
-      if (tile == 0)
+      if (tile == 0) {
         for (int i = wt; i < nqv * CPR; i += 256) {
           const int qi = i / CPR, ch = i % CPR;
-          const int r = qi / group, g = qi % group;
-          cp_async16(shQ + qi * HD + ch * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + g) * HD + ch * 8);
+          const int r = qi / group, gq = qi % group;
+          cp_async16(shQ + qi * RS + ch * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + gq) * HD + ch * 8);
         }
-      for (int i = wt; i < nk * CPR; i += 256) {
+        if (wt < 32) { shM[wt] = -INFINITY; shL[wt] = 0.f; shC[wt] = 1.f; }
+      }
+      const int nk16 = (nk + 15) & ~15;
+      for (int i = wt; i < nk16 * CPR; i += 256) {
         const int kk = i / CPR, ch = i % CPR;
-        const int key = kt + kk;
-        const int pg = pc->pg[(key >> a.page_shift) - pi0];
-        const size_t off = ((((size_t)pg * a.nkv + kvh) << a.page_shift) + (key & (a.page - 1))) * HD + ch * 8;
-        cp_async16(shK + kk * HD + ((ch ^ (kk & SWZ)) * 8), kpool + off);
-        cp_async16(shV + kk * HD + ch * 8, vpool + off);
+        if (kk < nk) {
+          const int key = kt + kk;
+          const int pg = pc->pg[(key >> a.page_shift) - pi0];
+          const size_t off = ((((size_t)pg * a.nkv + kvh) << a.page_shift) + (key & (a.page - 1))) * HD + ch * 8;
+          cp_async16(shK + kk * RS + ch * 8, kpool + off);
+          cp_async16(shV + kk * RS + ch * 8, vpool + off);
+        } else {                                                 // padding keys: P is 0 there, V must be finite
+          *reinterpret_cast<uint4 *>(shV + kk * RS + ch * 8) = make_uint4(0u, 0u, 0u, 0u);
+        }
       }
       prof_mark(a, wt, 5);
       cp_async_wait_all();
       worker_sync();
       prof_mark(a, wt, 6);
-      int qslot = 0;
-      for (int qi = warp; qi < nqv; qi += 8, ++qslot) {
-        const int qpos = pos0 + qi / group;
-        const uint4 *q4 = reinterpret_cast<const uint4 *>(shQ + qi * HD);
-        float sc[3];
-        float mx = -INFINITY;
-        {
-          // three 32-key sub-tiles at once, two accumulators each: six independent FMA chains
-          float acc[3][2];
-          const __nv_bfloat16 *krow[3];
-          int ksw[3];
+      // ---- S = scale * Q K^T, masked: (m-tile, 8-key n-tile) pairs over the warps
+      const int n_nt = (nk + 7) >> 3;
+#pragma unroll 1
+      for (int pair = warp; pair < n_mt * n_nt; pair += 8) {
+        const int mt = pair / n_nt, nt = pair % n_nt;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const __nv_bfloat16 *qa = shQ + (mt * 16 + g) * RS + 2 * t;
+        const __nv_bfloat16 *kb = shK + (nt * 8 + g) * RS + 2 * t;
 #pragma unroll
-          for (int j = 0; j < 3; ++j) {
-            const int kk = j * 32 + lane;
-            const int kr = kk < nk ? kk : nk - 1;                 // clamp: rows past the tile hold nothing
-            krow[j] = shK + kr * HD;
-            ksw[j] = kr & SWZ;
-            acc[j][0] = acc[j][1] = 0.f;
-          }
-#pragma unroll 2
-          for (int ch = 0; ch < CPR; ++ch) {
-            const uint4 qv = q4[ch];
-            const float q0 = bf_lo(qv.x), q1 = bf_hi(qv.x), q2 = bf_lo(qv.y), q3 = bf_hi(qv.y);
-            const float q4f = bf_lo(qv.z), q5 = bf_hi(qv.z), q6 = bf_lo(qv.w), q7 = bf_hi(qv.w);
-#pragma unroll
-            for (int j = 0; j < 3; ++j) {
-              if (j * 32 < nk) {
-                const uint4 kv = *reinterpret_cast<const uint4 *>(krow[j] + ((ch ^ ksw[j]) * 8));
-                acc[j][0] = fmaf(q0, bf_lo(kv.x), acc[j][0]); acc[j][1] = fmaf(q1, bf_hi(kv.x), acc[j][1]);
-                acc[j][0] = fmaf(q2, bf_lo(kv.y), acc[j][0]); acc[j][1] = fmaf(q3, bf_hi(kv.y), acc[j][1]);
-                acc[j][0] = fmaf(q4f, bf_lo(kv.z), acc[j][0]); acc[j][1] = fmaf(q5, bf_hi(kv.z), acc[j][1]);
-                acc[j][0] = fmaf(q6, bf_lo(kv.w), acc[j][0]); acc[j][1] = fmaf(q7, bf_hi(kv.w), acc[j][1]);
-              }
-            }
-          }
-#pragma unroll
-          for (int j = 0; j < 3; ++j) {
-            const int kk = j * 32 + lane;
-            float v = (acc[j][0] + acc[j][1]) * scale;
-            if (kk >= nk || kt + kk > qpos) v = -INFINITY;
-            sc[j] = v;
-            mx = fmaxf(mx, v);
-          }
+        for (int ks = 0; ks < KST; ++ks) {
+          unsigned af[4];
+          af[0] = *reinterpret_cast<const unsigned *>(qa + ks * 16);
+          af[1] = *reinterpret_cast<const unsigned *>(qa + 8 * RS + ks * 16);
+          af[2] = *reinterpret_cast<const unsigned *>(qa + ks * 16 + 8);
+          af[3] = *reinterpret_cast<const unsigned *>(qa + 8 * RS + ks * 16 + 8);
+          const unsigned b0 = *reinterpret_cast<const unsigned *>(kb + ks * 16);
+          const unsigned b1 = *reinterpret_cast<const unsigned *>(kb + ks * 16 + 8);
+          mma_bf16_16x8x16(acc, af, b0, b1);
         }
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
-        const float m_new = fmaxf(m_run[qslot], mx);
-        float corr = 1.f, ps = 0.f;
-        if (m_new > -INFINITY) corr = __expf(m_run[qslot] - m_new);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int row = mt * 16 + g + ((e & 2) ? 8 : 0), kk = nt * 8 + 2 * t + (e & 1);
+          const int qpos = pos0 + row / group;
+          float v = acc[e] * scale;
+          if (kk >= nk || kt + kk > qpos) v = -INFINITY;
+          shS[row * SS + kk] = v;
+        }
+      }
+      worker_sync();
+      // ---- online softmax per query row; P (bf16) overwrites the row of S it came from
+#pragma unroll 1
+      for (int row = warp; row < n_mt * 16; row += 8) {
+        float sv[3];
+        float mx = -INFINITY;
 #pragma unroll
         for (int j = 0; j < 3; ++j) {
-          const float p = (m_new > -INFINITY) ? __expf(sc[j] - m_new) : 0.f;
-          ps += p;
-          shP[warp * kAttnPStride + j * 32 + lane] = p;
+          const int kk = j * 32 + lane;
+          sv[j] = (kk < nk && row < nqv) ? shS[row * SS + kk] : -INFINITY;
+          mx = fmaxf(mx, sv[j]);
         }
-        for (int o = 16; o > 0; o >>= 1) ps += __shfl_xor_sync(0xFFFFFFFFu, ps, o);
-        l_run[qslot] = l_run[qslot] * corr + ps;
-        m_run[qslot] = m_new;
-        __syncwarp();
+        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
+        const float m_old = shM[row], m_new = fmaxf(m_old, mx);
+        const float corr = (m_new > -INFINITY) ? __expf(m_old - m_new) : 1.f;
+        float ps = 0.f;
+        __syncwarp();                                            // every lane has read its S values
+        __nv_bfloat16 *prow = reinterpret_cast<__nv_bfloat16 *>(shS + row * SS);
 #pragma unroll
-        for (int e = 0; e < DPL; ++e) o_run[qslot][e] *= corr;
-        {
-          float oe[2][DPL];
+        for (int j = 0; j < 3; ++j) {
+          const int kk = j * 32 + lane;
+          const float pv = (m_new > -INFINITY && sv[j] > -INFINITY) ? __expf(sv[j] - m_new) : 0.f;
+          const __nv_bfloat16 pb = __float2bfloat16_rn(pv);
+          ps += __bfloat162float(pb);                            // the sum uses the rounded P that multiplies V
+          if (kk < nk16) prow[kk] = pb;
+        }
+        for (int off = 16; off > 0; off >>= 1) ps += __shfl_xor_sync(0xFFFFFFFFu, ps, off);
+        if (lane == 0) { shM[row] = m_new; shL[row] = shL[row] * corr + ps; shC[row] = corr; }
+      }
+      worker_sync();
+      // ---- O = O * corr + P V: each warp owns NTW 8-wide slices of the head dimension
 #pragma unroll
-          for (int e = 0; e < DPL; ++e) oe[0][e] = oe[1][e] = 0.f;
-          const float *pw = shP + warp * kAttnPStride;
-          const int nk2 = (nk + 1) & ~1;                         // P is zero past nk (masked scores)
-#pragma unroll 4
-          for (int kk = 0; kk < nk2; kk += 2) {
+      for (int mt = 0; mt < 2; ++mt) {
+        if (mt < n_mt) {
+          const float c0 = shC[mt * 16 + g], c1 = shC[mt * 16 + g + 8];
+          const __nv_bfloat16 *pa = reinterpret_cast<const __nv_bfloat16 *>(shS + (mt * 16 + g) * SS) + 2 * t;
 #pragma unroll
-            for (int u = 0; u < 2; ++u) {
-              const float pk = pw[kk + u];
-              const __nv_bfloat16 *vr = shV + min(kk + u, nk - 1) * HD + lane * DPL;   // odd tail: P is 0, row must be valid
-              if (DPL == 4) {
-                const uint2 vv = *reinterpret_cast<const uint2 *>(vr);
-                oe[u][0] = fmaf(pk, bf_lo(vv.x), oe[u][0]);
-                oe[u][1] = fmaf(pk, bf_hi(vv.x), oe[u][1]);
-                oe[u][2] = fmaf(pk, bf_lo(vv.y), oe[u][2]);
-                oe[u][3] = fmaf(pk, bf_hi(vv.y), oe[u][3]);
-              } else {
-#pragma unroll
-                for (int e = 0; e < DPL; ++e) oe[u][e] = fmaf(pk, bf(vr[e]), oe[u][e]);
+          for (int n = 0; n < NTW; ++n) {
+            const int n0 = (warp * NTW + n) * 8;
+            if (n0 < HD) {
+              o[mt][n][0] *= c0; o[mt][n][1] *= c0; o[mt][n][2] *= c1; o[mt][n][3] *= c1;
+#pragma unroll 1
+              for (int ks = 0; ks < (nk16 >> 4); ++ks) {
+                unsigned af[4];
+                af[0] = *reinterpret_cast<const unsigned *>(pa + ks * 16);
+                af[1] = *reinterpret_cast<const unsigned *>(pa + 8 * SS * 2 + ks * 16);
+                af[2] = *reinterpret_cast<const unsigned *>(pa + ks * 16 + 8);
+                af[3] = *reinterpret_cast<const unsigned *>(pa + 8 * SS * 2 + ks * 16 + 8);
+                unsigned b0, b1;
+                ldmatrix_x2_trans(b0, b1, shV + (ks * 16 + (lane & 15)) * RS + n0);
+                mma_bf16_16x8x16(o[mt][n], af, b0, b1);
               }
             }
           }
-#pragma unroll
-          for (int e = 0; e < DPL; ++e) o_run[qslot][e] += oe[0][e] + oe[1][e];
         }
-        __syncwarp();
-        prof_mark(a, wt, 8 + (qslot > 0 ? 1 : 0));
       }
     }
     prof_mark(a, wt, 7);
-    int qslot = 0;
-    for (int qi = warp; qi < nqv; qi += 8, ++qslot) {
-      const int r = row0 + qi / group, h = kvh * group + qi % group;
-      float *dst = a.attn_partials + (((size_t)r * a.nq + h) * a.n_splits + split) * (HD + 2);
+    // ---- partial (o, m, l) of this split
 #pragma unroll
-      for (int e = 0; e < DPL; ++e) dst[lane * DPL + e] = o_run[qslot][e];
-      if (lane == 0) { dst[HD] = m_run[qslot]; dst[HD + 1] = l_run[qslot]; }
+    for (int mt = 0; mt < 2; ++mt) {
+      if (mt < n_mt) {
+#pragma unroll
+        for (int n = 0; n < NTW; ++n) {
+          const int n0 = (warp * NTW + n) * 8;
+          if (n0 < HD) {
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+              const int qi = mt * 16 + g + hh * 8;
+              if (qi < nqv) {
+                const int r = row0 + qi / group, h = kvh * group + qi % group;
+                float *dst = a.attn_partials + (((size_t)r * a.nq + h) * a.n_splits + split) * (HD + 2) + n0 + 2 * t;
+                dst[0] = o[mt][n][hh * 2];
+                dst[1] = o[mt][n][hh * 2 + 1];
+              }
+            }
+          }
+        }
+      }
+    }
+    if (wt < nqv) {
+      const int r = row0 + wt / group, h = kvh * group + wt % group;
+      float *dst = a.attn_partials + (((size_t)r * a.nq + h) * a.n_splits + split) * (HD + 2);
+      dst[HD] = shM[wt];
+      dst[HD + 1] = shL[wt];
     }
   }
 }
