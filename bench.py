@@ -87,6 +87,20 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def reduce_max_over_ranks(values, device="cuda"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch.distributed as dist
+    t = torch.tensor(values, device=device, dtype=torch.float64)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_tokens_per_s(world, n_new, ms_per_step):
+    """Whole-job throughput of `world` independent replicas generating n_new tokens per step each."""
+    return world * n_new / (ms_per_step / 1e3)
+
+
 def weight_bytes(cfg, n_layers):
     es = 2 if cfg["dtype"] == "bf16" else 4
     d, hd, ff, V = cfg["d_model"], cfg["head_dim"], cfg["d_ff"], cfg["vocab"]
@@ -183,10 +197,8 @@ def run_ours(args):
         out_host.copy_(toks, non_blocking=True)
         torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    t = torch.tensor([dec_ms / args.steps, step_ms, e2e_s * 1e3, pre_ms / args.steps], device="cuda", dtype=torch.float64)
-    if world > 1:
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-    dec_ms_step, step_ms, e2e_ms, pre_ms_step = t.tolist()
+    dec_ms_step, step_ms, e2e_ms, pre_ms_step = reduce_max_over_ranks(
+        [dec_ms / args.steps, step_ms, e2e_s * 1e3, pre_ms / args.steps])
     if rank != 0:
         return
     hbm_peak, peak_kind = peaks()
@@ -213,14 +225,14 @@ def run_ours(args):
     if os.path.exists(ratio_file):
         traffic = int(json.load(open(ratio_file))["dram_bytes_per_algorithmic_byte"] * tgt_bytes)
     line = {
-        "metric": METRIC, "value": round(world * n_new / (dec_ms_step / 1e3), 2), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": round(aggregate_tokens_per_s(world, n_new, dec_ms_step), 2), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dec_ms_step, 3), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
         "config": {"workload": args.workload, "batch": 1, "prompt_len": P, "n_new": n_new, "exits": list(wl["exits"]),
                    "T": T, "T_search": calib, "l2": "inputs larger than L2 (weights %.1f GB per target pass)"
                    % (weight_bytes(cfg, cfg["n_layers"]) / 1e9), "replicas": "independent sequence per GPU"},
         "prefill_ms": round(pre_ms_step, 3), "step_ms_with_prefill": round(step_ms, 3),
-        "e2e": {"value": round(world * n_new / (e2e_ms / 1e3), 2), "unit": UNIT, "h2d_bytes_per_step": P * 4,
+        "e2e": {"value": round(aggregate_tokens_per_s(world, n_new, e2e_ms), 2), "unit": UNIT, "h2d_bytes_per_step": P * 4,
                 "d2h_bytes_per_step": n_new * 4},
         "gpu_launches": int(launches),
         "clocks": clk.summary(),

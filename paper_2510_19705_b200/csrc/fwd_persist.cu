@@ -356,12 +356,14 @@ __device__ __forceinline__ void ldmatrix_x2_trans(unsigned &r0, unsigned &r1, co
 
 // Phase A on the (legacy) tensor path: S = Q K^T and O += P V with mma.sync m16n8k16, fp32 softmax in
 // between.  Shared memory: K, V, Q as bf16 rows padded by 16 bytes (conflict-free fragment loads),
-// S as fp32 [32][84] with P (bf16) written in place over each S row, running (m, l, corr) per query.
+// S as fp32 [32][84] with P (bf16 hi and lo halves) written in place over each S row, running (m, l,
+// corr) per query.
 template <int HD>
 __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt) {
   constexpr int CPR = HD / 8;                      // 16-byte chunks per row
   constexpr int RS = HD + 8;                       // padded row stride (bf16 elements)
   constexpr int SS = 84;                           // S row stride (floats)
+  constexpr int kPLoOff = 84;                      // bf16 offset of the low half of P inside its S row
   constexpr int KST = HD / 16;                     // k-steps of Q K^T
   constexpr int NTW = (HD / 8 + 7) / 8;            // output n-tiles (8 dims) per warp
   const int group = a.nq / a.nkv;
@@ -476,9 +478,12 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
         for (int j = 0; j < 3; ++j) {
           const int kk = j * 32 + lane;
           const float pv = (m_new > -INFINITY && sv[j] > -INFINITY) ? __expf(sv[j] - m_new) : 0.f;
-          const __nv_bfloat16 pb = __float2bfloat16_rn(pv);
-          ps += __bfloat162float(pb);                            // the sum uses the rounded P that multiplies V
-          if (kk < nk16) prow[kk] = pb;
+          // P = hi + lo in bf16 (two MMAs against V): the product keeps ~16 bits of P, so the attention
+          // output is as accurate as an fp32 P would give
+          const __nv_bfloat16 ph = __float2bfloat16_rn(pv);
+          const __nv_bfloat16 pl = __float2bfloat16_rn(pv - __bfloat162float(ph));
+          ps += pv;
+          if (kk < nk16) { prow[kk] = ph; prow[kPLoOff + kk] = pl; }
         }
         for (int off = 16; off > 0; off >>= 1) ps += __shfl_xor_sync(0xFFFFFFFFu, ps, off);
         if (lane == 0) { shM[row] = m_new; shL[row] = shL[row] * corr + ps; shC[row] = corr; }
@@ -504,6 +509,11 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
                 af[3] = *reinterpret_cast<const unsigned *>(pa + 8 * SS * 2 + ks * 16 + 8);
                 unsigned b0, b1;
                 ldmatrix_x2_trans(b0, b1, shV + (ks * 16 + (lane & 15)) * RS + n0);
+                mma_bf16_16x8x16(o[mt][n], af, b0, b1);
+                af[0] = *reinterpret_cast<const unsigned *>(pa + kPLoOff + ks * 16);
+                af[1] = *reinterpret_cast<const unsigned *>(pa + kPLoOff + 8 * SS * 2 + ks * 16);
+                af[2] = *reinterpret_cast<const unsigned *>(pa + kPLoOff + ks * 16 + 8);
+                af[3] = *reinterpret_cast<const unsigned *>(pa + kPLoOff + 8 * SS * 2 + ks * 16 + 8);
                 mma_bf16_16x8x16(o[mt][n], af, b0, b1);
               }
             }

@@ -106,3 +106,27 @@ def test_rows_are_prefix_consistent():
     for j in range(4):
         one = m.rows_from_scratch(2, toks[:5 + j], [])[0]
         assert np.abs(rows[j] - one).max() < 1e-6
+
+
+def test_bf16_forward_is_sensitive_to_fp32_level_noise():
+    """Why the bf16 logits tolerance is statistical: nudging every value by 2e-6 (the size of fp32 accumulation
+    error) before each bf16 rounding point moves the oracle's own logits by far more than 2e-6, because a
+    value near a rounding boundary flips by a whole bf16 step and the flips compound through the layers."""
+    from oracle import transformer as T
+    cfg = inputs.model_cfg(3, 256, 8, 2, 704, 512, "bf16", head_dim=32)
+    w = inputs.weights_to_numpy(inputs.make_weights(cfg, 3, std=0.05))
+    prompt = inputs.make_prompts(cfg["vocab"], 1, 24, 3)[0].tolist()
+    a = T.Transformer(cfg, w, (2, 3))
+    a.rows(0, prompt, [])
+    ref = a.last_logits64[0].copy()
+    orig = T.bf16_round
+    rng = np.random.default_rng(0)
+    T.bf16_round = lambda x: orig(np.asarray(x, dtype=np.float64) * (1.0 + 2e-6 * rng.standard_normal(np.shape(x))))
+    try:
+        b = T.Transformer(cfg, w, (2, 3))
+        b.rows(0, prompt, [])
+        got = b.last_logits64[0]
+    finally:
+        T.bf16_round = orig
+    rel = float(np.sqrt(((got - ref) ** 2).mean()) / ref.std())
+    assert 2e-4 < rel < 5e-2, rel          # orders of magnitude above the 2e-6 that went in, still small
