@@ -121,7 +121,7 @@ def to_cuda(w):
     return {k: (v.cuda() if k != "layers" else [{n: t.cuda() for n, t in l.items()} for l in v]) for k, v in w.items()}
 
 
-def choose_T(binding, cfg, weights, wl, prompts, n_calib=64):
+def choose_T(binding, cfg, weights, wl, prompts, n_calib=160):
     """Calibration run with T = (2, ..., 2), then the Theorem 3.2 search (monotone T, T_max 15)."""
     exits = wl["exits"]
     K = len(exits) - 1
@@ -248,6 +248,81 @@ def run_ours(args):
     print(json.dumps(line))
 
 
+def run_accept(args):
+    """Stand-alone acceptance / resample workload (batch 64, 8 drafted positions, vocabulary 32000, bf16):
+    one step = one hsd_verify_level call; four input sets are rotated so every call reads from HBM."""
+    from paper_2510_19705_b200 import binding, inputs
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    wl = inputs.WORKLOADS["accept"]
+    B, t, V = wl["batch"], wl["t"], wl["vocab"]
+    sets = []
+    for i in range(4):
+        p, q = inputs.make_accept_logits(B, t, V, seed=i, device="cuda")
+        x = binding.hsd_draft_sample(q, 100 + i, 0)
+        sets.append((p, q, x))
+    ws = torch.empty(max(16, binding.hsd_verify_workspace_bytes(B, t)), dtype=torch.uint8, device="cuda")
+    out = torch.empty(B, t + 1, dtype=torch.int32, device="cuda")
+    n = torch.empty(B, dtype=torch.int32, device="cuda")
+    steps, warm = max(args.steps, 20), max(args.warmup, 3)
+    for i in range(warm):
+        binding.hsd_verify_level(1, *sets[i % 4], 7, i, ws, out, n)
+    torch.cuda.synchronize()
+    l0 = binding.hsd_kernel_launches()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    with ClockSampler(torch.cuda.current_device()) as clk:
+        ev[0].record()
+        for i in range(steps):
+            binding.hsd_verify_level(1, *sets[i % 4], 7, i, ws, out, n)
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+    ms = ev[0].elapsed_time(ev[steps]) / steps
+    launches = binding.hsd_kernel_launches() - l0
+    # end to end from pinned host memory: logits upload, decision, result download
+    hp, hq, hx = (a.cpu().pin_memory() for a in sets[0])
+    ho = torch.empty(B, t + 1, dtype=torch.int32).pin_memory()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(3):
+        dp, dq, dx = hp.cuda(non_blocking=True), hq.cuda(non_blocking=True), hx.cuda(non_blocking=True)
+        binding.hsd_verify_level(1, dp, dq, dx, 7, i, ws, out, n)
+        ho.copy_(out, non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - t0) / 3 * 1e3
+    bytes_alg = (B * (t + 1) + B * t) * V * 2
+    hbm_peak, peak_kind = peaks()
+    achieved = bytes_alg / ms / 1e6
+    line = {"metric": "accept_positions_per_s", "value": round(B * t / (ms / 1e3), 1), "unit": "positions/s", "n_gpus": 1,
+            "steps": steps, "warmup": warm, "ms_per_step": round(ms, 5), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "accept", "batch": B, "t": t, "vocab": V,
+                       "l2": "4 input sets of 69.6 MB rotated (278 MB > L2)"},
+            "e2e": {"value": round(B * t / (e2e_ms / 1e3), 1), "unit": "positions/s", "h2d_bytes_per_step": bytes_alg + B * t * 4,
+                    "d2h_bytes_per_step": B * (t + 1) * 4},
+            "gpu_launches": int(launches), "clocks": clk.summary(),
+            "roofline": {"bound": "hbm", "kernel": "row_stats_vec_kernel + decide_kernel (one verification call)",
+                         "achieved": round(achieved, 1), "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
+                         "frac": round(achieved / hbm_peak, 4), "traffic": None, "bytes_per_launch": bytes_alg}}
+    if not args.no_cpu_baseline:
+        from oracle.hsd import SpecDecisions
+        from oracle.verify import verify
+
+        class Rows:
+            def __init__(self, rows):
+                self.r = rows
+
+            def rows(self, idx, ctx, draft):
+                return list(self.r)
+        p_np, q_np, x_np = inputs.logits_to_numpy(sets[0][0]), inputs.logits_to_numpy(sets[0][1]), sets[0][2].cpu().numpy()
+        t0 = time.perf_counter()
+        nb = 16
+        for b in range(nb):
+            verify(1, list(x_np[b]), list(q_np[b]), [0], Rows(p_np[b]), SpecDecisions(7, b), 0)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": round(nb * t / dt, 1), "unit": "positions/s", "cores": 1, "kind": "oracle",
+                                "sample": "%d of the %d sequences (%.1f s)" % (nb, B, dt)}
+    print(json.dumps(line))
+
+
 def cpu_baseline(workload, T, weights=None, rounds=1, prompt_len=8):
     """The oracle, as it stands, on a bounded sample: `rounds` top-level HSD rounds of the same model
     after a short prompt."""
@@ -319,7 +394,10 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-        run_ours(args)
+        if args.workload == "accept":
+            run_accept(args)
+        else:
+            run_ours(args)
 
 
 if __name__ == "__main__":

@@ -25,9 +25,17 @@ draft_sample_kernel(const T *__restrict__ logits, int V, const SampleRow *__rest
     d.level = 0;
   }
   const T *row = logits + (size_t)d.logit_row * V;
-  float m = row_max(row, V, shf);
   u32 U = uniform24(seed, d.j, d.serial, d.level, PURPOSE_DRAFT, d.seq);
-  int tok = block_inverse_cdf(V, U, [&](int k) { return (u64)exp_weight(to_f32(row[k]), m); }, sh64, nullptr);
+  int tok;
+  if (sizeof(T) == 2 && chunk_layout_ok(row, V, blockDim.x)) {
+    const int k0 = threadIdx.x * kChunkTokens;
+    const Chunk32 c = chunk_load(reinterpret_cast<const __nv_bfloat16 *>(row), V, k0);
+    const float m = block_max(chunk_max(c, V, k0), shf);
+    tok = block_inverse_cdf_chunk(V, k0, U, [&](int i) { return (u64)exp_weight(chunk_get(c, i), m); }, sh64, nullptr);
+  } else {
+    float m = row_max(row, V, shf);
+    tok = block_inverse_cdf(V, U, [&](int k) { return (u64)exp_weight(to_f32(row[k]), m); }, sh64, nullptr);
+  }
   if (threadIdx.x == 0) out[d.out_index] = tok;
 }
 
@@ -59,6 +67,93 @@ row_stats_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits,
   float m = row_max(row, V, shf);
   u64 local = 0;
   for (int k = threadIdx.x; k < V; k += blockDim.x) local += exp_weight(to_f32(row[k]), m);
+  u64 total;
+  block_exclusive_scan(local, sh64, &total);
+  if (threadIdx.x == 0) {
+    RowStat s;
+    s.m = m;
+    s.S = total;
+    s.Ex = (tok >= 0 && tok < V) ? exp_weight(to_f32(row[tok]), m) : 0u;
+    stats[(size_t)b * (2 * t_max + 1) + r] = s;
+  }
+}
+
+// Same statistics with the whole row held in registers: 16-byte loads, one pass over HBM, packed
+// arithmetic.  Needs V a multiple of the vector width, V <= 8 vectors per thread and 16-byte rows.
+template <typename T> struct StatVec;
+template <> struct StatVec<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ static void unpack(const uint4 &v, float *f) {
+    f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+    f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+    f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xFFFF0000u);
+    f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xFFFF0000u);
+  }
+};
+template <> struct StatVec<float> {
+  static constexpr int N = 4;
+  __device__ static void unpack(const uint4 &v, float *f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y); f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
+};
+constexpr int kStatVecPerThread = 8;
+
+template <typename T>
+__global__ void __launch_bounds__(kStatThreads)
+row_stats_vec_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, const int32_t *__restrict__ tokens,
+                     int V, int t_max, const VerifySeq *__restrict__ desc, int regular_t, RowStat *__restrict__ stats) {
+  constexpr int VN = StatVec<T>::N;
+  __shared__ float shf[32];
+  __shared__ u64 sh64[33];
+  int b = blockIdx.y, r = blockIdx.x;
+  VerifySeq d;
+  if (desc) d = desc[b];
+  else { d.t = regular_t; d.p_row0 = (long long)b * (regular_t + 1); d.q_row0 = (long long)b * regular_t; d.tok_off = (long long)b * regular_t; }
+  const T *row;
+  int tok = -1;
+  if (r <= t_max) {
+    if (r > d.t) return;
+    row = p_logits + (size_t)(d.p_row0 + r) * V;
+    if (r < d.t) tok = tokens[d.tok_off + r];
+  } else {
+    int j = r - t_max - 1;
+    if (j >= d.t) return;
+    row = q_logits + (size_t)(d.q_row0 + j) * V;
+    tok = tokens[d.tok_off + j];
+  }
+  const int nvec = V / VN;
+  const uint4 *row4 = reinterpret_cast<const uint4 *>(row);
+  uint4 regs[kStatVecPerThread];
+#pragma unroll
+  for (int j = 0; j < kStatVecPerThread; ++j) {
+    const int iv = threadIdx.x + kStatThreads * j;
+    regs[j] = iv < nvec ? __ldg(row4 + iv) : make_uint4(0u, 0u, 0u, 0u);
+  }
+  float m = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < kStatVecPerThread; ++j) {
+    if ((int)threadIdx.x + kStatThreads * j < nvec) {
+      float f[VN];
+      StatVec<T>::unpack(regs[j], f);
+#pragma unroll
+      for (int e = 0; e < VN; ++e) m = fmaxf(m, f[e]);
+    }
+  }
+  m = block_max(m, shf);
+  u64 local = 0;
+#pragma unroll
+  for (int j = 0; j < kStatVecPerThread; ++j) {
+    if ((int)threadIdx.x + kStatThreads * j < nvec) {
+      float f[VN];
+      StatVec<T>::unpack(regs[j], f);
+#pragma unroll
+      for (int e = 0; e < VN; e += 2) {
+        u32 e0, e1;
+        exp_weight2(f[e], f[e + 1], m, e0, e1);
+        local += (u64)e0 + (u64)e1;
+      }
+    }
+  }
   u64 total;
   block_exclusive_scan(local, sh64, &total);
   if (threadIdx.x == 0) {
@@ -107,7 +202,24 @@ decide_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, in
   const T *prow = p_logits + (size_t)(d.p_row0 + n) * V;
   float mp = st[n].m;
   int m_tok = -1;
-  if (n < d.t) {
+  const bool fast = sizeof(T) == 2 && chunk_layout_ok(prow, V, blockDim.x) &&
+                    (n >= d.t || chunk_layout_ok(q_logits + (size_t)(d.q_row0 + n) * V, V, blockDim.x));
+  if (fast) {
+    const int k0 = threadIdx.x * kChunkTokens;
+    const Chunk32 cp = chunk_load(reinterpret_cast<const __nv_bfloat16 *>(prow), V, k0);
+    if (n < d.t) {
+      const Chunk32 cq = chunk_load(reinterpret_cast<const __nv_bfloat16 *>(q_logits + (size_t)(d.q_row0 + n) * V), V, k0);
+      const float mq = st[t_max + 1 + n].m;
+      const ProbScale psp = prob_scale(st[n].S), psq = prob_scale(st[t_max + 1 + n].S);
+      m_tok = block_inverse_cdf_chunk(V, k0, U, [&](int i) {
+        u64 Pp = fixed_prob(exp_weight(chunk_get(cp, i), mp), psp);
+        u64 Pq = fixed_prob(exp_weight(chunk_get(cq, i), mq), psq);
+        return Pp > Pq ? Pp - Pq : 0ull;
+      }, sh64, nullptr);
+    }
+    if (m_tok < 0)
+      m_tok = block_inverse_cdf_chunk(V, k0, U, [&](int i) { return (u64)exp_weight(chunk_get(cp, i), mp); }, sh64, nullptr);
+  } else if (n < d.t) {
     const T *qrow = q_logits + (size_t)(d.q_row0 + n) * V;
     float mq = st[t_max + 1 + n].m;
     ProbScale psp = prob_scale(st[n].S), psq = prob_scale(st[t_max + 1 + n].S);
@@ -117,7 +229,7 @@ decide_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, in
       return Pp > Pq ? Pp - Pq : 0ull;
     }, sh64, nullptr);
   }
-  if (m_tok < 0)   // bonus token, or an all-zero residual: draw from the verifier's own row
+  if (!fast && m_tok < 0)   // bonus token, or an all-zero residual: draw from the verifier's own row
     m_tok = block_inverse_cdf(V, U, [&](int k) { return (u64)exp_weight(to_f32(prow[k]), mp); }, sh64, nullptr);
   if (threadIdx.x == 0) {
     out_n[b] = n;
@@ -158,7 +270,13 @@ static int launch_verify_t(const void *p, const void *q, int32_t *tokens, int V,
                            u64 seed, int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s) {
   RowStat *stats = (RowStat *)scratch;
   dim3 grid(2 * t_max + 1, batch);
-  row_stats_kernel<T><<<grid, kStatThreads, 0, s>>>((const T *)p, (const T *)q, tokens, V, t_max, desc, regular_t, stats);
+  constexpr int VN = StatVec<T>::N;
+  const bool vec_ok = V % VN == 0 && V / VN <= kStatVecPerThread * kStatThreads && ((uintptr_t)p & 15) == 0 &&
+                      (q == nullptr || ((uintptr_t)q & 15) == 0);
+  if (vec_ok)
+    row_stats_vec_kernel<T><<<grid, kStatThreads, 0, s>>>((const T *)p, (const T *)q, tokens, V, t_max, desc, regular_t, stats);
+  else
+    row_stats_kernel<T><<<grid, kStatThreads, 0, s>>>((const T *)p, (const T *)q, tokens, V, t_max, desc, regular_t, stats);
   if (cudaGetLastError() != cudaSuccess) return HSD_E_CUDA;
   decide_kernel<T><<<batch, kSampleThreads, 0, s>>>((const T *)p, (const T *)q, tokens, V, t_max, desc, regular_t,
                                                    regular_serial, regular_level, stats, seed, out_tokens, out_n,
