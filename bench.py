@@ -114,7 +114,7 @@ def pass_bytes(cfg, n_layers, ctx, rows, logit_rows):
     es = 2 if cfg["dtype"] == "bf16" else 4
     kv = 2 * cfg["n_kv_heads"] * cfg["head_dim"] * es
     return (weight_bytes(cfg, n_layers) + n_layers * kv * (ctx + rows) + rows * cfg["d_model"] * es
-            + logit_rows * cfg["vocab"] * es)
+            + logit_rows * cfg["vocab"] * es)      # ctx = context tokens summed over the sequences of the pass
 
 
 def to_cuda(w):
@@ -126,7 +126,8 @@ def choose_T(binding, cfg, weights, wl, prompts, n_calib=160):
     exits = wl["exits"]
     K = len(exits) - 1
     T0 = [2] * K
-    eng = binding.Hsd(cfg, weights, exits, T0, max_batch=1, max_seq=wl["prompt"] + n_calib + 64, page_size=wl["page"])
+    eng = binding.Hsd(cfg, weights, exits, T0, max_batch=prompts.shape[0], max_seq=wl["prompt"] + n_calib + 64,
+                      page_size=wl["page"])
     eng.generate(prompts, 8, 12345)                      # warm-up
     _, stats, _ = eng.generate(prompts, n_calib, 12345)
     eng.close()
@@ -147,10 +148,11 @@ def run_ours(args):
         dist.init_process_group("nccl")
     wl = inputs.WORKLOADS[args.workload]
     cfg = wl["model"]
-    n_new, P = (args.n_new or wl["n_new"]), wl["prompt"]
+    n_new, P = (args.n_new or wl["n_new"]), (args.prompt_len or wl["prompt"])
     # replicas only: each rank runs its own independent sequence (no data-path collective)
     weights = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
-    prompts_host = inputs.make_prompts(cfg["vocab"], 1, P, wl["prompt_seed"] + rank).pin_memory()
+    B = max(1, args.batch)
+    prompts_host = inputs.make_prompts(cfg["vocab"], B, P, wl["prompt_seed"] + rank).pin_memory()
     prompts = prompts_host.cuda()
     if args.T:
         T, calib = [int(v) for v in args.T.split(",")], None
@@ -160,7 +162,7 @@ def run_ours(args):
                  "expected_ms_per_token": round(lat, 4)}
     else:
         T, calib = list(wl["T"]), None
-    eng = binding.Hsd(cfg, weights, wl["exits"], T, max_batch=1, max_seq=P + n_new + sum(T) + 16, page_size=wl["page"])
+    eng = binding.Hsd(cfg, weights, wl["exits"], T, max_batch=B, max_seq=P + n_new + sum(T) + 16, page_size=wl["page"])
 
     def barrier():
         torch.cuda.synchronize()
@@ -187,7 +189,7 @@ def run_ours(args):
     launches = binding.hsd_kernel_launches() - launches0
     step_ms = ev0.elapsed_time(ev1) / args.steps
     # end to end through the public call, host buffers: prompt upload + prompt pass + generation + download
-    out_host = torch.empty(1, n_new, dtype=torch.int32).pin_memory()
+    out_host = torch.empty(B, n_new, dtype=torch.int32).pin_memory()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     e2e_steps = max(1, min(args.steps, 3))
@@ -207,7 +209,7 @@ def run_ours(args):
     tgt = agg[K]
     tgt_ms = tgt["ms"] / max(1, tgt["forwards"])
     mean_rows = tgt["rows"] / max(1, tgt["forwards"])
-    mean_ctx = P + n_new / 2.0
+    mean_ctx = B * (P + n_new / 2.0)
     levels = []
     for i, s in enumerate(agg):
         ms = s["ms"] / max(1, s["forwards"])
@@ -225,15 +227,15 @@ def run_ours(args):
     if os.path.exists(ratio_file):
         traffic = int(json.load(open(ratio_file))["dram_bytes_per_algorithmic_byte"] * tgt_bytes)
     line = {
-        "metric": METRIC, "value": round(aggregate_tokens_per_s(world, n_new, dec_ms_step), 2), "unit": UNIT, "n_gpus": world,
+        "metric": METRIC, "value": round(aggregate_tokens_per_s(world, B * n_new, dec_ms_step), 2), "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dec_ms_step, 3), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
-        "config": {"workload": args.workload, "batch": 1, "prompt_len": P, "n_new": n_new, "exits": list(wl["exits"]),
+        "config": {"workload": args.workload, "batch": B, "prompt_len": P, "n_new": n_new, "exits": list(wl["exits"]),
                    "T": T, "T_search": calib, "l2": "inputs larger than L2 (weights %.1f GB per target pass)"
                    % (weight_bytes(cfg, cfg["n_layers"]) / 1e9), "replicas": "independent sequence per GPU"},
         "prefill_ms": round(pre_ms_step, 3), "step_ms_with_prefill": round(step_ms, 3),
-        "e2e": {"value": round(aggregate_tokens_per_s(world, n_new, e2e_ms), 2), "unit": UNIT, "h2d_bytes_per_step": P * 4,
-                "d2h_bytes_per_step": n_new * 4},
+        "e2e": {"value": round(aggregate_tokens_per_s(world, B * n_new, e2e_ms), 2), "unit": UNIT, "h2d_bytes_per_step": B * P * 4,
+                "d2h_bytes_per_step": B * n_new * 4},
         "gpu_launches": int(launches),
         "clocks": clk.summary(),
         "roofline": {"bound": "hbm", "kernel": "fwd_persistent_kernel: one launch = the target level's whole "
@@ -387,6 +389,8 @@ def main():
     ap.add_argument("--workload", default="8b3")
     ap.add_argument("--n-new", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=1, help="sequences per GPU (the metric is quoted at 1)")
+    ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length (development runs)")
     ap.add_argument("--T", default="", help="fix T (comma separated) instead of calibrating / using the workload's")
     args = ap.parse_args()
     if args.impl == "reference":
