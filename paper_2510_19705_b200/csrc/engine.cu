@@ -746,7 +746,7 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
       int coop = 0, dev = 0;
       cudaGetDevice(&dev);
       cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-      c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 && md.n_layers <= 64 && (md.page & (md.page - 1)) == 0 &&
+      c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 && (md.d / kTcBlockM) * 2 <= c->sm_count && md.n_layers <= 64 && (md.page & (md.page - 1)) == 0 &&
                        getenv("HSD_NO_PERSIST") == nullptr;
     }
     if (!st && cudaMallocHost(&c->status_host, 4) != cudaSuccess) st = HSD_E_CUDA;

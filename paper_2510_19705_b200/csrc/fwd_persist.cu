@@ -260,39 +260,26 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
       graw[j] = iv < nvec ? __ldg(reinterpret_cast<const uint2 *>(gain) + iv) : make_uint2(0u, 0u);
     }
     if (pend) {
-      // every piece of every slot in one batch of loads (a tile of these projections has <= 4 pieces)
-      int np[MAXV];
-      const float *base[MAXV];
-      int np_max = 0;
+      // every piece of every slot in one batch of loads: the residual projections have at most d / 128
+      // = 32 tiles, so they are always cut the regular way (the launcher checks it), `parts` <= 4
+      // pieces per tile at a fixed stride
+      const int np = geo.parts;
+      float4 t[MAXV][PB];
 #pragma unroll
       for (int j = 0; j < MAXV; ++j) {
-        const int iv = wt + 256 * j;
-        np[j] = 0;
-        base[j] = a.pieces;
-        if (iv < nvec) {
-          const int k = iv << 2, tile = k >> 7, mm = k & 127;
-          int fo;
-          tile_pieces(*pend, geo, tile, fo, np[j]);
-          base[j] = a.pieces + ((size_t)tile * geo.pieces_max * NPAD + row) * kTcBlockM + mm;
+        const int iv = wt + 256 * j, k = iv << 2, tile = k >> 7, mm = k & 127;
+        const float *base = a.pieces + ((size_t)tile * np * NPAD + row) * kTcBlockM + mm;
+#pragma unroll
+        for (int pp = 0; pp < PB; ++pp)
+          t[j][pp] = (iv < nvec && pp < np) ? __ldcg(reinterpret_cast<const float4 *>(base + (size_t)pp * NPAD * kTcBlockM))
+                                            : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int j = 0; j < MAXV; ++j)
+#pragma unroll
+        for (int pp = 0; pp < PB; ++pp) {
+          v[j].x += t[j][pp].x; v[j].y += t[j][pp].y; v[j].z += t[j][pp].z; v[j].w += t[j][pp].w;
         }
-        np_max = max(np_max, np[j]);
-      }
-      for (int p0 = 0; p0 < np_max; p0 += PB) {
-        float4 t[MAXV][PB];
-#pragma unroll
-        for (int j = 0; j < MAXV; ++j)
-#pragma unroll
-          for (int pp = 0; pp < PB; ++pp)
-            t[j][pp] = (p0 + pp < np[j])
-                           ? __ldcg(reinterpret_cast<const float4 *>(base[j] + (size_t)(p0 + pp) * NPAD * kTcBlockM))
-                           : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int j = 0; j < MAXV; ++j)
-#pragma unroll
-          for (int pp = 0; pp < PB; ++pp) {
-            v[j].x += t[j][pp].x; v[j].y += t[j][pp].y; v[j].z += t[j][pp].z; v[j].w += t[j][pp].w;
-          }
-      }
     }
     float ss = 0.f;
 #pragma unroll
@@ -816,10 +803,22 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // The three pipeline roles below are single threads: a lone thread runs ~5 cycles per dependent
+  // instruction, and with whole-tile GEMMs one SM has to sustain up to twice its fair share of the
+  // weight stream (~90 GB/s = one 16 KiB stage per 180 ns).  So they keep wrapped slot counters and
+  // parities in registers instead of dividing a stage count, ring slots are handed back in pairs (a
+  // tcgen05.commit costs the tensor pipe as much as three MMAs of this shape), and
+  // tcgen05.fence::after_thread_sync (~0.1 us while MMAs are in flight) is issued only where another
+  // thread's tcgen05 operations must come first (accumulator reuse), not after the wait on TMA data.
+#ifndef HSD_WGS
+#define HSD_WGS 1
+#endif
+  constexpr int WGS = (STAGES % HSD_WGS == 0) ? HSD_WGS : 1;       // landing slots handed back together
   if (warp == 0) {
     // ------------------------------------------------------------ weight-tile producer (runs ahead)
     if (lane == 0) {
-      long long issued = 0;
+      int s = 0, n_issued = 0;
+      uint32_t par = 1;                                  // parity to wait for on the slot group's empty barrier
       bool ok = true;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
@@ -828,28 +827,29 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         while (ok && seg_next(g, it, sg)) {
           const Tile ti = tile_of(g, sg.tile);
           const bool second = (g.mode == MODE_SWIGLU) || (ti.row0 + kTcBoxRows < g.seg_n[ti.seg]);
-          for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++issued) {
-            const int s = (int)(issued % STAGES);
-            const uint32_t ph = (uint32_t)((issued / STAGES) & 1);
-            if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t dst = smem_u32(ring + (size_t)s * Cfg::kStageBytes);
-            mbar_expect_tx(full_bar(s), (second ? 2 : 1) * kBoxBytes);
-            if (g.mode == MODE_SWIGLU) {
-              tma_load_2d(dst, g.w[0], kb * kTcBlockK, ti.row0, full_bar(s));
-              tma_load_2d(dst + kBoxBytes, g.w[1], kb * kTcBlockK, ti.row0, full_bar(s));
-            } else {
-              tma_load_2d(dst, g.w[ti.seg], kb * kTcBlockK, ti.row0, full_bar(s));
-              if (second) tma_load_2d(dst + kBoxBytes, g.w[ti.seg], kb * kTcBlockK, ti.row0 + kTcBoxRows, full_bar(s));
-            }
+          const CUtensorMap *m0 = g.mode == MODE_SWIGLU ? g.w[0] : g.w[ti.seg];
+          const CUtensorMap *m1 = g.mode == MODE_SWIGLU ? g.w[1] : m0;
+          const int row1 = g.mode == MODE_SWIGLU ? ti.row0 : ti.row0 + kTcBoxRows;
+          const uint32_t tx = (second ? 2 : 1) * kBoxBytes;
+          for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+            if (s % WGS == 0 && !mbar_wait(empty_bar(s / WGS), par, abort_flag)) { ok = false; break; }
+            const uint32_t dst = smem_u32(ring) + (uint32_t)(s * Cfg::kStageBytes);
+            mbar_expect_tx(full_bar(s), tx);
+            tma_load_2d(dst, m0, kb * kTcBlockK, ti.row0, full_bar(s));
+            if (second) tma_load_2d(dst + kBoxBytes, m1, kb * kTcBlockK, row1, full_bar(s));
+            ++n_issued;
+            if (++s == STAGES) { s = 0; par ^= 1u; }
           }
         }
       }
       if (!ok) {
         atomicExch(a.status, 1);
-        long long first = issued > STAGES ? issued - STAGES : 0;     // let copies in flight land (bounded)
-        for (long long i = first; i < issued; ++i) {
+        // let copies in flight land (bounded): the last min(n_issued, STAGES) slots, newest first
+        uint32_t fpar = par ^ 1u;                        // full-barrier parity of the current round
+        for (int i = 0, sl = s; i < STAGES && i < n_issued; ++i) {
+          if (--sl < 0) { sl = STAGES - 1; fpar ^= 1u; }
           unsigned long long t0 = globaltimer_ns();
-          while (!mbar_try_wait(full_bar((int)(i % STAGES)), (uint32_t)((i / STAGES) & 1)))
+          while (!mbar_try_wait(full_bar(sl), fpar))
             if (globaltimer_ns() - t0 > kWaitLimitNs / 4) break;
         }
       }
@@ -857,7 +857,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   } else if (warp == 1) {
     // ------------------------------------------------------------ activation-tile producer
     if (lane == 0) {
-      long long issued = 0;
+      int s = 0;
+      uint32_t par = 1;
       bool ok = true;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
@@ -866,13 +867,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         SegIter it = seg_begin(g, G, c);
         Seg sg;
         while (ok && seg_next(g, it, sg)) {
-          for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++issued) {
-            const int s = (int)(issued % STAGES);
-            const uint32_t ph = (uint32_t)((issued / STAGES) & 1);
-            if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t dst = smem_u32(ring + (size_t)s * Cfg::kStageBytes) + kWBytes;
+          for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+            if (s % WGS == 0 && !mbar_wait(empty_bar(s / WGS), par, abort_flag)) { ok = false; break; }
+            const uint32_t dst = smem_u32(ring) + (uint32_t)(s * Cfg::kStageBytes) + kWBytes;
             mbar_expect_tx(full_bar(s), NPAD * kTcBlockK * 2);
             tma_load_2d(dst, g.amap, kb * kTcBlockK, 0, full_bar(s));
+            if (++s == STAGES) { s = 0; par ^= 1u; }
           }
         }
       }
@@ -882,29 +882,29 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint32_t idesc = umma_idesc_bf16(NPAD);
-      long long consumed = 0;
-      int seg_idx = 0;
+      const uint64_t da0 = umma_desc(smem_u32(ring));
+      int s = 0, seg_idx = 0;
+      uint32_t par = 0;
       bool ok = true;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
         SegIter it = seg_begin(g, G, c);
         Seg sg;
         for (; ok && seg_next(g, it, sg); ++seg_idx) {
-          const int kb0 = sg.kb0, kb1 = sg.kb1;
           const int ab = seg_idx & 1;
           if (!mbar_wait(acce_bar(ab), (uint32_t)(((seg_idx >> 1) & 1) ^ 1), abort_flag)) { ok = false; break; }
-          tc_fence_after();
+          tc_fence_after();                              // the epilogue's tcgen05.ld of this accumulator come first
           const uint32_t d_tmem = tmem_base + (uint32_t)(ab * NPAD);
-          for (int kb = kb0; kb < kb1; ++kb, ++consumed) {
-            const int s = (int)(consumed % STAGES);
-            if (!mbar_wait(full_bar(s), (uint32_t)((consumed / STAGES) & 1), abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const uint32_t wa = smem_u32(ring + (size_t)s * Cfg::kStageBytes);
-            const uint64_t da = umma_desc(wa), db = umma_desc(wa + kWBytes);
+          uint32_t acc = 0u;
+          for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+            if (!mbar_wait(full_bar(s), par, abort_flag)) { ok = false; break; }
+            const uint64_t da = da0 + (uint64_t)(s * (Cfg::kStageBytes >> 4)), db = da + (uint64_t)(kWBytes >> 4);
+            umma_bf16(d_tmem, da, db, idesc, acc);
 #pragma unroll
-            for (int k = 0; k < kTcBlockK / 16; ++k)
-              umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-            umma_commit(empty_bar(s));
+            for (int k = 1; k < kTcBlockK / 16; ++k) umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, 1u);
+            acc = 1u;
+            if (s % WGS == WGS - 1) umma_commit(empty_bar(s / WGS));
+            if (++s == STAGES) { s = 0; par ^= 1u; }
           }
           if (ok) umma_commit(accf_bar(ab));
         }
@@ -1041,6 +1041,7 @@ bool fwd_persist_supported(int hd, int group) {
 int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaStream_t s) {
   if (args.R < 1 || args.R > npad || args.L > npad) return HSD_E_INVALID_ARG;
   if (args.n_run > kMaxLayersSh) return HSD_E_UNSUPPORTED;
+  if (((args.d + kTcBlockM - 1) / kTcBlockM) * 2 > sm_count) return HSD_E_UNSUPPORTED;   // norm phase: regular split only
   {  // unit arithmetic on the device is 32-bit
     long long tiles = std::max<long long>((args.V + 127) / 128, (args.ff + 63) / 64);
     long long kb = std::max(args.ff, std::max(args.d, args.nq * args.hd)) / kTcBlockK;
