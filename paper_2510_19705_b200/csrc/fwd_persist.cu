@@ -380,39 +380,51 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
       for (int n = 0; n < NTW; ++n)
 #pragma unroll
         for (int e = 0; e < 4; ++e) o[mt][n][e] = 0.f;
-#pragma unroll 1
-    for (int kt = key_lo, tile = 0; kt < key_hi; kt += kAttnTile, ++tile) {
-      const int nk = min(kAttnTile, key_hi - kt);
+    // K and V of a tile travel as two cp.async groups, each into its single buffer: K of tile t + 1 is
+    // fetched under the softmax and P V of tile t, V of tile t + 1 under the Q K^T and softmax of t + 1.
+    auto load_pages = [&](int kt, int nk, int tile) {            // page ids of a tile (tile 0 of the CTA's first item: kept across layers)
       const int pi0 = kt >> a.page_shift, n_pg = ((kt + nk - 1) >> a.page_shift) - pi0 + 1;
-      worker_sync();                                             // previous tile / item fully consumed
-      if (!(pc->tag_item == wi && pc->tag_tile == tile)) {       // page ids of this tile (kept across layers)
+      if (!(pc->tag_item == wi && pc->tag_tile == tile)) {
         if (wt < n_pg) pc->pg[wt] = a.page_table[(size_t)seq * a.pages_per_seq + pi0 + wt];
         worker_sync();
-        if (wt == 0) pc->tag_item = (wi == (int)blockIdx.x && tile == 0) ? wi : -1, pc->tag_tile = 0;
+        if (wt == 0) pc->tag_item = (wi == (int)blockIdx.x && tile == 0 && key_lo + kAttnTile >= key_hi) ? wi : -1, pc->tag_tile = 0;
       }
-      if (tile == 0) {
-        for (int i = wt; i < nqv * CPR; i += 256) {
-          const int qi = i / CPR, ch = i % CPR;
-          const int r = qi / group, gq = qi % group;
-          cp_async16(shQ + qi * RS + ch * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + gq) * HD + ch * 8);
-        }
-        if (wt < 32) { shM[wt] = -INFINITY; shL[wt] = 0.f; shC[wt] = 1.f; }
-      }
-      const int nk16 = (nk + 15) & ~15;
+    };
+    auto issue_kv = [&](const __nv_bfloat16 *pool, __nv_bfloat16 *sh, int kt, int nk, bool zero_pad) {
+      const int pi0 = kt >> a.page_shift, nk16 = (nk + 15) & ~15;
       for (int i = wt; i < nk16 * CPR; i += 256) {
         const int kk = i / CPR, ch = i % CPR;
         if (kk < nk) {
           const int key = kt + kk;
           const int pg = pc->pg[(key >> a.page_shift) - pi0];
           const size_t off = ((((size_t)pg * a.nkv + kvh) << a.page_shift) + (key & (a.page - 1))) * HD + ch * 8;
-          cp_async16(shK + kk * RS + ch * 8, kpool + off);
-          cp_async16(shV + kk * RS + ch * 8, vpool + off);
-        } else {                                                 // padding keys: P is 0 there, V must be finite
-          *reinterpret_cast<uint4 *>(shV + kk * RS + ch * 8) = make_uint4(0u, 0u, 0u, 0u);
+          cp_async16(sh + kk * RS + ch * 8, pool + off);
+        } else if (zero_pad) {                                   // padding keys: P is 0 there, V must be finite
+          *reinterpret_cast<uint4 *>(sh + kk * RS + ch * 8) = make_uint4(0u, 0u, 0u, 0u);
         }
       }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    worker_sync();                                               // previous item fully consumed
+    {
+      const int nk0 = min(kAttnTile, key_hi - key_lo);
+      load_pages(key_lo, nk0, 0);
+      for (int i = wt; i < nqv * CPR; i += 256) {
+        const int qi = i / CPR, ch = i % CPR;
+        const int r = qi / group, gq = qi % group;
+        cp_async16(shQ + qi * RS + ch * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + gq) * HD + ch * 8);
+      }
+      if (wt < 32) { shM[wt] = -INFINITY; shL[wt] = 0.f; shC[wt] = 1.f; }
+      issue_kv(kpool, shK, key_lo, nk0, false);                  // group: Q + K of tile 0
+      issue_kv(vpool, shV, key_lo, nk0, true);                   // group: V of tile 0
+    }
+#pragma unroll 1
+    for (int kt = key_lo, tile = 0; kt < key_hi; kt += kAttnTile, ++tile) {
+      const int nk = min(kAttnTile, key_hi - kt);
+      const int nk16 = (nk + 15) & ~15;
+      const int kt_next = kt + kAttnTile, nk_next = min(kAttnTile, key_hi - kt_next);
       prof_mark(a, wt, 5);
-      cp_async_wait_all();
+      asm volatile("cp.async.wait_group 1;" ::: "memory");       // K of this tile (and Q) landed; V may be in flight
       worker_sync();
       prof_mark(a, wt, 6);
       // ---- S = scale * Q K^T, masked: (m-tile, 8-key n-tile) pairs over the warps
@@ -444,6 +456,12 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
         }
       }
       worker_sync();
+      if (nk_next > 0) {                                         // K buffer is free: fetch the next tile's keys
+        load_pages(kt_next, nk_next, tile + 1);
+        issue_kv(kpool, shK, kt_next, nk_next, false);
+      } else {
+        asm volatile("cp.async.commit_group;" ::: "memory");     // keep the group count uniform
+      }
       // ---- online softmax per query row; P (bf16) overwrites the row of S it came from
 #pragma unroll 1
       for (int row = warp; row < n_mt * 16; row += 8) {
@@ -475,6 +493,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
         for (int off = 16; off > 0; off >>= 1) ps += __shfl_xor_sync(0xFFFFFFFFu, ps, off);
         if (lane == 0) { shM[row] = m_new; shL[row] = shL[row] * corr + ps; shC[row] = corr; }
       }
+      asm volatile("cp.async.wait_group 1;" ::: "memory");       // V of this tile landed; the next K may be in flight
       worker_sync();
       // ---- O = O * corr + P V: each warp owns NTW 8-wide slices of the head dimension
 #pragma unroll
@@ -507,7 +526,14 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
           }
         }
       }
+      if (nk_next > 0) {
+        worker_sync();                                           // V buffer is free: fetch the next tile's values
+        issue_kv(vpool, shV, kt_next, nk_next, true);
+      } else {
+        asm volatile("cp.async.commit_group;" ::: "memory");
+      }
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     prof_mark(a, wt, 7);
     // ---- partial (o, m, l) of this split
 #pragma unroll

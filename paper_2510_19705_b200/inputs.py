@@ -36,6 +36,11 @@ WORKLOADS = {
     # CPU oracle finishes in seconds; spans several GEMM tiles and ragged tails.
     "mini3": dict(model=model_cfg(6, 256, 8, 2, 704, 2048, "bf16", head_dim=32), exits=(1, 3, 6),
                   T=(3, 2), batch=1, prompt=24, n_new=48, page=16, weight_seed=7, prompt_seed=7),
+    # small stand-in with the long-context config's structure: 4 levels, draft lengths (2, 2, 3), a batch,
+    # 16-token pages, head size 128, and prompts long enough that every attention key split spans
+    # several key tiles and many pages.
+    "mini4long": dict(model=model_cfg(6, 256, 4, 1, 704, 2048, "bf16", head_dim=128), exits=(1, 2, 4, 6),
+                      T=(2, 2, 3), batch=2, prompt=1900, n_new=24, page=16, weight_seed=9, prompt_seed=9),
 }
 
 

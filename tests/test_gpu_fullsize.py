@@ -180,3 +180,38 @@ def test_bf16_batch_decisions_and_logits(lib, tmp_path):
         om.rows(2, ctx_b, drafts_b)
         ref_p = _perturbed_oracle_logits(cfg, om.w, wl["exits"], 2, ctx_b, drafts_b)
         _assert_bf16_logits_close(rec["logits"], om.last_logits64, ref_p, ("mini3 batch", b))
+
+
+def test_long_context_four_levels_paged_batch(lib, tmp_path):
+    """The long-context configuration's structure at a size the oracle can follow: 4 levels with draft lengths
+    (2, 2, 3), two sequences, 16-token pages, 1900-token prompts (every attention key split spans more than one
+    key tile and several pages).  Every decision follows the oracle on the logged logits; each sequence's first
+    verification at the top level and at level 1 matches the oracle's forward."""
+    wl = inputs.WORKLOADS["mini4long"]
+    cfg, T, B, n_new, seed = wl["model"], wl["T"], wl["batch"], wl["n_new"], 6
+    w_cpu = inputs.make_weights(cfg, wl["weight_seed"])
+    w = {k: (v.cuda() if k != "layers" else [{n: t.cuda() for n, t in l.items()} for l in v]) for k, v in w_cpu.items()}
+    prompts = inputs.make_prompts(cfg["vocab"], B, wl["prompt"], wl["prompt_seed"])
+    eng = lib.Hsd(cfg, w, wl["exits"], T, max_batch=B, max_seq=wl["prompt"] + n_new + 32, page_size=wl["page"])
+    path = str(tmp_path / "trace.bin")
+    eng.set_trace(path, logit_calls=10 ** 6)
+    toks, stats, _ = eng.generate(prompts.cuda(), n_new, seed)
+    eng.set_trace(None)
+    eng.close()
+    _check_run_properties(stats, T, n_new * B)
+    recs = lib.read_trace(path)
+    assert _replay_decisions(recs, seed, n_seq=B) == sum(s["calls"] for s in stats[1:])
+    w_np = inputs.weights_to_numpy(w_cpu)
+    om = Transformer(cfg, w_np, wl["exits"])
+    for b in range(B):
+        prompt = prompts[b].tolist()
+        final = _context_of(recs, None, prompt, b)
+        assert final[len(prompt):len(prompt) + n_new] == toks[b].cpu().tolist()
+        for lvl in (1, len(T)):
+            rec = next(r for r in recs if r["seq"] == b and r["level"] == lvl)
+            om.reset()
+            ctx_b, drafts_b = _context_of(recs, rec, prompt, b), rec["tokens"][:-1].tolist()
+            om.rows(lvl, ctx_b, drafts_b)
+            ref = om.last_logits64.copy()
+            ref_p = _perturbed_oracle_logits(cfg, w_np, wl["exits"], lvl, ctx_b, drafts_b)
+            _assert_bf16_logits_close(rec["logits"], ref, ref_p, ("mini4long", b, lvl))
