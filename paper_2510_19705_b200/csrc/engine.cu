@@ -178,6 +178,7 @@ struct hsd_ctx {
   uint64_t seed;
   // tensor-core GEMM state (bf16 models)
   bool use_tc, use_persist;
+  int attn_single_max = 0;                    // contexts up to this many keys use one attention key split
   int sm_count;
   std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + 1]: wq wk wv wo wg wu wd per layer, then lm_head
   CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
@@ -352,8 +353,10 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
 
   // attention split: enough blocks to fill the GPU, never more partial rows than the buffer holds
   const int blocks_target = c->use_persist ? c->sm_count : kAttnBlocksTarget;
-  const int max_splits = c->use_persist ? 20 : kMaxSplits;      // the persistent merge phase takes <= 20 splits
+  int max_splits = c->use_persist ? 20 : kMaxSplits;      // the persistent merge phase takes <= 20 splits
+  if (c->use_persist) if (const char *e = getenv("HSD_ATTN_SPLITS_MAX")) max_splits = std::max(1, std::min(20, atoi(e)));
   int n_splits = std::max(1, std::min(max_splits, blocks_target / std::max(1, n_attn * md.nkv)));
+  if (c->use_persist && max_kv <= c->attn_single_max) n_splits = 1;   // short contexts: one split, no merge phase
   int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, c->use_persist ? 16 : kAttnKeyTile);
   n_splits = (max_kv + keys_per_split - 1) / keys_per_split;
   if ((size_t)R * n_splits > (size_t)L.partial_rows) return HSD_E_INVALID_ARG;
@@ -746,8 +749,9 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
       int coop = 0, dev = 0;
       cudaGetDevice(&dev);
       cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-      c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 && (md.d / kTcBlockM) * 2 <= c->sm_count && md.n_layers <= 64 && (md.page & (md.page - 1)) == 0 &&
+      c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 && (md.d / kTcBlockM) * 2 <= c->sm_count && md.n_layers <= 64 && (md.page & (md.page - 1)) == 0 && md.page >= 16 &&
                        getenv("HSD_NO_PERSIST") == nullptr;
+      if (const char *e = getenv("HSD_ATTN_SINGLE_MAX")) c->attn_single_max = atoi(e);
     }
     if (!st && cudaMallocHost(&c->status_host, 4) != cudaSuccess) st = HSD_E_CUDA;
     if (st) {

@@ -23,7 +23,7 @@ using namespace ptx;
 
 constexpr int kWBytes = kTcBlockM * kTcBlockK * 2;     // 16 KiB weight tile
 constexpr int kBoxBytes = kTcBoxRows * kTcBlockK * 2;  // 8 KiB TMA box
-constexpr int kScratchBytes = 78 * 1024;               // union: epilogue staging / attention tiles, + rope cache
+constexpr int kScratchBytes = 78 * 1024;               // union: epilogue staging / attention buffers, + rope cache
 constexpr int kCtrlBytes = 4096;                       // barriers, flags, page-id cache, per-row info
 constexpr int kSmemTotal = 232448;
 constexpr int kKeyTile = 32;
@@ -168,9 +168,10 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
 }
 __device__ __forceinline__ float bf(const __nv_bfloat16 v) { return __bfloat162float(v); }
 
-// Debug timeline: CTA 0's first worker thread stamps slot 960 + k (only when profiling is on).
+// Debug timeline: CTA 0's first worker thread adds the time to slot 960 + k (only when profiling is on;
+// differences of two slots hit equally often give summed intervals).
 __device__ __forceinline__ void prof_mark(const FwdArgs &a, int wt, int k) {
-  if (a.prof && wt == 0 && blockIdx.x == 0) a.prof[960 + k] = globaltimer_ns();
+  if (a.prof && wt == 0 && blockIdx.x == 0) a.prof[960 + k] += globaltimer_ns();
 }
 
 // Grid-wide barrier of the worker threads.  `epoch` counts barriers; the counter only grows.
@@ -312,13 +313,10 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
 
 // ------------------------------------------------------------------------------ attention phases
 // Under the weight stream every dependent global round trip costs microseconds, so the attention is
-// two phases of one load batch each.  Phase A: work item = (attention item, KV head, key split); the
-// q rows and a tile of up to kAttnTile keys (K and V) arrive together through cp.async, scores /
-// softmax / P.V run out of shared memory, the partial (o, m, l) goes to global memory.  Phase B
-// (after a grid barrier): one (row, head) per 128 threads merges the partials of its splits.
-constexpr int kAttnTile = 80;                          // keys per tile (three 32-key sub-tiles, the last partial)
-constexpr int kAttnPStride = 96;
-constexpr int kRopeCacheRows = 16;                     // rows whose cos / sin values are kept in shared memory
+// two phases.  Phase A: work item = (attention item, KV head, key split), partial (o, m, l) to global
+// memory.  Phase B (after a grid barrier): one (row, head) per 128 threads merges the partials of its
+// splits.
+constexpr int kRopeCacheRows = 12;                     // rows whose cos / sin values are kept in shared memory
 constexpr int kAttnMaxSplits = 20;
 
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
@@ -330,7 +328,7 @@ __device__ __forceinline__ void cp_async_wait_all() {
 __device__ __forceinline__ float bf_lo(unsigned w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf_hi(unsigned w) { return __uint_as_float(w & 0xFFFF0000u); }
 
-struct PageCache { int tag_item, tag_tile; int pg[128]; };
+struct PageCache { int tag_item, tag_tile; int pg[128]; };   // pg[warp * 16 + j]: page of the warp's j-th sub-tile
 
 __device__ __forceinline__ void mma_bf16_16x8x16(float *c, const unsigned *a, unsigned b0, unsigned b1) {
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -341,31 +339,43 @@ __device__ __forceinline__ void ldmatrix_x2_trans(unsigned &r0, unsigned &r1, co
   asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(smem_u32(row_ptr)));
 }
 
-// Phase A on the (legacy) tensor path: S = Q K^T and O += P V with mma.sync m16n8k16, fp32 softmax in
-// between.  Shared memory: K, V, Q as bf16 rows padded by 16 bytes (conflict-free fragment loads),
-// S as fp32 [32][84] with P (bf16 hi and lo halves) written in place over each S row, running (m, l,
-// corr) per query.
+// Phase A: warp-level online softmax.  A work item is (attention item, KV head, key split); its keys
+// are cut into 16-key sub-tiles (one KV page or part of one: the launcher requires pages of >= 16
+// tokens) that the warps take in turn, each warp with its own running (m, l, O) in registers and its
+// own K and V sub-tile buffers, so nothing synchronises the CTA inside the key loop.  S = Q K^T and
+// O += P V run on mma.sync m16n8k16 (the S accumulators are re-packed as the A operand of P V; P is
+// split into bf16 hi + lo halves, so P V keeps ~16 bits of P); K of the warp's next sub-tile is fetched
+// under the softmax and P V of this one, the next V under the next Q K^T.  With up to 16 query vectors
+// (rows x group) every warp works on its own sub-tiles; with 17..32 the warps pair up on a sub-tile,
+// one 16-row m-tile each.  At the end the warps' states are merged through shared memory and the
+// split's partial (o, m, l) goes to global memory.
 template <int HD>
-__device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt) {
+__device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt, long long *dbg) {
   constexpr int CPR = HD / 8;                      // 16-byte chunks per row
-  constexpr int RS = HD + 8;                       // padded row stride (bf16 elements)
-  constexpr int SS = 84;                           // S row stride (floats)
-  constexpr int kPLoOff = 84;                      // bf16 offset of the low half of P inside its S row
+  // Rows of Q, K, V in shared memory: HD >= 64: unpadded, the 16-byte chunk index XORed with the row's low
+  // three bits; HD = 32: padded by 16 bytes.  Either way the fragment loads (eight rows, same chunk) and
+  // ldmatrix (eight rows of one 8x8 block) touch all banks once.
+  constexpr bool SWZ = HD >= 64;
+  constexpr int RS = SWZ ? HD : HD + 8;            // row stride (bf16 elements)
+  auto swz = [](int row, int chunk) { return SWZ ? (chunk ^ (row & 7)) : chunk; };
   constexpr int KST = HD / 16;                     // k-steps of Q K^T
-  constexpr int NTW = (HD / 8 + 7) / 8;            // output n-tiles (8 dims) per warp
+  constexpr int NT = HD / 8;                       // 8-wide output n-tiles
+  constexpr int MS = HD + 8;                       // merge row: o[HD], m, l; stride = 8 mod 32 words: conflict-free float2 stores
   const int group = a.nq / a.nkv;
   const int warp = wt >> 5, lane = wt & 31, g = lane >> 2, t = lane & 3;
-  __nv_bfloat16 *shK = reinterpret_cast<__nv_bfloat16 *>(scratch);             // [kAttnTile][RS]
-  __nv_bfloat16 *shV = shK + kAttnTile * RS;                                   // [kAttnTile][RS]
-  __nv_bfloat16 *shQ = shV + kAttnTile * RS;                                   // [32][RS]
-  float *shS = reinterpret_cast<float *>(shQ + 32 * RS);                       // [32][SS]; P in place
-  float *shM = shS + 32 * SS, *shL = shM + 32, *shC = shL + 32;                // running max, sum, correction
+  __nv_bfloat16 *shQ = reinterpret_cast<__nv_bfloat16 *>(scratch);                              // [32][RS]
+  __nv_bfloat16 *shK = shQ + 32 * RS + warp * (32 * RS);                                        // this warp's [16][RS]
+  __nv_bfloat16 *shV = shK + 16 * RS;                                                           // this warp's [16][RS]
+  float *shMerge = reinterpret_cast<float *>(scratch);                                          // [8 warps][16][MS], over Q and the K/V buffers
+  static_assert(8 * 16 * MS * 4 <= 9 * 32 * RS * 2, "merge area must fit the Q and K/V buffers");
+  static_assert(9 * 32 * RS * 2 <= kScratchBytes - 2 * kRopeCacheRows * (HD / 2) * 4, "attention buffers overlap the rope cache");
   const __nv_bfloat16 *kpool = lay.k_pool, *vpool = lay.v_pool;
   const float scale = rsqrtf((float)HD);
   const int n_work = a.n_attn * a.nkv * a.n_splits;
 #pragma unroll 1
   for (int wi = blockIdx.x; wi < n_work; wi += gridDim.x) {
-    prof_mark(a, wt, 4);
+    long long cyc = clock64();
+    auto lap = [&](int k) { if (a.prof && wt == 0 && blockIdx.x == 0) { const long long n_ = clock64(); dbg[k] += n_ - cyc; cyc = n_; } };
     const int split = wi % a.n_splits, kvh = (wi / a.n_splits) % a.nkv, ai = wi / (a.n_splits * a.nkv);
     const int4 it = a.attn_items[ai];
     const int row0 = it.x, nrows = it.y, seq = it.z, pos0 = it.w;
@@ -373,196 +383,211 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
     const int key_lo = split * a.keys_per_split, key_hi = min(kv_len, key_lo + a.keys_per_split);
     if (key_lo >= kv_len) continue;                              // uniform over the CTA
     const int nqv = nrows * group, n_mt = (nqv + 15) >> 4;
-    float o[2][NTW][4];
-#pragma unroll
-    for (int mt = 0; mt < 2; ++mt)
-#pragma unroll
-      for (int n = 0; n < NTW; ++n)
-#pragma unroll
-        for (int e = 0; e < 4; ++e) o[mt][n][e] = 0.f;
-    // K and V of a tile travel as two cp.async groups, each into its single buffer: K of tile t + 1 is
-    // fetched under the softmax and P V of tile t, V of tile t + 1 under the Q K^T and softmax of t + 1.
-    auto load_pages = [&](int kt, int nk, int tile) {            // page ids of a tile (tile 0 of the CTA's first item: kept across layers)
-      const int pi0 = kt >> a.page_shift, n_pg = ((kt + nk - 1) >> a.page_shift) - pi0 + 1;
-      if (!(pc->tag_item == wi && pc->tag_tile == tile)) {
-        if (wt < n_pg) pc->pg[wt] = a.page_table[(size_t)seq * a.pages_per_seq + pi0 + wt];
-        worker_sync();
-        if (wt == 0) pc->tag_item = (wi == (int)blockIdx.x && tile == 0 && key_lo + kAttnTile >= key_hi) ? wi : -1, pc->tag_tile = 0;
+    const int n_sub = (key_hi - key_lo + 15) >> 4;
+    const int first = n_mt == 2 ? (warp >> 1) : warp, step = n_mt == 2 ? 4 : 8, mt = n_mt == 2 ? (warp & 1) : 0;
+    const int n_mine = first < n_sub ? (n_sub - first + step - 1) / step : 0;       // sub-tiles of this warp
+    worker_sync();                                               // previous item's merge area fully read
+    // ---- q rows of the item (whole CTA) and this warp's page ids: lane j holds the page of the warp's j-th
+    //      sub-tile (re-read every 32 sub-tiles); kept in shared memory across layers when the CTA has one item
+    for (int i = wt; i < nqv * CPR; i += 256) {
+      const int qi = i / CPR, ch = i % CPR;
+      const int r = qi / group, gq = qi % group;
+      cp_async16(shQ + qi * RS + swz(qi, ch) * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + gq) * HD + ch * 8);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    const bool pages_cached = (pc->tag_item == wi) && n_mine <= 16;
+    int pg_reg = 0, pg_base = 0;
+    auto load_pages = [&](int j0) {                              // pages of sub-tiles j0 .. j0 + 31 of this warp
+      pg_base = j0;
+      const int j = j0 + lane;
+      if (j < n_mine) {
+        if (pages_cached) pg_reg = pc->pg[warp * 16 + j];
+        else {
+          const int key = key_lo + (first + j * step) * 16;
+          pg_reg = a.page_table[(size_t)seq * a.pages_per_seq + (key >> a.page_shift)];
+          if (n_mine <= 16) pc->pg[warp * 16 + j] = pg_reg;
+        }
       }
     };
-    auto issue_kv = [&](const __nv_bfloat16 *pool, __nv_bfloat16 *sh, int kt, int nk, bool zero_pad) {
-      const int pi0 = kt >> a.page_shift, nk16 = (nk + 15) & ~15;
-      for (int i = wt; i < nk16 * CPR; i += 256) {
-        const int kk = i / CPR, ch = i % CPR;
-        if (kk < nk) {
-          const int key = kt + kk;
-          const int pg = pc->pg[(key >> a.page_shift) - pi0];
-          const size_t off = ((((size_t)pg * a.nkv + kvh) << a.page_shift) + (key & (a.page - 1))) * HD + ch * 8;
-          cp_async16(sh + kk * RS + ch * 8, pool + off);
-        } else if (zero_pad) {                                   // padding keys: P is 0 there, V must be finite
-          *reinterpret_cast<uint4 *>(sh + kk * RS + ch * 8) = make_uint4(0u, 0u, 0u, 0u);
-        }
+    load_pages(0);
+    auto issue = [&](const __nv_bfloat16 *pool, __nv_bfloat16 *sh, int j, bool zero_pad) {    // one sub-tile, one operand
+      const int kt = key_lo + (first + j * step) * 16, nk = min(16, key_hi - kt);
+      const int pg = __shfl_sync(0xFFFFFFFFu, pg_reg, j - pg_base);
+      const size_t base = ((((size_t)pg * a.nkv + kvh) << a.page_shift) + (kt & (a.page - 1))) * HD;
+#pragma unroll
+      for (int i = 0; i < 16 * CPR / 32; ++i) {
+        const int idx = i * 32 + lane, kk = idx / CPR, ch = idx % CPR;
+        if (kk < nk) cp_async16(sh + kk * RS + swz(kk, ch) * 8, pool + base + (size_t)kk * HD + ch * 8);
+        else if (zero_pad) *reinterpret_cast<uint4 *>(sh + kk * RS + ch * 8) = make_uint4(0u, 0u, 0u, 0u);   // P is 0 there, V must be finite
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    worker_sync();                                               // previous item fully consumed
-    {
-      const int nk0 = min(kAttnTile, key_hi - key_lo);
-      load_pages(key_lo, nk0, 0);
-      for (int i = wt; i < nqv * CPR; i += 256) {
-        const int qi = i / CPR, ch = i % CPR;
-        const int r = qi / group, gq = qi % group;
-        cp_async16(shQ + qi * RS + ch * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + gq) * HD + ch * 8);
-      }
-      if (wt < 32) { shM[wt] = -INFINITY; shL[wt] = 0.f; shC[wt] = 1.f; }
-      issue_kv(kpool, shK, key_lo, nk0, false);                  // group: Q + K of tile 0
-      issue_kv(vpool, shV, key_lo, nk0, true);                   // group: V of tile 0
-    }
-#pragma unroll 1
-    for (int kt = key_lo, tile = 0; kt < key_hi; kt += kAttnTile, ++tile) {
-      const int nk = min(kAttnTile, key_hi - kt);
-      const int nk16 = (nk + 15) & ~15;
-      const int kt_next = kt + kAttnTile, nk_next = min(kAttnTile, key_hi - kt_next);
-      prof_mark(a, wt, 5);
-      asm volatile("cp.async.wait_group 1;" ::: "memory");       // K of this tile (and Q) landed; V may be in flight
-      worker_sync();
-      prof_mark(a, wt, 6);
-      // ---- S = scale * Q K^T, masked: (m-tile, 8-key n-tile) pairs over the warps
-      const int n_nt = (nk + 7) >> 3;
-#pragma unroll 1
-      for (int pair = warp; pair < n_mt * n_nt; pair += 8) {
-        const int mt = pair / n_nt, nt = pair % n_nt;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        const __nv_bfloat16 *qa = shQ + (mt * 16 + g) * RS + 2 * t;
-        const __nv_bfloat16 *kb = shK + (nt * 8 + g) * RS + 2 * t;
+    if (n_mine > 0) { issue(kpool, shK, 0, false); issue(vpool, shV, 0, true); }
+    else { asm volatile("cp.async.commit_group;\n\tcp.async.commit_group;" ::: "memory"); }
+    float o[NT][4];
 #pragma unroll
-        for (int ks = 0; ks < KST; ++ks) {
-          unsigned af[4];
-          af[0] = *reinterpret_cast<const unsigned *>(qa + ks * 16);
-          af[1] = *reinterpret_cast<const unsigned *>(qa + 8 * RS + ks * 16);
-          af[2] = *reinterpret_cast<const unsigned *>(qa + ks * 16 + 8);
-          af[3] = *reinterpret_cast<const unsigned *>(qa + 8 * RS + ks * 16 + 8);
-          const unsigned b0 = *reinterpret_cast<const unsigned *>(kb + ks * 16);
-          const unsigned b1 = *reinterpret_cast<const unsigned *>(kb + ks * 16 + 8);
-          mma_bf16_16x8x16(acc, af, b0, b1);
-        }
+    for (int n = 0; n < NT; ++n)
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const int row = mt * 16 + g + ((e & 2) ? 8 : 0), kk = nt * 8 + 2 * t + (e & 1);
-          const int qpos = pos0 + row / group;
-          float v = acc[e] * scale;
-          if (kk >= nk || kt + kk > qpos) v = -INFINITY;
-          shS[row * SS + kk] = v;
+      for (int e = 0; e < 4; ++e) o[n][e] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    const int qrow[2] = {mt * 16 + g, mt * 16 + g + 8};          // query vectors of this thread's accumulator rows
+    const int qpos[2] = {pos0 + qrow[0] / group, pos0 + qrow[1] / group};
+    asm volatile("cp.async.wait_group 2;" ::: "memory");         // q rows landed (this thread's copies)
+    worker_sync();                                               // ... and everybody's; page ids of the item stored
+    if (wt == 0) pc->tag_item = (wi == (int)blockIdx.x && n_work <= (int)gridDim.x) ? wi : -1;
+    lap(0);
+#pragma unroll 1
+    for (int j = 0; j < n_mine; ++j) {
+      const int kt = key_lo + (first + j * step) * 16;
+      if (j + 1 < n_mine && j + 1 - pg_base >= 32) load_pages(j + 1);
+      asm volatile("cp.async.wait_group 1;" ::: "memory");       // K of this sub-tile landed; V may be in flight
+      __syncwarp();
+      // ---- S = Q K^T for 16 query vectors x 16 keys
+      float sacc[2][4];
+#pragma unroll
+      for (int n = 0; n < 2; ++n)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) sacc[n][e] = 0.f;
+      // rows g and g + 8 of a fragment share the low row bits (g), so one swizzled chunk offset serves both
+      const __nv_bfloat16 *qa = shQ + (mt * 16 + g) * RS + 2 * t;
+#pragma unroll
+      for (int ks = 0; ks < KST; ++ks) {
+        const int c0 = swz(g, 2 * ks) * 8, c1 = swz(g, 2 * ks + 1) * 8;
+        unsigned af[4];
+        af[0] = *reinterpret_cast<const unsigned *>(qa + c0);
+        af[1] = *reinterpret_cast<const unsigned *>(qa + 8 * RS + c0);
+        af[2] = *reinterpret_cast<const unsigned *>(qa + c1);
+        af[3] = *reinterpret_cast<const unsigned *>(qa + 8 * RS + c1);
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+          const __nv_bfloat16 *kb = shK + (n * 8 + g) * RS + 2 * t;
+          mma_bf16_16x8x16(sacc[n], af, *reinterpret_cast<const unsigned *>(kb + c0), *reinterpret_cast<const unsigned *>(kb + c1));
         }
       }
-      worker_sync();
-      if (nk_next > 0) {                                         // K buffer is free: fetch the next tile's keys
-        load_pages(kt_next, nk_next, tile + 1);
-        issue_kv(kpool, shK, kt_next, nk_next, false);
-      } else {
-        asm volatile("cp.async.commit_group;" ::: "memory");     // keep the group count uniform
-      }
-      // ---- online softmax per query row; P (bf16) overwrites the row of S it came from
-#pragma unroll 1
-      for (int row = warp; row < n_mt * 16; row += 8) {
-        float sv[3];
+      __syncwarp();                                              // every lane is done with the K buffer
+      if (j + 1 < n_mine) issue(kpool, shK, j + 1, false);
+      else asm volatile("cp.async.commit_group;" ::: "memory");  // keep the group count uniform
+      // ---- online softmax on the accumulator rows (g and g + 8); P re-packed as the A operand of P V
+      unsigned ph[4], pl[4];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        float sv[4];
         float mx = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 3; ++j) {
-          const int kk = j * 32 + lane;
-          sv[j] = (kk < nk && row < nqv) ? shS[row * SS + kk] : -INFINITY;
-          mx = fmaxf(mx, sv[j]);
-        }
-        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, off));
-        const float m_old = shM[row], m_new = fmaxf(m_old, mx);
-        const float corr = (m_new > -INFINITY) ? __expf(m_old - m_new) : 1.f;
-        float ps = 0.f;
-        __syncwarp();                                            // every lane has read its S values
-        __nv_bfloat16 *prow = reinterpret_cast<__nv_bfloat16 *>(shS + row * SS);
+        for (int n = 0; n < 2; ++n)
 #pragma unroll
-        for (int j = 0; j < 3; ++j) {
-          const int kk = j * 32 + lane;
-          const float pv = (m_new > -INFINITY && sv[j] > -INFINITY) ? __expf(sv[j] - m_new) : 0.f;
-          // P = hi + lo in bf16 (two MMAs against V): the product keeps ~16 bits of P, so the attention
-          // output is as accurate as an fp32 P would give
-          const __nv_bfloat16 ph = __float2bfloat16_rn(pv);
-          const __nv_bfloat16 pl = __float2bfloat16_rn(pv - __bfloat162float(ph));
-          ps += pv;
-          if (kk < nk16) { prow[kk] = ph; prow[kPLoOff + kk] = pl; }
-        }
-        for (int off = 16; off > 0; off >>= 1) ps += __shfl_xor_sync(0xFFFFFFFFu, ps, off);
-        if (lane == 0) { shM[row] = m_new; shL[row] = shL[row] * corr + ps; shC[row] = corr; }
-      }
-      asm volatile("cp.async.wait_group 1;" ::: "memory");       // V of this tile landed; the next K may be in flight
-      worker_sync();
-      // ---- O = O * corr + P V: each warp owns NTW 8-wide slices of the head dimension
-#pragma unroll
-      for (int mt = 0; mt < 2; ++mt) {
-        if (mt < n_mt) {
-          const float c0 = shC[mt * 16 + g], c1 = shC[mt * 16 + g + 8];
-          const __nv_bfloat16 *pa = reinterpret_cast<const __nv_bfloat16 *>(shS + (mt * 16 + g) * SS) + 2 * t;
-#pragma unroll
-          for (int n = 0; n < NTW; ++n) {
-            const int n0 = (warp * NTW + n) * 8;
-            if (n0 < HD) {
-              o[mt][n][0] *= c0; o[mt][n][1] *= c0; o[mt][n][2] *= c1; o[mt][n][3] *= c1;
-#pragma unroll 1
-              for (int ks = 0; ks < (nk16 >> 4); ++ks) {
-                unsigned af[4];
-                af[0] = *reinterpret_cast<const unsigned *>(pa + ks * 16);
-                af[1] = *reinterpret_cast<const unsigned *>(pa + 8 * SS * 2 + ks * 16);
-                af[2] = *reinterpret_cast<const unsigned *>(pa + ks * 16 + 8);
-                af[3] = *reinterpret_cast<const unsigned *>(pa + 8 * SS * 2 + ks * 16 + 8);
-                unsigned b0, b1;
-                ldmatrix_x2_trans(b0, b1, shV + (ks * 16 + (lane & 15)) * RS + n0);
-                mma_bf16_16x8x16(o[mt][n], af, b0, b1);
-                af[0] = *reinterpret_cast<const unsigned *>(pa + kPLoOff + ks * 16);
-                af[1] = *reinterpret_cast<const unsigned *>(pa + kPLoOff + 8 * SS * 2 + ks * 16);
-                af[2] = *reinterpret_cast<const unsigned *>(pa + kPLoOff + ks * 16 + 8);
-                af[3] = *reinterpret_cast<const unsigned *>(pa + kPLoOff + 8 * SS * 2 + ks * 16 + 8);
-                mma_bf16_16x8x16(o[mt][n], af, b0, b1);
-              }
-            }
+          for (int e = 0; e < 2; ++e) {
+            const int key = kt + n * 8 + 2 * t + e;
+            float v = sacc[n][h * 2 + e] * scale;
+            if (key >= key_hi || key > qpos[h] || qrow[h] >= nqv) v = -INFINITY;
+            sv[n * 2 + e] = v;
+            mx = fmaxf(mx, v);
           }
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, 2));
+        const float m_new = fmaxf(m_run[h], mx);
+        const float corr = (m_new > -INFINITY) ? __expf(m_run[h] - m_new) : 1.f;
+        float ps = 0.f, pv[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          pv[i] = (sv[i] > -INFINITY) ? __expf(sv[i] - m_new) : 0.f;
+          ps += pv[i];
+        }
+        m_run[h] = m_new;
+        l_run[h] = l_run[h] * corr + ps;                         // this thread's columns only; summed over t at the end
+#pragma unroll
+        for (int n = 0; n < NT; ++n) { o[n][h * 2] *= corr; o[n][h * 2 + 1] *= corr; }
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {                            // A fragment: a[h] <- keys 2t.. of n-tile 0, a[2 + h] <- n-tile 1
+          const __nv_bfloat162 hi = __floats2bfloat162_rn(pv[n * 2], pv[n * 2 + 1]);
+          const float2 hf = __bfloat1622float2(hi);
+          const __nv_bfloat162 lo = __floats2bfloat162_rn(pv[n * 2] - hf.x, pv[n * 2 + 1] - hf.y);
+          ph[n * 2 + h] = *reinterpret_cast<const unsigned *>(&hi);
+          pl[n * 2 + h] = *reinterpret_cast<const unsigned *>(&lo);
         }
       }
-      if (nk_next > 0) {
-        worker_sync();                                           // V buffer is free: fetch the next tile's values
-        issue_kv(vpool, shV, kt_next, nk_next, true);
-      } else {
-        asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 1;" ::: "memory");       // V of this sub-tile landed; the next K may be in flight
+      __syncwarp();
+      // ---- O += P V
+#pragma unroll
+      for (int n = 0; n < NT; ++n) {
+        unsigned b0, b1;
+        ldmatrix_x2_trans(b0, b1, shV + (lane & 15) * RS + swz(lane & 15, n) * 8);
+        mma_bf16_16x8x16(o[n], ph, b0, b1);
+        mma_bf16_16x8x16(o[n], pl, b0, b1);
       }
+      __syncwarp();                                              // every lane is done with the V buffer
+      if (j + 1 < n_mine) issue(vpool, shV, j + 1, true);
+      else asm volatile("cp.async.commit_group;" ::: "memory");
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-    prof_mark(a, wt, 7);
-    // ---- partial (o, m, l) of this split
+    lap(1);
+    // ---- merge the warps' states: each warp writes (o, m, l) of its 16 query vectors over the K/V buffers
 #pragma unroll
-    for (int mt = 0; mt < 2; ++mt) {
-      if (mt < n_mt) {
+    for (int h = 0; h < 2; ++h) {
+      l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 1);
+      l_run[h] += __shfl_xor_sync(0xFFFFFFFFu, l_run[h], 2);
+    }
+    worker_sync();                                               // all warps are done with their K/V buffers
+    lap(2);
+    {
+      float *mine = shMerge + (size_t)warp * 16 * MS;
+      if (n_mine > 0) {
 #pragma unroll
-        for (int n = 0; n < NTW; ++n) {
-          const int n0 = (warp * NTW + n) * 8;
-          if (n0 < HD) {
-#pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-              const int qi = mt * 16 + g + hh * 8;
-              if (qi < nqv) {
-                const int r = row0 + qi / group, h = kvh * group + qi % group;
-                float *dst = a.attn_partials + (((size_t)r * a.nq + h) * a.n_splits + split) * (HD + 2) + n0 + 2 * t;
-                dst[0] = o[mt][n][hh * 2];
-                dst[1] = o[mt][n][hh * 2 + 1];
-              }
-            }
-          }
+        for (int n = 0; n < NT; ++n) {
+          if (qrow[0] < nqv) *reinterpret_cast<float2 *>(mine + g * MS + n * 8 + 2 * t) = make_float2(o[n][0], o[n][1]);
+          if (qrow[1] < nqv) *reinterpret_cast<float2 *>(mine + (g + 8) * MS + n * 8 + 2 * t) = make_float2(o[n][2], o[n][3]);
         }
       }
+      if (t == 0) {                                              // a warp without keys contributes m = -inf only
+        mine[g * MS + HD] = m_run[0]; mine[g * MS + HD + 1] = l_run[0];
+        mine[(g + 8) * MS + HD] = m_run[1]; mine[(g + 8) * MS + HD + 1] = l_run[1];
+      }
     }
-    if (wt < nqv) {
-      const int r = row0 + wt / group, h = kvh * group + wt % group;
-      float *dst = a.attn_partials + (((size_t)r * a.nq + h) * a.n_splits + split) * (HD + 2);
-      dst[HD] = shM[wt];
-      dst[HD + 1] = shL[wt];
+    worker_sync();
+    lap(3);
+#pragma unroll 1
+    for (int idx = wt; idx < nqv * (HD / 2); idx += 256) {       // two output dims per thread
+      const int qi = idx / (HD / 2), dd = (idx % (HD / 2)) * 2;
+      const int w0 = n_mt == 2 ? (qi >> 4) : 0, wstep = n_mt == 2 ? 2 : 1, rr = qi & 15;
+      const float *src0 = shMerge + ((size_t)w0 * 16 + rr) * MS;
+      const int wstride = wstep * 16 * MS, nw = min(n_mt == 2 ? 4 : 8, n_sub);     // warps (pairs) that had keys
+      // one pass, all loads of four warps' states in flight together
+      float mm = -INFINITY, l = 0.f, ox = 0.f, oy = 0.f;
+#pragma unroll 1
+      for (int k0 = 0; k0 < nw; k0 += 4) {
+        float mw[4], lw[4];
+        float2 ov[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float *src = src0 + (k0 + i) * wstride;
+          const bool on = k0 + i < nw;
+          mw[i] = on ? src[HD] : -INFINITY;
+          lw[i] = on ? src[HD + 1] : 0.f;
+          ov[i] = on ? *reinterpret_cast<const float2 *>(src + dd) : make_float2(0.f, 0.f);
+        }
+        float mn = mm;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) mn = fmaxf(mn, mw[i]);
+        const float c0 = (mn > -INFINITY) ? __expf(mm - mn) : 1.f;
+        l *= c0; ox *= c0; oy *= c0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float sc = (mw[i] > -INFINITY) ? __expf(mw[i] - mn) : 0.f;
+          l += sc * lw[i]; ox += sc * ov[i].x; oy += sc * ov[i].y;
+        }
+        mm = mn;
+      }
+      const int r = row0 + qi / group, hq = kvh * group + qi % group;
+      if (a.n_splits == 1) {                                     // the only split: this is the attention output
+        *reinterpret_cast<__nv_bfloat162 *>(a.att + ((size_t)r * a.nq + hq) * HD + dd) = __floats2bfloat162_rn(ox / l, oy / l);
+      } else {
+        float *dst = a.attn_partials + (((size_t)r * a.nq + hq) * a.n_splits + split) * (HD + 2);
+        *reinterpret_cast<float2 *>(dst + dd) = make_float2(ox, oy);
+        if (dd == 0) { dst[HD] = mm; dst[HD + 1] = l; }
+      }
     }
+    lap(4);
   }
 }
 
@@ -799,6 +824,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   int *row_pos_sh = reinterpret_cast<int *>(ctl + 160);                 // [128] position of each packed row
   int *row_pg_sh = reinterpret_cast<int *>(ctl + 288);                  // [128] KV page holding that position
   FwdLayerDev *layers_sh = reinterpret_cast<FwdLayerDev *>(ctl + 416);  // [<= kMaxLayersSh] pointer table
+  long long *dbg_cy = reinterpret_cast<long long *>(reinterpret_cast<uint8_t *>(bars) + kCtrlBytes - 128);   // debug cycle counters [16]
   // cos / sin of the launch's rows (the tables are touched once per layer, so the weight stream would
   // evict them from L2 between uses): [kRopeCacheRows][hd / 2] each, after the attention / staging area
   float *rope_cos_sh = reinterpret_cast<float *>(scratch + kScratchBytes - 2 * kRopeCacheRows * (HD / 2) * 4);
@@ -819,6 +845,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); mbar_init(ready_bar(b), 1); }
     *abort_flag = 0;
     *last_flag = 0;
+    for (int i = 0; i < 16; ++i) dbg_cy[i] = 0;
     pcache->tag_item = -1;
     pcache->tag_tile = -1;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -990,8 +1017,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         switch (sstep) {
           case 0: kind = K_EPI; gp = p; break;
           case 1: kind = K_FIN; gp = p; break;
-          case 2: kind = K_ATTN_A; break;
-          case 3: kind = K_ATTN_B; ready = p + 1; break;
+          case 2: kind = K_ATTN_A; if (a.n_splits == 1) ready = p + 1; break;       // a single key split needs no merge phase
+          case 3:
+            if (a.n_splits == 1) { kind = K_NONE; barrier = false; }
+            else { kind = K_ATTN_B; ready = p + 1; }
+            break;
           case 4: kind = K_EPI; gp = p + 1; break;
           case 5: kind = K_NORM; gp = p + 1; ready = p + 2; break;
           case 6: kind = K_EPI; gp = p + 2; break;
@@ -1006,7 +1036,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       switch (kind) {
         case K_EPI: if (is_epi) gemm_epilogue<NPAD>(a, w, gp); break;
         case K_FIN: gemm_finish<NPAD>(a, w, gp); break;
-        case K_ATTN_A: attn_tiles_phase<HD>(a, layers_sh[l], scratch, pcache, wt); break;
+        case K_ATTN_A: attn_tiles_phase<HD>(a, layers_sh[l], scratch, pcache, wt, dbg_cy); break;
         case K_ATTN_B: attn_merge_phase<HD>(a, row_pos_sh, wt); break;
         case K_NORM: {
           const bool first = (t == 0);
@@ -1024,6 +1054,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       if (barrier) alive = grid_barrier(a, epoch, abort_flag, wt, ready >= 0 ? ready_bar(ready & 1) : 0u);
     }
   }
+  if (a.prof && blockIdx.x == 0 && threadIdx.x == 128) for (int i = 0; i < 16; ++i) a.prof[940 + i] = (unsigned long long)dbg_cy[i];
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
