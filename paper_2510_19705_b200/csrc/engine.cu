@@ -395,7 +395,8 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     for (int b = 0; b < 4; ++b) a.amap[b] = c->amaps[b][pi];
     // debugging aid: HSD_PROFILE=<file> dumps the barrier timeline of the latest top-level pass
     const char *prof_path = getenv("HSD_PROFILE");
-    const bool prof = prof_path && level == c->n_levels - 1 && n_logit > 0;
+    const char *prof_rows = getenv("HSD_PROFILE_MIN_ROWS");       // e.g. 100: the prompt's chunks instead of decode passes
+    const bool prof = prof_path && level == c->n_levels - 1 && (prof_rows ? R >= atoi(prof_rows) : n_logit > 0);
     a.prof = prof ? c->dev<unsigned long long>(L.prof) : nullptr;
     if (prof) HSD_CUDA_OK(cudaMemsetAsync(a.prof, 0, (size_t)c->sm_count * kFwdProfEvents * 8, s));
     HSD_CUDA_OK(cudaMemsetAsync(a.grid_counter, 0, 4, s));

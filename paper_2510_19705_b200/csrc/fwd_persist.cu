@@ -741,64 +741,66 @@ __device__ __forceinline__ void gemm_epilogue(const FwdArgs &a, WorkerCtx &w, in
     }
   }
 
-// Finish phase of GEMM p (QKV, gate/up, output head): tiles round-robin over the CTAs, two at a time
-// (one per 128-thread group); the pieces of a tile are added in piece order and the result goes
-// through the projection's own epilogue.  All loads of a chunk are issued before the first use.
+// Finish phase of GEMM p (QKV, gate/up, output head): units of (tile, block of up to 32 token rows)
+// round-robin over the CTAs, two at a time (one per 128-thread group); the pieces of a tile (at most
+// four) are added in piece order and the result goes through the projection's own epilogue.  The
+// loads of the next four rows (pieces, rope values) are in flight while the current four are stored.
 template <int NPAD>
 __device__ __forceinline__ void gemm_finish(const FwdArgs &a, WorkerCtx &w, int p) {
   constexpr int RG = 4;                          // token rows per load batch (decode passes have few rows)
-  constexpr int PBF = 4;                         // pieces per load batch
+  constexpr int PBF = 4;                         // pieces per tile at most (regular: <= 4 parts; dealt units: <= 3)
+  constexpr int RB = 32;                         // token rows per unit
   const Gemm g = make_gemm(a, p);
   const SplitGeom geo = split_geom(g, w.G);
   const int layer = p >> 2;
-  const int gidx = w.wt >> 7, gm = w.wt & 127;   // two groups of 128 threads, one tile each at a time
+  const int gidx = w.wt >> 7, gm = w.wt & 127;   // two groups of 128 threads, one unit each at a time
   float *gstage = w.staging + gidx * (kTcBlockM * (RG + 1));
+  const int n_rb = (g.rows + RB - 1) / RB, n_units = g.n_tiles * n_rb;
+  const bool rope_cached = a.R <= kRopeCacheRows;
 #pragma unroll 1
-  for (int tile = w.c + gidx * w.G; tile < g.n_tiles; tile += 2 * w.G) {
-    if (g.mode == MODE_QKV) prof_mark(a, w.wt, 0);
+  for (int u = w.c + gidx * w.G; u < n_units; u += 2 * w.G) {
+    const int tile = u / n_rb, r_lo = (u - tile * n_rb) * RB, r_hi = min(g.rows, r_lo + RB);
     const Tile ti = tile_of(g, tile);
     int fo, n_pieces;
     tile_pieces(g, geo, tile, fo, n_pieces);
     const float *base = a.pieces + (size_t)tile * geo.pieces_max * NPAD * kTcBlockM + gm;
     const int half = a.hd >> 1, dh = ((ti.row0 + gm) % a.hd) % half;
     const bool rope = (g.mode == MODE_QKV && ti.seg < 2);
-#pragma unroll 1
-    for (int c0 = 0; c0 < g.rows; c0 += RG) {
-      float v[RG], cs[RG], sn[RG];
+    float tn[PBF][RG], csn[RG], snn[RG];
+    auto fetch = [&](int c0) {                   // pieces and rope values of rows c0 .. c0 + RG - 1
 #pragma unroll
-      for (int i = 0; i < RG; ++i) { v[i] = 0.f; cs[i] = 1.f; sn[i] = 0.f; }
-      if (rope) {
+      for (int pp = 0; pp < PBF; ++pp)
 #pragma unroll
         for (int i = 0; i < RG; ++i)
-          if (c0 + i < g.rows) {
-            if (a.R <= kRopeCacheRows) {
-              cs[i] = w.rope_cos_sh[(c0 + i) * half + dh];
-              sn[i] = w.rope_sin_sh[(c0 + i) * half + dh];
-            } else {
-              cs[i] = __ldg(a.cos_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
-              sn[i] = __ldg(a.sin_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
-            }
+          tn[pp][i] = (pp < n_pieces && c0 + i < r_hi) ? __ldcg(base + ((size_t)pp * NPAD + c0 + i) * kTcBlockM) : 0.f;
+#pragma unroll
+      for (int i = 0; i < RG; ++i) {
+        csn[i] = 1.f; snn[i] = 0.f;
+        if (rope && c0 + i < r_hi) {
+          if (rope_cached) {
+            csn[i] = w.rope_cos_sh[(c0 + i) * half + dh];
+            snn[i] = w.rope_sin_sh[(c0 + i) * half + dh];
+          } else {
+            csn[i] = __ldg(a.cos_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
+            snn[i] = __ldg(a.sin_tab + (size_t)w.row_pos_sh[c0 + i] * half + dh);
           }
+        }
       }
+    };
+    fetch(r_lo);
 #pragma unroll 1
-      for (int p0 = 0; p0 < n_pieces; p0 += PBF) {
-        float t[PBF][RG];
+    for (int c0 = r_lo; c0 < r_hi; c0 += RG) {
+      float v[RG], cs[RG], sn[RG];
 #pragma unroll
-        for (int pp = 0; pp < PBF; ++pp)
+      for (int i = 0; i < RG; ++i) {
+        v[i] = 0.f;
 #pragma unroll
-          for (int i = 0; i < RG; ++i)
-            t[pp][i] = (p0 + pp < n_pieces && c0 + i < g.rows)
-                           ? __ldcg(base + ((size_t)(p0 + pp) * NPAD + c0 + i) * kTcBlockM)
-                           : 0.f;
-#pragma unroll
-        for (int pp = 0; pp < PBF; ++pp)
-#pragma unroll
-          for (int i = 0; i < RG; ++i) v[i] += t[pp][i];
+        for (int pp = 0; pp < PBF; ++pp) v[i] += tn[pp][i];
+        cs[i] = csn[i]; sn[i] = snn[i];
       }
-      if (g.mode == MODE_QKV) prof_mark(a, w.wt, 1);
+      if (c0 + RG < r_hi) fetch(c0 + RG);
       final_store<RG>(a, g, ti, w.layers_sh[layer < a.n_run ? layer : 0], gm, gm, c0, v, gstage, w.row_pos_sh,
                       w.row_pg_sh, cs, sn, 1 + 2 * gidx);
-      if (g.mode == MODE_QKV) prof_mark(a, w.wt, 2);
     }
   }
 }
