@@ -178,21 +178,23 @@ __device__ __forceinline__ void prof_mark(const FwdArgs &a, int wt, int k) {
 // If ready_bar != 0 the spinning thread then releases the activation producer for the next GEMM.
 __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, volatile int *abort_flag, int wt,
                                              uint32_t ready_bar) {
-  prof_mark(a, wt, 10);
-  __threadfence();
-  prof_mark(a, wt, 11);
+  // The CTA's writes of this phase are ordered before the arrival by the CTA barrier plus ONE release at gpu
+  // scope by the arriving thread (cumulative over what it has observed through the barrier), instead of a
+  // fence in every thread.
   worker_sync();
   ++epoch;
   if (*abort_flag) return false;
   if (wt == 0) {
     const unsigned target = epoch * gridDim.x;
-    atomicAdd(a.grid_counter, 1u);
-    unsigned long long t0 = globaltimer_ns();
-    if (a.prof && 2 * epoch + 1 < (unsigned)kFwdProfEvents) a.prof[(size_t)blockIdx.x * kFwdProfEvents + 2 * epoch] = t0;
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.grid_counter) : "memory");
+    if (a.prof && 2 * epoch + 1 < (unsigned)kFwdProfEvents) a.prof[(size_t)blockIdx.x * kFwdProfEvents + 2 * epoch] = globaltimer_ns();
     bool ok = true;
+    unsigned long long t0 = 0;                       // the clock is read only once the wait has lasted a while
     for (uint32_t it = 0; (int)(ld_acquire_u32(a.grid_counter) - target) < 0; ++it) {
       if ((it & 31u) == 31u) {
-        if (*abort_flag || *reinterpret_cast<volatile int *>(a.status) != 0 || globaltimer_ns() - t0 > kWaitLimitNs) {
+        const unsigned long long now = globaltimer_ns();
+        if (t0 == 0) t0 = now;
+        if (*abort_flag || *reinterpret_cast<volatile int *>(a.status) != 0 || now - t0 > kWaitLimitNs) {
           ok = false;
           break;
         }
@@ -204,7 +206,7 @@ __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, 
     } else {
       if (a.prof && 2 * epoch + 1 < (unsigned)kFwdProfEvents)
         a.prof[(size_t)blockIdx.x * kFwdProfEvents + 2 * epoch + 1] = globaltimer_ns();
-      __threadfence();
+      // the acquire load that left the spin orders everything after it; the CTA barrier below hands that on
       if (ready_bar) {
         asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> visible to TMA reads
         mbar_arrive(ready_bar);
