@@ -352,7 +352,8 @@ __device__ __forceinline__ void ldmatrix_x2_trans(unsigned &r0, unsigned &r1, co
 // one 16-row m-tile each.  At the end the warps' states are merged through shared memory and the
 // split's partial (o, m, l) goes to global memory.
 template <int HD>
-__device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt, long long *dbg) {
+__device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt, long long *dbg,
+                                                 const int *first_item) {
   constexpr int CPR = HD / 8;                      // 16-byte chunks per row
   // Rows of Q, K, V in shared memory: HD >= 64: unpadded, the 16-byte chunk index XORed with the row's low
   // three bits; HD = 32: padded by 16 bytes.  Either way the fragment loads (eight rows, same chunk) and
@@ -379,7 +380,8 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
     long long cyc = clock64();
     auto lap = [&](int k) { if (a.prof && wt == 0 && blockIdx.x == 0) { const long long n_ = clock64(); dbg[k] += n_ - cyc; cyc = n_; } };
     const int split = wi % a.n_splits, kvh = (wi / a.n_splits) % a.nkv, ai = wi / (a.n_splits * a.nkv);
-    const int4 it = a.attn_items[ai];
+    const int4 it = wi == (int)blockIdx.x ? make_int4(first_item[0], first_item[1], first_item[2], first_item[3])
+                                          : a.attn_items[ai];   // the CTA's first item was fetched at kernel start
     const int row0 = it.x, nrows = it.y, seq = it.z, pos0 = it.w;
     const int kv_len = pos0 + nrows;
     const int key_lo = split * a.keys_per_split, key_hi = min(kv_len, key_lo + a.keys_per_split);
@@ -713,16 +715,16 @@ __device__ __forceinline__ void gemm_epilogue(const FwdArgs &a, WorkerCtx &w, in
     Seg sg;
     for (; seg_next(g, it, sg); ++w.seg_idx) {
       const int ab = w.seg_idx & 1;
+      // this CTA's piece of the tile (the next phase sums the pieces): worked out while the MMAs run
+      int fo, np_tile;
+      tile_pieces(g, geo, sg.tile, fo, np_tile);
+      const int piece = w.c - fo;
+      float *mine = a.pieces + ((size_t)sg.tile * geo.pieces_max + piece) * NPAD * kTcBlockM;
       if (w.wt == 0) w.wait_ok[w.seg_idx & 1] = mbar_wait((w.accf_bar0 + 8u * ab), (uint32_t)((w.seg_idx >> 1) & 1), w.abort_flag) ? 1 : 0;
       epi_sync();
       if (!w.wait_ok[w.seg_idx & 1]) return;
       tc_fence_after();
       const uint32_t tbase = w.tmem_base + ((uint32_t)(w.q * 32) << 16) + (uint32_t)(ab * NPAD);
-      // this CTA's piece of the tile; the next phase sums the pieces
-      int fo, np_tile;
-      tile_pieces(g, geo, sg.tile, fo, np_tile);
-      const int piece = w.c - fo;
-      float *mine = a.pieces + ((size_t)sg.tile * geo.pieces_max + piece) * NPAD * kTcBlockM;
 #pragma unroll 1
       for (int c0 = 0; c0 < NPAD; c0 += CH) {
         float v[CH];
@@ -821,7 +823,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   uint32_t *ctl = reinterpret_cast<uint32_t *>(bars + 2 * STAGES + 6);
   uint32_t *tmem_slot = ctl;
   volatile int *abort_flag = reinterpret_cast<volatile int *>(ctl + 1);
-  volatile int *last_flag = reinterpret_cast<volatile int *>(ctl + 2);
+  int *first_item_sh = reinterpret_cast<int *>(ctl + 148);               // [4] this CTA's first attention item
   volatile int *wait_ok = reinterpret_cast<volatile int *>(ctl + 4);   // [2]
   float *red = reinterpret_cast<float *>(ctl + 8);                      // [8]
   PageCache *pcache = reinterpret_cast<PageCache *>(ctl + 16);          // 130 words
@@ -848,7 +850,6 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); mbar_init(ready_bar(b), 1); }
     *abort_flag = 0;
-    *last_flag = 0;
     for (int i = 0; i < 16; ++i) dbg_cy[i] = 0;
     pcache->tag_item = -1;
     pcache->tag_tile = -1;
@@ -919,10 +920,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       bool ok = true;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
-        // the operand of phase p is complete once the workers have passed the barrier before it
-        if (!mbar_wait(ready_bar(p & 1), (uint32_t)((p >> 1) & 1), abort_flag)) { ok = false; break; }
         SegIter it = seg_begin(g, G, c);
         Seg sg;
+        // the operand of phase p is complete once the workers have passed the barrier before it
+        if (!mbar_wait(ready_bar(p & 1), (uint32_t)((p >> 1) & 1), abort_flag)) { ok = false; break; }
         while (ok && seg_next(g, it, sg)) {
           for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
             if (s % WGS == 0 && !mbar_wait(empty_bar(s / WGS), par, abort_flag)) { ok = false; break; }
@@ -999,6 +1000,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       row_pos_sh[r] = pos;
       row_pg_sh[r] = a.page_table[(size_t)a.row_seq[r] * a.pages_per_seq + pos / a.page];
     }
+    // descriptor of this CTA's first attention work item, kept in shared memory (the same in every layer; a
+    // dependent global load at the start of every attention phase otherwise)
+    if (wt == 0) {
+      const int n_work = a.n_attn * a.nkv * a.n_splits;
+      int4 fi = make_int4(0, 0, 0, 0);
+      if ((int)blockIdx.x < n_work) fi = a.attn_items[blockIdx.x / (a.n_splits * a.nkv)];
+      first_item_sh[0] = fi.x; first_item_sh[1] = fi.y; first_item_sh[2] = fi.z; first_item_sh[3] = fi.w;
+    }
     // One step loop, one call site per phase body: the whole per-layer program has to stay resident in
     // the instruction cache (every phase runs once per layer, so code that does not fit is fetched
     // cold through the saturated memory system every single time).
@@ -1040,7 +1049,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       switch (kind) {
         case K_EPI: if (is_epi) gemm_epilogue<NPAD>(a, w, gp); break;
         case K_FIN: gemm_finish<NPAD>(a, w, gp); break;
-        case K_ATTN_A: attn_tiles_phase<HD>(a, layers_sh[l], scratch, pcache, wt, dbg_cy); break;
+        case K_ATTN_A: attn_tiles_phase<HD>(a, layers_sh[l], scratch, pcache, wt, dbg_cy, first_item_sh); break;
         case K_ATTN_B: attn_merge_phase<HD>(a, row_pos_sh, wt); break;
         case K_NORM: {
           const bool first = (t == 0);
