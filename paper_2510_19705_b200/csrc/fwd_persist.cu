@@ -181,6 +181,9 @@ __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, 
   // The CTA's writes of this phase are ordered before the arrival by the CTA barrier plus ONE release at gpu
   // scope by the arriving thread (cumulative over what it has observed through the barrier), instead of a
   // fence in every thread.
+  // The activations this phase wrote with plain stores are read by the next GEMM's TMA loads (async proxy):
+  // every writer orders its generic-proxy writes before async-proxy accesses here, ahead of the release.
+  if (ready_bar) asm volatile("fence.proxy.async.global;" ::: "memory");
   worker_sync();
   ++epoch;
   if (*abort_flag) return false;
@@ -208,7 +211,6 @@ __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, 
         a.prof[(size_t)blockIdx.x * kFwdProfEvents + 2 * epoch + 1] = globaltimer_ns();
       // the acquire load that left the spin orders everything after it; the CTA barrier below hands that on
       if (ready_bar) {
-        asm volatile("fence.proxy.async;" ::: "memory");   // generic-proxy writes -> visible to TMA reads
         mbar_arrive(ready_bar);
       }
     }
