@@ -97,11 +97,10 @@ __device__ __forceinline__ Tile tile_of(const Gemm &g, int tile) {
 }
 // Unit arithmetic in 32 bits (the launcher checks n_tiles * KB * grid < 2^31).
 __device__ __forceinline__ int cta_begin(int U, int G, int c) { return (int)(((unsigned)U * (unsigned)c) / (unsigned)G); }
+// CTA c owns units [floor(U c / G), floor(U (c + 1) / G)): the owner of unit u is the largest c with
+// floor(U c / G) <= u, i.e. c < (u + 1) G / U, i.e. c = floor(((u + 1) G - 1) / U).
 __device__ __forceinline__ int unit_owner(int U, int G, int u) {
-  int c = (int)(((unsigned)u * (unsigned)G) / (unsigned)U);
-  while (c + 1 < G && cta_begin(U, G, c + 1) <= u) ++c;
-  while (c > 0 && cta_begin(U, G, c) > u) --c;
-  return c;
+  return (int)((((unsigned)u + 1u) * (unsigned)G - 1u) / (unsigned)U);
 }
 // Work of one CTA in one GEMM, a segment (tile, k-block range) at a time.  One SM can pull only its
 // share of HBM bandwidth, so every GEMM is split evenly over all CTAs in (tile, k-block) units;
