@@ -107,7 +107,7 @@ __device__ __forceinline__ int unit_owner(int U, int G, int u) {
 // each segment's partial sums go to a piece buffer and the next phase adds the pieces of a tile in
 // fixed piece order (bit-reproducible; no CTA waits for another inside a GEMM).
 struct Seg { int tile, kb0, kb1; };
-struct SegIter { int cur, end; };
+struct SegIter { int tile, kb, left; };        // next k-block (tile, kb) and the k-blocks still to hand out
 // regular: every tile is cut into `parts` equal k-ranges (GEMMs with few tiles: at most 4 pieces per
 // tile, so the consumer can fetch all of them in one batch); otherwise the (tile, k-block) units are
 // dealt out evenly (tiles >= CTAs / 2: a tile then spans at most 3 CTAs).
@@ -127,27 +127,31 @@ __device__ __forceinline__ SplitGeom split_geom(const Gemm &g, int G) {
   }
   return sg;
 }
+// The divisions happen once, here; seg_next only counts (the pipeline roles call it on their critical path).
 __device__ __forceinline__ SegIter seg_begin(const Gemm &g, int G, int c) {
   SegIter it;
   const SplitGeom sg = split_geom(g, G);
-  it.cur = it.end = 0;
+  it.tile = 0; it.kb = 0; it.left = 0;
   if (c < sg.Gp) {
     if (sg.parts) {
-      const int tile = c / sg.parts, part = c % sg.parts;
-      it.cur = tile * g.KB + cta_begin(g.KB, sg.parts, part);
-      it.end = tile * g.KB + cta_begin(g.KB, sg.parts, part + 1);
+      const int tile = c / sg.parts, part = c - tile * sg.parts;
+      it.tile = tile;
+      it.kb = cta_begin(g.KB, sg.parts, part);
+      it.left = cta_begin(g.KB, sg.parts, part + 1) - it.kb;
     } else {
-      it.cur = cta_begin(sg.U, sg.Gp, c);
-      it.end = cta_begin(sg.U, sg.Gp, c + 1);
+      const int cur = cta_begin(sg.U, sg.Gp, c);
+      it.left = cta_begin(sg.U, sg.Gp, c + 1) - cur;
+      it.tile = cur / g.KB;
+      it.kb = cur - it.tile * g.KB;
     }
   }
   return it;
 }
 __device__ __forceinline__ bool seg_next(const Gemm &g, SegIter &it, Seg &s) {
-  if (it.cur >= it.end) return false;
-  s.tile = it.cur / g.KB; s.kb0 = it.cur % g.KB;
-  s.kb1 = min(g.KB, s.kb0 + (it.end - it.cur));
-  it.cur += s.kb1 - s.kb0;
+  if (it.left <= 0) return false;
+  const int n = min(g.KB - it.kb, it.left);
+  s.tile = it.tile; s.kb0 = it.kb; s.kb1 = it.kb + n;
+  it.left -= n; it.kb = 0; ++it.tile;
   return true;
 }
 // Pieces of a tile: they belong to consecutive CTAs first_owner .. first_owner + n - 1.
@@ -923,9 +927,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         const Gemm g = make_gemm(a, p);
         SegIter it = seg_begin(g, G, c);
         Seg sg;
+        bool have = seg_next(g, it, sg);
         // the operand of phase p is complete once the workers have passed the barrier before it
         if (!mbar_wait(ready_bar(p & 1), (uint32_t)((p >> 1) & 1), abort_flag)) { ok = false; break; }
-        while (ok && seg_next(g, it, sg)) {
+        while (ok && have) {
           for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
             if (s % WGS == 0 && !mbar_wait(empty_bar(s / WGS), par, abort_flag)) { ok = false; break; }
             const uint32_t dst = smem_u32(ring) + (uint32_t)(s * Cfg::kStageBytes) + kWBytes;
@@ -933,6 +938,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
             tma_load_2d(dst, g.amap, kb * kTcBlockK, 0, full_bar(s));
             if (++s == STAGES) { s = 0; par ^= 1u; }
           }
+          have = seg_next(g, it, sg);
         }
       }
       if (!ok) atomicExch(a.status, 1);
