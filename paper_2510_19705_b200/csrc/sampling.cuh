@@ -33,8 +33,13 @@ __device__ __forceinline__ u32 uniform24(u64 seed, u32 j, u32 serial, u32 level,
 __device__ __forceinline__ u32 exp_weight(float l, float m) {
   float x = __fsub_rn(l, m);
   x = fmaxf(x, -32.0f);
-  float t = __fmul_rn(x, __uint_as_float(0x3FB8AA3Bu));     // * log2(e)
-  float j = rintf(t);                                      // half to even
+  float t = __fmul_rn(x, __uint_as_float(0x3FB8AA3Bu));     // * log2(e), in [-46.2, 0]
+  // rint(t), half to even, without the quarter-rate conversion instructions: at 1.5 * 2^23 the fp32 spacing is
+  // 1, so the add rounds t to the nearest integer (ties to even), the subtraction is exact, and the integer
+  // itself sits in the low mantissa bits of the sum
+  const float magic = __uint_as_float(0x4B400000u);        // 12582912
+  float tm = __fadd_rn(t, magic);
+  float j = __fsub_rn(tm, magic);
   float f = __fsub_rn(t, j);                               // exact, in [-1/2, 1/2]
   float p = __uint_as_float(0x3AADDD0Au);
   p = __fadd_rn(__fmul_rn(p, f), __uint_as_float(0x3C1E7544u));
@@ -42,7 +47,7 @@ __device__ __forceinline__ u32 exp_weight(float l, float m) {
   p = __fadd_rn(__fmul_rn(p, f), __uint_as_float(0x3E75FCDEu));
   p = __fadd_rn(__fmul_rn(p, f), __uint_as_float(0x3F317215u));
   p = __fadd_rn(__fmul_rn(p, f), 1.0f);
-  int e = (int)j + 32;                                     // in [-14, 32]
+  int e = (__float_as_int(tm) - 0x4B400000) + 32;          // (int)j + 32, in [-14, 32]
   float w = __fmul_rn(p, __int_as_float((e + 127) << 23)); // exact power-of-two scaling
   return __float2uint_rz(w);                               // floor; saturates at 2^32 - 1
 }
@@ -56,8 +61,10 @@ __device__ __forceinline__ void exp_weight2(float l0, float l1, float m, u32 &e0
   x.y = fmaxf(x.y, -32.0f);
   const float log2e = __uint_as_float(0x3FB8AA3Bu);
   const float2 t = __fmul2_rn(x, make_float2(log2e, log2e));
-  const float j0 = rintf(t.x), j1 = rintf(t.y);
-  const float2 f = __fadd2_rn(t, make_float2(-j0, -j1));
+  const float magic = __uint_as_float(0x4B400000u);        // see exp_weight
+  const float2 tm = __fadd2_rn(t, make_float2(magic, magic));
+  const float2 jj = __fadd2_rn(tm, make_float2(-magic, -magic));
+  const float2 f = __fadd2_rn(t, make_float2(-jj.x, -jj.y));
   float c = __uint_as_float(0x3AADDD0Au);
   float2 p = make_float2(c, c);
   c = __uint_as_float(0x3C1E7544u); p = __fadd2_rn(__fmul2_rn(p, f), make_float2(c, c));
@@ -65,7 +72,8 @@ __device__ __forceinline__ void exp_weight2(float l0, float l1, float m, u32 &e0
   c = __uint_as_float(0x3E75FCDEu); p = __fadd2_rn(__fmul2_rn(p, f), make_float2(c, c));
   c = __uint_as_float(0x3F317215u); p = __fadd2_rn(__fmul2_rn(p, f), make_float2(c, c));
   p = __fadd2_rn(__fmul2_rn(p, f), make_float2(1.0f, 1.0f));
-  const float2 sc = make_float2(__int_as_float(((int)j0 + 32 + 127) << 23), __int_as_float(((int)j1 + 32 + 127) << 23));
+  const float2 sc = make_float2(__int_as_float((__float_as_int(tm.x) - 0x4B400000 + 32 + 127) << 23),
+                                __int_as_float((__float_as_int(tm.y) - 0x4B400000 + 32 + 127) << 23));
   const float2 w = __fmul2_rn(p, sc);
   e0 = __float2uint_rz(w.x);
   e1 = __float2uint_rz(w.y);
