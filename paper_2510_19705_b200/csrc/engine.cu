@@ -182,6 +182,7 @@ struct hsd_ctx {
   int sm_count;
   std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + 1]: wq wk wv wo wg wu wd per layer, then lm_head
   CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
+  CUtensorMap amaps_rows[4][16];              // the same buffers with a box of exactly 1..16 rows (persistent forward, few rows)
   int *status_host;
 
   template <typename U> U *dev(size_t off) const { return reinterpret_cast<U *>(ws + off); }
@@ -392,7 +393,11 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     a.grid_counter = c->dev<unsigned>(L.grid_counter); a.status = (int *)(c->ws + L.tc_scratch);
     const int np = tc_npad(std::max(R, n_logit));
     const int pi = np == 16 ? 0 : np == 32 ? 1 : np == 64 ? 2 : 3;
-    for (int b = 0; b < 4; ++b) a.amap[b] = c->amaps[b][pi];
+    // few rows: fetch exactly the rows that exist (the MMA still reads `np` rows of the stage; the rest is stale
+    // shared memory that only feeds accumulator columns nobody reads): 148 CTAs x K / 64 boxes per GEMM add up
+    const int box_rows = std::max(R, n_logit) <= 16 ? std::max(R, n_logit) : np;
+    a.a_box_rows = box_rows;
+    for (int b = 0; b < 4; ++b) a.amap[b] = box_rows <= 16 ? c->amaps_rows[b][box_rows - 1] : c->amaps[b][pi];
     // debugging aid: HSD_PROFILE=<file> dumps the barrier timeline of the latest top-level pass
     const char *prof_path = getenv("HSD_PROFILE");
     const char *prof_rows = getenv("HSD_PROFILE_MIN_ROWS");       // e.g. 100: the prompt's chunks instead of decode passes
@@ -733,6 +738,8 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
     const int npads[4] = {16, 32, 64, 128};
     for (int b = 0; b < 4 && !st; ++b)
       for (int p = 0; p < 4 && !st; ++p) st = tc_make_map(&c->amaps[b][p], c->ws + abuf_off[b], arows[b], acols[b], npads[p]);
+    for (int b = 0; b < 4 && !st; ++b)
+      for (int r = 1; r <= 16 && !st; ++r) st = tc_make_map(&c->amaps_rows[b][r - 1], c->ws + abuf_off[b], arows[b], acols[b], r);
     if (!st && cudaMemset(c->ws + lay.tc_scratch, 0, kTcCtrlBytes) != cudaSuccess) st = HSD_E_CUDA;
     // tables of the persistent forward: tensor maps and per-layer pointers in device memory
     if (!st) {

@@ -923,6 +923,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       int s = 0;
       uint32_t par = 1;
       bool ok = true;
+      const uint32_t a_bytes = (uint32_t)a.a_box_rows * kTcBlockK * 2;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
         SegIter it = seg_begin(g, G, c);
@@ -934,7 +935,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
           for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
             if (s % WGS == 0 && !mbar_wait(empty_bar(s / WGS), par, abort_flag)) { ok = false; break; }
             const uint32_t dst = smem_u32(ring) + (uint32_t)(s * Cfg::kStageBytes) + kWBytes;
-            mbar_expect_tx(full_bar(s), NPAD * kTcBlockK * 2);
+            mbar_expect_tx(full_bar(s), a_bytes);
             tma_load_2d(dst, g.amap, kb * kTcBlockK, 0, full_bar(s));
             if (++s == STAGES) { s = 0; par ^= 1u; }
           }
