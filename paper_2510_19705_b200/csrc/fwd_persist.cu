@@ -750,7 +750,7 @@ __device__ __forceinline__ void gemm_epilogue(const FwdArgs &a, WorkerCtx &w, in
     }
   }
 
-// Finish phase of GEMM p (QKV, gate/up, output head): units of (tile, block of up to 32 token rows)
+// Finish phase of GEMM p (QKV, gate/up, output head): units of (tile, block of up to 8 token rows)
 // round-robin over the CTAs, two at a time (one per 128-thread group); the pieces of a tile (at most
 // four) are added in piece order and the result goes through the projection's own epilogue.  The
 // loads of the next four rows (pieces, rope values) are in flight while the current four are stored.
@@ -758,7 +758,7 @@ template <int NPAD>
 __device__ __forceinline__ void gemm_finish(const FwdArgs &a, WorkerCtx &w, int p) {
   constexpr int RG = 4;                          // token rows per load batch (decode passes have few rows)
   constexpr int PBF = 4;                         // pieces per tile at most (regular: <= 4 parts; dealt units: <= 3)
-  constexpr int RB = 32;                         // token rows per unit
+  constexpr int RB = 8;                          // token rows per unit (two load batches; more units than 2 x CTAs at 24+ rows)
   const Gemm g = make_gemm(a, p);
   const SplitGeom geo = split_geom(g, w.G);
   const int layer = p >> 2;
