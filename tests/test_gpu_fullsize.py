@@ -154,23 +154,25 @@ def test_model_shapes_decisions_and_sampled_logits(lib, tmp_path, name, n_new, o
     assert len(seen) == oracle_calls
 
 
-def test_bf16_batch_decisions_and_logits(lib, tmp_path):
-    # two sequences in one bf16 batch: every decision follows the oracle on the logged logits, and each
-    # sequence's first verification logits match the oracle's forward of that sequence
+@pytest.mark.parametrize("B", [2, 8])
+def test_bf16_batch_decisions_and_logits(lib, tmp_path, B):
+    # several sequences in one bf16 batch (8: passes of 17-32 rows, the 32-row padding of the GEMMs): every
+    # decision follows the oracle on the logged logits, and each sequence's first verification logits match the
+    # oracle's forward of that sequence
     wl = inputs.WORKLOADS["mini3"]
     cfg = wl["model"]
     w_cpu = inputs.make_weights(cfg, wl["weight_seed"])
     w = {k: (v.cuda() if k != "layers" else [{n: t.cuda() for n, t in l.items()} for l in v]) for k, v in w_cpu.items()}
-    prompts = inputs.make_prompts(cfg["vocab"], 2, wl["prompt"], 11)
-    eng = lib.Hsd(cfg, w, wl["exits"], wl["T"], max_batch=2, max_seq=128, page_size=16)
+    prompts = inputs.make_prompts(cfg["vocab"], B, wl["prompt"], 11)
+    eng = lib.Hsd(cfg, w, wl["exits"], wl["T"], max_batch=B, max_seq=128, page_size=16)
     path = str(tmp_path / "trace.bin")
     eng.set_trace(path, logit_calls=10 ** 6)
     toks, stats, _ = eng.generate(prompts.cuda(), 32, 4)
     eng.set_trace(None)
     recs = lib.read_trace(path)
-    assert _replay_decisions(recs, 4, n_seq=2) == sum(s["calls"] for s in stats[1:])
+    assert _replay_decisions(recs, 4, n_seq=B) == sum(s["calls"] for s in stats[1:])
     om = Transformer(cfg, inputs.weights_to_numpy(w_cpu), wl["exits"])
-    for b in range(2):
+    for b in range(B):
         prompt = prompts[b].tolist()
         final = _context_of(recs, None, prompt, b)
         assert final[len(prompt):len(prompt) + 32] == toks[b].cpu().tolist()
