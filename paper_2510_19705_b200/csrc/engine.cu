@@ -82,7 +82,8 @@ Layout make_layout(const hsd_model_desc *m, int n_levels, const int32_t *T) {
   L.max_rows = std::max(kPrefillRows, decode_rows);
   L.pages_per_seq = (m->max_seq + page - 1) / page;
   L.n_pages = B * L.pages_per_seq;
-  L.partial_rows = L.max_rows + kAttnRows * kAttnBlocksTarget / nkv + kAttnRows * kMaxSplits;
+  L.partial_rows = std::max(L.max_rows + kAttnRows * kAttnBlocksTarget / nkv + kAttnRows * kMaxSplits,
+                            L.max_rows * 20);   // the persistent forward may cut every row's keys into up to 20 splits
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   L.tokens = take((size_t)B * m->max_seq * 4);
@@ -338,6 +339,12 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
       }
     }
   }
+  // Attention work items are dealt to the CTAs round-robin in this order: the most expensive first (keys x
+  // 16-row query tiles), so that a CTA's items sample the whole cost range.
+  const int qgroup = md.nq / md.nkv;
+  auto item_cost = [&](const int4 &it) { return (long long)(it.w + it.y) * ((it.y * qgroup + 15) / 16); };
+  if (c->use_persist && n_attn > 1)
+    std::stable_sort(attn, attn + n_attn, [&](const int4 &x, const int4 &y) { return item_cost(x) > item_cost(y); });
   HSD_CUDA_OK(cudaMemcpyAsync(devp, host, bytes, cudaMemcpyHostToDevice, c->stream));
   st = upload_page_tables(c);
   if (st) return st;
@@ -358,6 +365,44 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   if (c->use_persist) if (const char *e = getenv("HSD_ATTN_SPLITS_MAX")) max_splits = std::max(1, std::min(20, atoi(e)));
   int n_splits = std::max(1, std::min(max_splits, blocks_target / std::max(1, n_attn * md.nkv)));
   if (c->use_persist && max_kv <= c->attn_single_max) n_splits = 1;   // short contexts: one split, no merge phase
+  if (c->use_persist && max_kv >= 2048) {
+    // Long contexts: the key loop dominates and the items differ in cost, so the split count is chosen by a
+    // small model of the tiles phase: a work unit (item, KV head, split) costs a fixed part plus its keys x
+    // query tiles, units go to the CTAs round-robin in item order (as the kernel deals them), the phase lasts
+    // as long as the most loaded CTA; more than one split adds the merge phase.
+    const int G = c->sm_count;
+    double best = 1e30;
+    int best_s = 1;
+    std::vector<double> diff(G + 1);
+    for (int s_try : {1, 2, 3, 4, 6, 8, 10, 12, 16, 20}) {
+      const int kps = (int)align_up((size_t)(max_kv + s_try - 1) / s_try, 16);
+      if (s_try > 1 && kps < 256) break;
+      std::fill(diff.begin(), diff.end(), 0.0);
+      double everywhere = 0;
+      long long off = 0;
+      for (int i = 0; i < n_attn; ++i) {
+        const int kv = attn[i].w + attn[i].y, mt = (attn[i].y * qgroup + 15) / 16;
+        const double unit = 5.0 + mt * ((std::min(kps, kv) + 127) / 128) * 1.9;
+        // all s_try x nkv slots of the item are dealt out; splits past its last key return at once
+        const long long used = (long long)std::min(s_try, (kv + kps - 1) / kps) * md.nkv, slots = (long long)s_try * md.nkv;
+        everywhere += unit * (double)(used / G);
+        const int rem = (int)(used % G), at = (int)(off % G);
+        if (rem) {
+          diff[at] += unit;
+          if (at + rem <= G) diff[at + rem] -= unit;
+          else { diff[G] -= unit; diff[0] += unit; diff[at + rem - G] -= unit; }
+        }
+        off += slots;
+      }
+      double load = 0, worst = 0;
+      for (int g = 0; g < G; ++g) { load += diff[g]; worst = std::max(worst, load); }
+      // merge phase: a barrier and a load round trip, then one (row, head) per 128 threads
+      const double merge = 6.0 + 1.5 * (((double)R * md.nq + 2 * G - 1) / (2 * G));
+      const double t = everywhere + worst + (s_try > 1 ? merge : 0.0);
+      if (t < best) { best = t; best_s = s_try; }
+    }
+    n_splits = best_s;
+  }
   int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, c->use_persist ? 16 : kAttnKeyTile);
   n_splits = (max_kv + keys_per_split - 1) / keys_per_split;
   if ((size_t)R * n_splits > (size_t)L.partial_rows) return HSD_E_INVALID_ARG;
