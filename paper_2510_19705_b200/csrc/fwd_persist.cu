@@ -342,8 +342,15 @@ __device__ __forceinline__ void mma_bf16_16x8x16(float *c, const unsigned *a, un
                : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
-__device__ __forceinline__ void ldmatrix_x2_trans(unsigned &r0, unsigned &r1, const void *row_ptr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x2.trans.shared.b16 {%0,%1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(smem_u32(row_ptr)));
+// Four 8x8 b16 matrices; lane l gives the address of row l % 8 of matrix l / 8; register i of lane (g, t) holds
+// matrix i's elements [g][2t .. 2t + 1] (.trans: [2t .. 2t + 1][g]).
+__device__ __forceinline__ void ldmatrix_x4(unsigned *r, const void *row_ptr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(row_ptr)));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(unsigned *r, const void *row_ptr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(row_ptr)));
 }
 
 // Phase A: warp-level online softmax.  A work item is (attention item, KV head, key split); its keys
@@ -457,20 +464,19 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
       for (int n = 0; n < 2; ++n)
 #pragma unroll
         for (int e = 0; e < 4; ++e) sacc[n][e] = 0.f;
-      // rows g and g + 8 of a fragment share the low row bits (g), so one swizzled chunk offset serves both
-      const __nv_bfloat16 *qa = shQ + (mt * 16 + g) * RS + 2 * t;
+      // fragments by ldmatrix: Q as the A operand (matrices: rows 0-7 / 8-15 x k 0-7 / 8-15), K as the B operand
+      // of both 8-key n-tiles (keys 0-7 / 8-15 x k 0-7 / 8-15)
+      {
+        const int mi = lane >> 3, r8 = lane & 7;
+        const int qrow_l = (mi & 1) * 8 + r8, krow_l = (mi >> 1) * 8 + r8;
+        const __nv_bfloat16 *qbase = shQ + (mt * 16 + qrow_l) * RS, *kbase = shK + krow_l * RS;
 #pragma unroll
-      for (int ks = 0; ks < KST; ++ks) {
-        const int c0 = swz(g, 2 * ks) * 8, c1 = swz(g, 2 * ks + 1) * 8;
-        unsigned af[4];
-        af[0] = *reinterpret_cast<const unsigned *>(qa + c0);
-        af[1] = *reinterpret_cast<const unsigned *>(qa + 8 * RS + c0);
-        af[2] = *reinterpret_cast<const unsigned *>(qa + c1);
-        af[3] = *reinterpret_cast<const unsigned *>(qa + 8 * RS + c1);
-#pragma unroll
-        for (int n = 0; n < 2; ++n) {
-          const __nv_bfloat16 *kb = shK + (n * 8 + g) * RS + 2 * t;
-          mma_bf16_16x8x16(sacc[n], af, *reinterpret_cast<const unsigned *>(kb + c0), *reinterpret_cast<const unsigned *>(kb + c1));
+        for (int ks = 0; ks < KST; ++ks) {
+          unsigned af[4], bf4[4];
+          ldmatrix_x4(af, qbase + swz(qrow_l, 2 * ks + (mi >> 1)) * 8);
+          ldmatrix_x4(bf4, kbase + swz(krow_l, 2 * ks + (mi & 1)) * 8);
+          mma_bf16_16x8x16(sacc[0], af, bf4[0], bf4[1]);
+          mma_bf16_16x8x16(sacc[1], af, bf4[2], bf4[3]);
         }
       }
       __syncwarp();                                              // every lane is done with the K buffer
@@ -478,6 +484,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
       else asm volatile("cp.async.commit_group;" ::: "memory");  // keep the group count uniform
       // ---- online softmax on the accumulator rows (g and g + 8); P re-packed as the A operand of P V
       unsigned ph[4], pl[4];
+      float corr_h[2];
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         float sv[4];
@@ -504,8 +511,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
         }
         m_run[h] = m_new;
         l_run[h] = l_run[h] * corr + ps;                         // this thread's columns only; summed over t at the end
-#pragma unroll
-        for (int n = 0; n < NT; ++n) { o[n][h * 2] *= corr; o[n][h * 2 + 1] *= corr; }
+        corr_h[h] = corr;
 #pragma unroll
         for (int n = 0; n < 2; ++n) {                            // A fragment: a[h] <- keys 2t.. of n-tile 0, a[2 + h] <- n-tile 1
           const __nv_bfloat162 hi = __floats2bfloat162_rn(pv[n * 2], pv[n * 2 + 1]);
@@ -517,13 +523,23 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
       }
       asm volatile("cp.async.wait_group 1;" ::: "memory");       // V of this sub-tile landed; the next K may be in flight
       __syncwarp();
-      // ---- O += P V
+      // ---- O = O * corr + P V (the rescale is skipped while no row of the warp has a new maximum)
+      if (__any_sync(0xFFFFFFFFu, corr_h[0] != 1.f || corr_h[1] != 1.f)) {
 #pragma unroll
-      for (int n = 0; n < NT; ++n) {
-        unsigned b0, b1;
-        ldmatrix_x2_trans(b0, b1, shV + (lane & 15) * RS + swz(lane & 15, n) * 8);
-        mma_bf16_16x8x16(o[n], ph, b0, b1);
-        mma_bf16_16x8x16(o[n], pl, b0, b1);
+        for (int n = 0; n < NT; ++n) { o[n][0] *= corr_h[0]; o[n][1] *= corr_h[0]; o[n][2] *= corr_h[1]; o[n][3] *= corr_h[1]; }
+      }
+      {
+        const int mi = lane >> 3, key_l = (mi & 1) * 8 + (lane & 7);
+        const __nv_bfloat16 *vbase = shV + key_l * RS;
+#pragma unroll
+        for (int n = 0; n < NT; n += 2) {          // two 8-wide slices of the head dimension per ldmatrix
+          unsigned bv[4];
+          ldmatrix_x4_trans(bv, vbase + swz(key_l, n + (mi >> 1)) * 8);
+          mma_bf16_16x8x16(o[n], ph, bv[0], bv[1]);
+          mma_bf16_16x8x16(o[n], pl, bv[0], bv[1]);
+          mma_bf16_16x8x16(o[n + 1], ph, bv[2], bv[3]);
+          mma_bf16_16x8x16(o[n + 1], pl, bv[2], bv[3]);
+        }
       }
       __syncwarp();                                              // every lane is done with the V buffer
       if (j + 1 < n_mine) issue(vpool, shV, j + 1, true);
