@@ -193,6 +193,25 @@ int hsd_search_T(const double *costs, const double *alphas, int n_levels, int T_
                  double *out_latency);
 
 /* ---------------------------------------------------------------------------------------
+ * Latency-optimal hierarchy (Section 4.2, Corollary 4.1): among the ordered subsets sigma of the models
+ * 0 .. n_models-1 that end in the target (model n_models-1) and the draft lengths T_k in [1, T_max] with
+ * T_k >= T_{k-1}, the pair (sigma, T) with the smallest expected latency per token L(sigma, T).  The
+ * paper's reduction graph (vertices = (model, batch size)) is acyclic once its self-loops are dropped, so
+ * the cheapest path is found by a cost-to-go recursion, O(n_models^2 T_max^2) evaluations of gamma.
+ *   costs host [n_models]: c_i, cost of one forward of model i (any unit);
+ *   alpha host [n_models * n_models], row-major: alpha[i * n_models + j] = acceptance rate of drafter i
+ *     under verifier j; only entries with i < j are read;
+ *   out_sigma host [n_models]: the chosen models in ascending order, the last one is the target;
+ *   out_n_levels host [1]: how many models were chosen (1 = the target alone);
+ *   out_T host [n_models-1]: T_0 .. T_{n_levels-2} for the chosen chain (may be null when n_models = 1);
+ *   out_latency host [1] or null.
+ * Ties keep the first candidate in the order (smaller drafter index, smaller batch).  Host-only.
+ * Errors: INVALID_ARG (null pointers, n_models outside 1..64, T_max outside 1..64, a rate outside [0, 1],
+ * a negative or NaN cost). */
+int hsd_search_hierarchy(const double *costs, const double *alpha, int n_models, int T_max, int32_t *out_sigma,
+                         int32_t *out_n_levels, int32_t *out_T, double *out_latency);
+
+/* ---------------------------------------------------------------------------------------
  * One weight-streaming matrix product of the verifier forward in isolation (the contraction
  * behind every projection of Algorithm 2's multi-row forward pass): out[r, n] = sum_k A[r, k] W[n, k],
  * bf16 inputs, fp32 accumulation on the tensor cores, fp32 output.

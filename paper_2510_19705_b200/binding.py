@@ -161,6 +161,9 @@ def _declare_engine(lib):
     lib.hsd_search_T.restype = i32
     lib.hsd_search_T.argtypes = [c.POINTER(c.c_double), c.POINTER(c.c_double), i32, i32, i32, c.POINTER(c.c_int32),
                                  c.POINTER(c.c_double)]
+    lib.hsd_search_hierarchy.restype = i32
+    lib.hsd_search_hierarchy.argtypes = [c.POINTER(c.c_double), c.POINTER(c.c_double), i32, i32, c.POINTER(c.c_int32),
+                                         c.POINTER(c.c_int32), c.POINTER(c.c_int32), c.POINTER(c.c_double)]
     lib.hsd_kernel_launches.restype = c.c_uint64
     lib.hsd_kernel_launches.argtypes = []
     lib.hsd_gemm_workspace_bytes.restype = sz
@@ -281,6 +284,27 @@ def hsd_search_T(costs, alphas, T_max=15, monotone=True):
                             1 if monotone else 0, out_T, ctypes.byref(out)))
     return tuple(out_T[i] for i in range(n - 1)), out.value
 
+
+
+def hsd_search_hierarchy(costs, alpha, T_max=15):
+    """Latency-optimal (sigma, T) over ordered subsets of the models ending in the target.
+    costs: c_0..c_K; alpha[i][j]: acceptance rate of drafter i under verifier j (i < j).
+    -> (latency, sigma tuple, T tuple)."""
+    lib = library()
+    _declare_engine(lib)
+    n = len(costs)
+    flat = [0.0] * (n * n)
+    for i in range(n):
+        for j in range(i + 1, n):
+            flat[i * n + j] = float(alpha[i][j])
+    sigma = (ctypes.c_int32 * n)()
+    n_lev = ctypes.c_int32()
+    out_T = (ctypes.c_int32 * max(1, n - 1))()
+    out = ctypes.c_double()
+    _check(lib.hsd_search_hierarchy((ctypes.c_double * n)(*costs), (ctypes.c_double * (n * n))(*flat), n, T_max, sigma,
+                                    ctypes.byref(n_lev), out_T, ctypes.byref(out)))
+    k = n_lev.value
+    return out.value, tuple(sigma[i] for i in range(k)), tuple(out_T[i] for i in range(k - 1))
 
 def hsd_kernel_launches():
     lib = library()

@@ -1,5 +1,5 @@
-// Expected latency of a hierarchy (Theorem 3.2) and the search for its parameters T (Section 4),
-// host side.  gamma(alpha, T_in, T_out), for which the paper gives no formula, is the expected
+// Expected latency of a hierarchy (Theorem 3.2), the search for its parameters T and the search for
+// the hierarchy itself (Section 4, Corollary 4.1), host side.  gamma(alpha, T_in, T_out), for which the paper gives no formula, is the expected
 // number of draft/verify rounds until the yields sum to T_out when acceptances are IID with rate
 // alpha and a round yields k tokens with probability alpha^(k-1) (1 - alpha), k <= T_in, or
 // T_in + 1 with probability alpha^T_in.
@@ -74,6 +74,64 @@ int hsd_search_T(const double *costs, const double *alphas, int n_levels, int T_
     T[k]++;
   }
   for (int k = 0; k < K; ++k) out_T[k] = best[k];
+  if (out_latency) *out_latency = best_l;
+  return HSD_OK;
+}
+
+// Latency-optimal hierarchy (Section 4.2).  The paper reduces the choice of (sigma, T) to a cheapest augmented
+// path in a graph whose vertices are (model, batch size); without its self-loops that graph is acyclic (an
+// edge always leads to a strictly smaller model index), so the cheapest path is a cost-to-go recursion:
+//   down(i, j) = cheapest expected cost for a sub-hierarchy topped by model i to hand up a batch of j tokens
+//              = min( j c_i                                            (model i is the bottom level),
+//                     min_{k < i, l <= j} gamma(alpha_{k,i}, l, j) (c_i + down(k, l)) )
+//   L*        = min( c_K,  min_{i < K, j} (1 - a) / (1 - a^(j+1)) (c_K + down(i, j)) ),  a = alpha_{i,K}.
+int hsd_search_hierarchy(const double *costs, const double *alpha, int n_models, int T_max, int32_t *out_sigma,
+                         int32_t *out_n_levels, int32_t *out_T, double *out_latency) {
+  if (!costs || !out_sigma || !out_n_levels || n_models < 1 || n_models > 64 || T_max < 1 || T_max > 64)
+    return HSD_E_INVALID_ARG;
+  const int K = n_models - 1;
+  if (K > 0 && (!alpha || !out_T)) return HSD_E_INVALID_ARG;
+  for (int i = 0; i < n_models; ++i) {
+    if (!(costs[i] >= 0.0)) return HSD_E_INVALID_ARG;
+    for (int j = i + 1; j < n_models; ++j)
+      if (!(alpha[(size_t)i * n_models + j] >= 0.0 && alpha[(size_t)i * n_models + j] <= 1.0)) return HSD_E_INVALID_ARG;
+  }
+  struct Node { double cost; int prev_model, prev_T; };     // prev_model < 0: bottom level
+  std::vector<Node> down((size_t)(K > 0 ? K : 1) * (T_max + 1));
+  auto at = [&](int i, int j) -> Node & { return down[(size_t)i * (T_max + 1) + j]; };
+  for (int i = 0; i < K; ++i)
+    for (int j = 1; j <= T_max; ++j) {
+      Node best = {j * costs[i], -1, 0};
+      for (int k = 0; k < i; ++k) {
+        const double a = alpha[(size_t)k * n_models + i];
+        for (int l = 1; l <= j; ++l) {
+          const double c = gamma_rounds(a, l, j) * (costs[i] + at(k, l).cost);
+          if (c < best.cost) best = {c, k, l};
+        }
+      }
+      at(i, j) = best;
+    }
+  double best_l = costs[K];
+  int top_model = -1, top_T = 0;
+  for (int i = 0; i < K; ++i)
+    for (int j = 1; j <= T_max; ++j) {
+      const double c = top_multiplier(alpha[(size_t)i * n_models + K], j) * (costs[K] + at(i, j).cost);
+      if (c < best_l) { best_l = c; top_model = i; top_T = j; }
+    }
+  // walk the chain down from the target, then reverse it
+  std::vector<int32_t> sig, Ts;
+  sig.push_back(K);
+  for (int i = top_model, j = top_T; i >= 0;) {
+    sig.push_back(i);
+    Ts.push_back(j);
+    const Node &n = at(i, j);
+    i = n.prev_model;
+    j = n.prev_T;
+  }
+  const int n_lev = (int)sig.size();
+  for (int k = 0; k < n_lev; ++k) out_sigma[k] = sig[n_lev - 1 - k];
+  for (int k = 0; k + 1 < n_lev; ++k) out_T[k] = Ts[n_lev - 2 - k];
+  *out_n_levels = n_lev;
   if (out_latency) *out_latency = best_l;
   return HSD_OK;
 }
