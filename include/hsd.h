@@ -212,6 +212,23 @@ int hsd_search_hierarchy(const double *costs, const double *alpha, int n_models,
                          int32_t *out_n_levels, int32_t *out_T, double *out_latency);
 
 /* ---------------------------------------------------------------------------------------
+ * Calibration for the hierarchy search (Section 4.2 takes the acceptance rate alpha_{i,j} of every drafter
+ * i under every verifier j as given; Section 2: alpha = 1 - TV(p_i, p_j) = sum_x min(p_i(x), p_j(x))).
+ * From the logits of n_models models (exit layers) at the same n_rows positions, the n_models x n_models
+ * matrix of the rates averaged over the positions: alpha[i][j] = mean_r sum_x min(softmax(l_i[r])(x),
+ * softmax(l_j[r])(x)); symmetric, diagonal 1.  fp32 softmax (exp by the hardware approximation), sums in
+ * fixed order (fp32 per 128 tokens, fp64 across), no atomics: repeatable bit for bit.
+ *   logits device: model m's rows at logits + m * model_stride elements, each [n_rows, vocab] row-major,
+ *     dtype HSD_F32 or HSD_BF16; model_stride >= n_rows * vocab;
+ *   workspace device, 256-byte aligned, at least hsd_pairwise_alpha_workspace_bytes(...) (0 = bad sizes);
+ *   alpha device [n_models * n_models] doubles, row-major, written by the call (asynchronously on stream).
+ * The caller owns every buffer.  n_models <= 32.  Errors: INVALID_ARG (null, sizes, alignment, workspace too
+ * small), TOO_LARGE (n_models beyond what one block's shared memory holds), CUDA. */
+size_t hsd_pairwise_alpha_workspace_bytes(int n_models, int n_rows, int vocab);
+int hsd_pairwise_alpha(const void *logits, int dtype, int n_models, int n_rows, int vocab, long long model_stride,
+                       void *workspace, size_t workspace_bytes, double *alpha, void *stream);
+
+/* ---------------------------------------------------------------------------------------
  * One weight-streaming matrix product of the verifier forward in isolation (the contraction
  * behind every projection of Algorithm 2's multi-row forward pass): out[r, n] = sum_k A[r, k] W[n, k],
  * bf16 inputs, fp32 accumulation on the tensor cores, fp32 output.

@@ -70,6 +70,19 @@ def acceptance_rate(p, q):
     return 1.0 - 0.5 * float(np.abs(np.asarray(p, np.float64) - np.asarray(q, np.float64)).sum())
 
 
+def pairwise_acceptance(logits):
+    """alpha[i][j] = mean over positions of the acceptance rate of drafter i under verifier j (Section 2's alpha
+    between every pair of models, the input of the hierarchy search of Section 4.2).  logits: [models, rows, vocab]."""
+    logits = np.asarray(logits, np.float64)
+    L, R, _ = logits.shape
+    probs = [[softmax64(logits[l, r]) for r in range(R)] for l in range(L)]
+    alpha = np.ones((L, L))
+    for i in range(L):
+        for j in range(i + 1, L):
+            alpha[i, j] = alpha[j, i] = sum(acceptance_rate(probs[i][r], probs[j][r]) for r in range(R)) / R
+    return alpha
+
+
 # ----------------------------------------------------------------------------- layer 2
 def exp_weights(logits):
     """Integer softmax numerators E (uint64 array) of one row of stored logits.

@@ -164,6 +164,10 @@ def _declare_engine(lib):
     lib.hsd_search_hierarchy.restype = i32
     lib.hsd_search_hierarchy.argtypes = [c.POINTER(c.c_double), c.POINTER(c.c_double), i32, i32, c.POINTER(c.c_int32),
                                          c.POINTER(c.c_int32), c.POINTER(c.c_int32), c.POINTER(c.c_double)]
+    lib.hsd_pairwise_alpha_workspace_bytes.restype = sz
+    lib.hsd_pairwise_alpha_workspace_bytes.argtypes = [i32, i32, i32]
+    lib.hsd_pairwise_alpha.restype = i32
+    lib.hsd_pairwise_alpha.argtypes = [vp, i32, i32, i32, i32, c.c_longlong, vp, sz, vp, vp]
     lib.hsd_kernel_launches.restype = c.c_uint64
     lib.hsd_kernel_launches.argtypes = []
     lib.hsd_gemm_workspace_bytes.restype = sz
@@ -284,6 +288,27 @@ def hsd_search_T(costs, alphas, T_max=15, monotone=True):
                             1 if monotone else 0, out_T, ctypes.byref(out)))
     return tuple(out_T[i] for i in range(n - 1)), out.value
 
+
+
+def hsd_pairwise_alpha(logits):
+    """logits: CUDA tensor [n_models, n_rows, vocab] (fp32 or bf16) -> float64 CUDA tensor [n_models, n_models] of the
+    acceptance rates alpha[i][j] = mean over rows of sum_x min(p_i(x), p_j(x))."""
+    lib = library()
+    _declare_engine(lib)
+    L, R, V = logits.shape
+    logits = logits.contiguous()
+    need = lib.hsd_pairwise_alpha_workspace_bytes(L, R, V)
+    if need == 0:
+        raise HsdError("hsd_pairwise_alpha: unsupported sizes %s" % (tuple(logits.shape),))
+    ws = torch.empty(need + 256, dtype=torch.uint8, device=logits.device)
+    base = (ws.data_ptr() + 255) // 256 * 256
+    out = torch.empty(L, L, dtype=torch.float64, device=logits.device)
+    dtype = 1 if logits.dtype == torch.bfloat16 else 0
+    if logits.dtype not in (torch.bfloat16, torch.float32):
+        raise HsdError("hsd_pairwise_alpha: logits must be fp32 or bf16")
+    _check(lib.hsd_pairwise_alpha(_dev(logits), dtype, L, R, V, R * V, ctypes.c_void_p(base),
+                                  ws.numel() - (base - ws.data_ptr()), _dev(out), _stream()))
+    return out
 
 
 def hsd_search_hierarchy(costs, alpha, T_max=15):

@@ -150,3 +150,28 @@ def test_philox_driven_draws_follow_the_softmax():
         counts[S.categorical(l, philox.uniform24(9, j, 0, 0, 0, 0))] += 1
     chi2 = float((((counts - N * p) ** 2) / (N * p)).sum())
     assert chi2 < 45.0            # 15 degrees of freedom, p-value ~ 1e-4
+
+
+def test_pairwise_acceptance_matrix():
+    """alpha[i][j] of Section 2 between every pair of models: symmetric, ones on the diagonal, equal to the mass
+    shared by the two distributions (sum of minima), 1 for identical and 0 for disjoint models, and equal to
+    the empirical acceptance frequency of the speculative rule."""
+    rng = np.random.default_rng(3)
+    logits = rng.normal(0, 2.0, size=(4, 5, 37))
+    logits[3] = logits[0]                                   # model 3 = model 0
+    a = S.pairwise_acceptance(logits)
+    assert a.shape == (4, 4) and np.allclose(a, a.T) and np.allclose(np.diag(a), 1.0)
+    assert abs(a[0, 3] - 1.0) < 1e-12 and np.allclose(a[3, 1:3], a[0, 1:3])
+    for i in range(3):
+        for j in range(i + 1, 3):
+            shared = np.mean([np.minimum(S.softmax64(logits[i, r]), S.softmax64(logits[j, r])).sum() for r in range(5)])
+            assert abs(a[i, j] - shared) < 1e-12
+    disjoint = np.full((2, 1, 8), -1e30)
+    disjoint[0, 0, :4] = 0.0
+    disjoint[1, 0, 4:] = 0.0
+    assert abs(S.pairwise_acceptance(disjoint)[0, 1]) < 1e-12
+    # empirical: draft x ~ q, accept with probability min(1, p(x) / q(x))
+    q, p = S.softmax64(logits[1, 0]), S.softmax64(logits[2, 0])
+    xs = rng.choice(len(q), size=200000, p=q)
+    freq = float((rng.random(xs.size) < np.minimum(1.0, p[xs] / q[xs])).mean())
+    assert abs(freq - S.pairwise_acceptance(logits[1:3, :1])[0, 1]) < 5e-3
