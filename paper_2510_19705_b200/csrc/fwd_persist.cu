@@ -898,6 +898,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     if (lane == 0) {
       int s = 0, n_issued = 0;
       uint32_t par = 1;                                  // parity to wait for on the slot group's empty barrier
+      const uint64_t w_policy = l2_policy_evict_first();  // weights are read once per pass: first out of L2
       bool ok = true;
       for (int p = 0; p < n_phases && ok; ++p) {
         const Gemm g = make_gemm(a, p);
@@ -914,8 +915,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
             if (s % WGS == 0 && !mbar_wait(empty_bar(s / WGS), par, abort_flag)) { ok = false; break; }
             const uint32_t dst = smem_u32(ring) + (uint32_t)(s * Cfg::kStageBytes);
             mbar_expect_tx(full_bar(s), tx);
-            tma_load_2d(dst, m0, kb * kTcBlockK, ti.row0, full_bar(s));
-            if (second) tma_load_2d(dst + kBoxBytes, m1, kb * kTcBlockK, row1, full_bar(s));
+            tma_load_2d_hint(dst, m0, kb * kTcBlockK, ti.row0, full_bar(s), w_policy);
+            if (second) tma_load_2d_hint(dst + kBoxBytes, m1, kb * kTcBlockK, row1, full_bar(s), w_policy);
             ++n_issued;
             if (++s == STAGES) { s = 0; par ^= 1u; }
           }
