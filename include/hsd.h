@@ -212,6 +212,21 @@ int hsd_search_hierarchy(const double *costs, const double *alpha, int n_models,
                          int32_t *out_n_levels, int32_t *out_T, double *out_latency);
 
 /* ---------------------------------------------------------------------------------------
+ * Logits of chosen exit layers at every position of one token sequence (the candidates of Section 4.2's
+ * hierarchy search are early exits that share the target's final norm and output head, Section 5): one
+ * causal pass over tokens 0 .. n_tokens-1; after each layer in `layers` the shared final norm and head are
+ * applied to all rows.  Feeds hsd_pairwise_alpha.
+ *   ctx: a context from hsd_create (any hierarchy over the same model); the call uses its workspace and
+ *     resets its sequences and KV cache as a generation does, so it must not overlap one;
+ *   token_ids device [n_tokens], 1 <= n_tokens <= 128 (and <= max_seq);
+ *   layers host [n_sel]: exit layers, strictly ascending, each in 1 .. n_layers (n_layers = the full model);
+ *   out_logits device [n_sel, n_tokens, vocab] in the model's storage dtype, written by the call;
+ *   stream: the call returns after its work on the stream has completed.
+ * Errors: INVALID_ARG, OUT_OF_PAGES, CUDA, DEVICE_TIMEOUT. */
+int hsd_layer_logits(hsd_ctx *ctx, const int32_t *token_ids, int n_tokens, const int32_t *layers, int n_sel,
+                     void *out_logits, void *stream);
+
+/* ---------------------------------------------------------------------------------------
  * Calibration for the hierarchy search (Section 4.2 takes the acceptance rate alpha_{i,j} of every drafter
  * i under every verifier j as given; Section 2: alpha = 1 - TV(p_i, p_j) = sum_x min(p_i(x), p_j(x))).
  * From the logits of n_models models (exit layers) at the same n_rows positions, the n_models x n_models

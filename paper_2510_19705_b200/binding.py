@@ -168,6 +168,8 @@ def _declare_engine(lib):
     lib.hsd_pairwise_alpha_workspace_bytes.argtypes = [i32, i32, i32]
     lib.hsd_pairwise_alpha.restype = i32
     lib.hsd_pairwise_alpha.argtypes = [vp, i32, i32, i32, i32, c.c_longlong, vp, sz, vp, vp]
+    lib.hsd_layer_logits.restype = i32
+    lib.hsd_layer_logits.argtypes = [vp, vp, i32, c.POINTER(c.c_int32), i32, vp, vp]
     lib.hsd_kernel_launches.restype = c.c_uint64
     lib.hsd_kernel_launches.argtypes = []
     lib.hsd_gemm_workspace_bytes.restype = sz
@@ -230,6 +232,16 @@ class Hsd:
         _check(self._lib.hsd_generate(self._ctx, _dev(prompt_ids), batch, plen, n_new, seed, _stream(), _dev(out),
                                       stats, timing))
         return out, [s.as_dict() for s in stats], (timing[0], timing[1])
+
+    def layer_logits(self, token_ids, layers):
+        """token_ids: CUDA int32 [n_tokens] (<= 128); layers: ascending exit layers -> logits CUDA tensor
+        [len(layers), n_tokens, vocab] in the model's storage dtype (shared final norm + head after each layer)."""
+        n = int(token_ids.numel())
+        lay = (ctypes.c_int32 * len(layers))(*[int(x) for x in layers])
+        dt = torch.float32 if self.cfg["dtype"] == "fp32" else torch.bfloat16
+        out = torch.empty(len(layers), n, self.cfg["vocab"], dtype=dt, device=token_ids.device)
+        _check(self._lib.hsd_layer_logits(self._ctx, _dev(token_ids), n, lay, len(layers), _dev(out), _stream()))
+        return out
 
     def close(self):
         if getattr(self, "_ctx", None):

@@ -876,6 +876,84 @@ int hsd_generate(hsd_ctx *c, const int32_t *prompt_ids, int batch, int prompt_le
   return st;
 }
 
+// Logits of chosen exit layers at every position of one token sequence: the input of the calibration of
+// Section 4.2 (acceptance rates between all candidate drafters).  One pass over the layers with the
+// one-kernel-per-op path; after each chosen layer the shared final norm and output head are applied to all rows.
+int hsd_layer_logits(hsd_ctx *c, const int32_t *token_ids, int n_tokens, const int32_t *layers, int n_layers_sel,
+                     void *out_logits, void *stream) {
+  if (!c || !token_ids || !layers || !out_logits || n_tokens < 1 || n_layers_sel < 1) return HSD_E_INVALID_ARG;
+  const ModelDims &md = c->md;
+  const Layout &L = c->lay;
+  if (n_tokens > L.max_rows || n_tokens > md.max_seq || n_tokens > 128) return HSD_E_INVALID_ARG;
+  for (int i = 0; i < n_layers_sel; ++i)
+    if (layers[i] < 1 || layers[i] > md.n_layers || (i > 0 && layers[i] <= layers[i - 1])) return HSD_E_INVALID_ARG;
+  c->stream = (cudaStream_t)stream;
+  cudaStream_t s = c->stream;
+  // the call owns the context like a generation does: sequence 0 holds the tokens, its pages are (re)assigned
+  c->buf_len.assign(c->max_batch, 0);
+  c->len_g.assign(c->max_batch, std::vector<int>(c->n_levels, 0));
+  c->n_pages_of.assign(c->max_batch, 0);
+  c->pt_dirty.assign(c->max_batch, 0);
+  c->free_pages.clear();
+  for (int p = L.n_pages - 1; p >= 0; --p) c->free_pages.push_back(p);
+  HSD_CUDA_OK(cudaMemcpyAsync(c->dev<int>(L.tokens), token_ids, (size_t)n_tokens * 4, cudaMemcpyDeviceToDevice, s));
+  HSD_TRY(ensure_pages(c, 0, n_tokens));
+  const int R = n_tokens, n_attn = (R + kAttnRows - 1) / kAttnRows;
+  char *host, *devp;
+  HSD_TRY(ring_acquire(c, &host, &devp));
+  size_t o_seq = 0, o_pos = align_up(o_seq + (size_t)R * 4, 16), o_attn = align_up(o_pos + (size_t)R * 4, 16),
+         o_src = align_up(o_attn + (size_t)n_attn * 16, 16), o_dst = align_up(o_src + (size_t)R * 4, 16),
+         bytes = o_dst + (size_t)R * 8;
+  if (bytes > L.ring_slot) return HSD_E_INVALID_ARG;
+  int *row_seq = (int *)(host + o_seq), *row_pos = (int *)(host + o_pos), *lsrc = (int *)(host + o_src);
+  int4 *attn = (int4 *)(host + o_attn);
+  long long *ldst = (long long *)(host + o_dst);
+  for (int r = 0; r < R; ++r) { row_seq[r] = 0; row_pos[r] = r; lsrc[r] = r; ldst[r] = r; }
+  for (int i = 0; i < n_attn; ++i) attn[i] = make_int4(i * kAttnRows, std::min(kAttnRows, R - i * kAttnRows), 0, i * kAttnRows);
+  HSD_CUDA_OK(cudaMemcpyAsync(devp, host, bytes, cudaMemcpyHostToDevice, s));
+  HSD_TRY(upload_page_tables(c));
+  RowBatch rb;
+  rb.R = R; rb.row_seq = (const int *)(devp + o_seq); rb.row_pos = (const int *)(devp + o_pos);
+  rb.n_attn = n_attn; rb.attn = (const int4 *)(devp + o_attn); rb.max_kv_len = R; rb.L = R;
+  rb.lrow_src = (const int *)(devp + o_src); rb.lrow_dst = (const long long *)(devp + o_dst);
+  int n_splits = std::max(1, std::min((int)kMaxSplits, kAttnBlocksTarget / std::max(1, n_attn * md.nkv)));
+  int keys_per_split = (int)align_up((size_t)(R + n_splits - 1) / n_splits, kAttnKeyTile);
+  n_splits = (R + keys_per_split - 1) / keys_per_split;
+  float *x = c->dev<float>(L.x);
+  void *h = c->dev<void>(L.h), *q = c->dev<void>(L.q), *att = c->dev<void>(L.att), *act = c->dev<void>(L.act);
+  float *qkv = c->dev<float>(L.qkv);
+  const int *pt = c->dev<int>(L.page_table);
+  const size_t es = elem_size(md.dtype);
+  HSD_TRY(launch_embed(md, c->embed, c->dev<int>(L.tokens), rb, x, s));
+  int next = 0;
+  for (int l = 0; l < md.n_layers && next < n_layers_sel; ++l) {
+    const void *const *w = &c->lw[(size_t)l * 9];
+    void *kp = c->ws + L.k_pool + L.pool_layer_stride * l, *vp = c->ws + L.v_pool + L.pool_layer_stride * l;
+    HSD_TRY(launch_rmsnorm(md, x, w[0], nullptr, R, h, s));
+    GemmSegs qkv_segs = {{w[1], w[2], w[3]}, {md.nq * md.hd, md.nkv * md.hd, md.nkv * md.hd}, 3};
+    HSD_TRY(gemm(c, 0, h, R, md.d, qkv_segs, l * 7 + 0, GEMM_STORE_F32, qkv, nullptr, nullptr));
+    HSD_TRY(launch_rope_kv(md, qkv, rb, c->dev<float>(L.cos_tab), c->dev<float>(L.sin_tab), pt, kp, vp, q, s));
+    HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(L.partials), keys_per_split, n_splits, att, s));
+    GemmSegs o_segs = {{w[4], nullptr, nullptr}, {md.d, 0, 0}, 1};
+    HSD_TRY(gemm(c, 1, att, R, md.nq * md.hd, o_segs, l * 7 + 3, GEMM_ADD_F32, x, nullptr, nullptr));
+    HSD_TRY(launch_rmsnorm(md, x, w[5], nullptr, R, h, s));
+    GemmSegs gu_segs = {{w[6], w[7], nullptr}, {md.ff, md.ff, 0}, 2};
+    HSD_TRY(gemm(c, 0, h, R, md.d, gu_segs, l * 7 + 4, GEMM_SWIGLU_T, nullptr, act, nullptr));
+    GemmSegs d_segs = {{w[8], nullptr, nullptr}, {md.d, 0, 0}, 1};
+    HSD_TRY(gemm(c, 2, act, R, md.ff, d_segs, l * 7 + 6, GEMM_ADD_F32, x, nullptr, nullptr));
+    if (layers[next] == l + 1) {                         // exit after layer l + 1: shared final norm + head on every row
+      // (the normalised rows go to the h buffer, free between two layers and large enough for every row; the
+      // buffer of the generation path's final norm holds the few logit rows of a verification only)
+      HSD_TRY(launch_rmsnorm(md, x, c->final_norm, rb.lrow_src, R, h, s));
+      GemmSegs lm_segs = {{c->lm_head, nullptr, nullptr}, {md.V, 0, 0}, 1};
+      HSD_TRY(gemm(c, 0, h, R, md.d, lm_segs, md.n_layers * 7, GEMM_STORE_T_SCATTER, nullptr,
+                   (char *)out_logits + (size_t)next * R * md.V * es, rb.lrow_dst));
+      ++next;
+    }
+  }
+  return sync_stream(c);
+}
+
 int hsd_set_trace(hsd_ctx *c, const char *path, int logit_calls) {
   if (!c) return HSD_E_INVALID_ARG;
   if (c->trace) { fclose(c->trace); c->trace = nullptr; }
