@@ -137,6 +137,37 @@ def choose_T(binding, cfg, weights, wl, prompts, n_calib=160):
     return list(T), costs, alphas, lat
 
 
+def choose_hierarchy(binding, cfg, weights, wl, prompts, T_bar=15):
+    """Section 4.2 end to end: acceptance rates between ALL exit layers measured on the prompts (shared head on
+    every layer's hidden state), a linear cost model of an exit fitted to the measured level costs, then the
+    latency-optimal (sigma, T).  Returns (exits, T, record)."""
+    n_layers = cfg["n_layers"]
+    layers = list(range(1, n_layers + 1))
+    base_exits = list(wl["exits"])
+    T0 = [2] * (len(base_exits) - 1)
+    eng = binding.Hsd(cfg, weights, base_exits, T0, max_batch=1, max_seq=wl["prompt"] + 256, page_size=wl["page"])
+    rows = [eng.layer_logits(prompts[b % prompts.shape[0], 128 * k:128 * (k + 1)].contiguous(), layers)
+            for b, k in ((0, 0), (0, 1))]
+    alpha = binding.hsd_pairwise_alpha(torch.cat(rows, dim=1)).cpu().tolist()
+    del rows
+    eng.generate(prompts[:1], 8, 12345)
+    _, stats, _ = eng.generate(prompts[:1], 96, 12345)
+    eng.close()
+    ms = [s["ms"] / max(1, s["forwards"]) for s in stats]
+    # least-squares line through (exit layer, measured pass time): cost(e) = a e + b
+    n = len(base_exits)
+    mx, my = sum(base_exits) / n, sum(ms) / n
+    a = sum((x - mx) * (y - my) for x, y in zip(base_exits, ms)) / max(1e-12, sum((x - mx) ** 2 for x in base_exits))
+    b = my - a * mx
+    costs = [a * e + b for e in layers]
+    lat, sigma, T = binding.hsd_search_hierarchy(costs, alpha, T_bar)
+    exits = [layers[i] for i in sigma]
+    rec = {"candidates": n_layers, "cost_ms_per_layer": round(a, 5), "cost_ms_fixed": round(b, 5),
+           "alpha_to_target": [round(alpha[i][n_layers - 1], 3) for i in sigma[:-1]],
+           "expected_ms_per_token": round(lat, 4), "exits": exits, "T": list(T)}
+    return exits, list(T), rec
+
+
 def run_ours(args):
     from paper_2510_19705_b200 import binding, inputs
     rank = int(os.environ.get("RANK", "0"))
@@ -154,7 +185,15 @@ def run_ours(args):
     B = max(1, args.batch)
     prompts_host = inputs.make_prompts(cfg["vocab"], B, P, wl["prompt_seed"] + rank).pin_memory()
     prompts = prompts_host.cuda()
-    if args.T:
+    hier = None
+    if args.search_hierarchy:
+        exits, T, hier = choose_hierarchy(binding, cfg, weights, wl, prompts)
+        wl = dict(wl, exits=tuple(exits), T=tuple(T))
+        if len(exits) == 1:
+            T = []
+    if args.search_hierarchy:
+        calib = None
+    elif args.T:
         T, calib = [int(v) for v in args.T.split(",")], None
     elif wl["T"] is None:
         T, costs, alphas, lat = choose_T(binding, cfg, weights, wl, prompts)
@@ -231,7 +270,7 @@ def run_ours(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dec_ms_step, 3), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
         "config": {"workload": args.workload, "batch": B, "prompt_len": P, "n_new": n_new, "exits": list(wl["exits"]),
-                   "T": T, "T_search": calib, "l2": "inputs larger than L2 (weights %.1f GB per target pass)"
+                   "T": T, "T_search": calib, "hierarchy_search": hier, "l2": "inputs larger than L2 (weights %.1f GB per target pass)"
                    % (weight_bytes(cfg, cfg["n_layers"]) / 1e9), "replicas": "independent sequence per GPU"},
         "prefill_ms": round(pre_ms_step, 3), "step_ms_with_prefill": round(step_ms, 3),
         "e2e": {"value": round(aggregate_tokens_per_s(world, B * n_new, e2e_ms), 2), "unit": UNIT, "h2d_bytes_per_step": B * P * 4,
@@ -392,6 +431,8 @@ def main():
     ap.add_argument("--batch", type=int, default=1, help="sequences per GPU (the metric is quoted at 1)")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length (development runs)")
     ap.add_argument("--T", default="", help="fix T (comma separated) instead of calibrating / using the workload's")
+    ap.add_argument("--search-hierarchy", action="store_true",
+                    help="choose the exit layers and T by the latency-optimal hierarchy search over all layers (not the default config)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
