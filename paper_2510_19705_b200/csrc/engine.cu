@@ -180,6 +180,7 @@ struct hsd_ctx {
   // tensor-core GEMM state (bf16 models)
   bool use_tc, use_persist;
   int attn_single_max = 0;                    // contexts up to this many keys use one attention key split
+  bool no_fuse_qkv = false;                   // debugging aid (HSD_NO_FUSE_QKV): keep the QKV finish phase in every pass
   int sm_count;
   std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + 1]: wq wk wv wo wg wu wd per layer, then lm_head
   CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
@@ -295,12 +296,14 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   const ModelDims &md = c->md;
   const Layout &L = c->lay;
   int R = 0, n_attn = 0, n_logit = 0, max_kv = 0;
+  bool one_item_per_seq = true;
   const int arows = c->use_persist ? fwd_attn_rows(md.nq / md.nkv, md.hd) : kAttnRows;   // rows per attention item
   for (const SeqWork &w : work) {
     int rows = w.end - w.start;
     if (rows <= 0 || w.start < 0 || w.end > md.max_seq) return HSD_E_INVALID_ARG;
     R += rows;
     n_attn += (rows + arows - 1) / arows;
+    if (rows > arows) one_item_per_seq = false;
     if (w.logit_first >= 0) {
       if (w.logit_first < w.start || w.logit_first >= w.end) return HSD_E_INVALID_ARG;
       n_logit += w.end - w.logit_first;
@@ -442,6 +445,8 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     // shared memory that only feeds accumulator columns nobody reads): 148 CTAs x K / 64 boxes per GEMM add up
     const int box_rows = std::max(R, n_logit) <= 16 ? std::max(R, n_logit) : np;
     a.a_box_rows = box_rows;
+    // the new keys of an attention item are then its own rows only: the QKV finish phase folds into attention
+    a.fuse_qkv = (one_item_per_seq && !c->no_fuse_qkv) ? 1 : 0;
     for (int b = 0; b < 4; ++b) a.amap[b] = box_rows <= 16 ? c->amaps_rows[b][box_rows - 1] : c->amaps[b][pi];
     // debugging aid: HSD_PROFILE=<file> dumps the barrier timeline of the latest top-level pass
     const char *prof_path = getenv("HSD_PROFILE");
@@ -805,6 +810,7 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
       c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 && (md.d / kTcBlockM) * 2 <= c->sm_count && md.n_layers <= 64 && (md.page & (md.page - 1)) == 0 && md.page >= 16 &&
                        getenv("HSD_NO_PERSIST") == nullptr;
       if (const char *e = getenv("HSD_ATTN_SINGLE_MAX")) c->attn_single_max = atoi(e);
+      c->no_fuse_qkv = getenv("HSD_NO_FUSE_QKV") != nullptr;
     }
     if (!st && cudaMallocHost(&c->status_host, 4) != cudaSuccess) st = HSD_E_CUDA;
     if (st) {

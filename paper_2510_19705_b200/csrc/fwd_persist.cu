@@ -363,9 +363,10 @@ __device__ __forceinline__ void ldmatrix_x4_trans(unsigned *r, const void *row_p
 // (rows x group) every warp works on its own sub-tiles; with 17..32 the warps pair up on a sub-tile,
 // one 16-row m-tile each.  At the end the warps' states are merged through shared memory and the
 // split's partial (o, m, l) goes to global memory.
-template <int HD>
+template <int NPAD, int HD>
 __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt, long long *dbg,
-                                                 const int *first_item) {
+                                                 const int *first_item, const int *qkv_geom, const int *row_pg_sh, const float *rope_cos_sh,
+                                                 const float *rope_sin_sh) {
   constexpr int CPR = HD / 8;                      // 16-byte chunks per row
   // Rows of Q, K, V in shared memory: HD >= 64: unpadded, the 16-byte chunk index XORed with the row's low
   // three bits; HD = 32: padded by 16 bytes.  Either way the fragment loads (eight rows, same chunk) and
@@ -385,7 +386,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
   static_assert(8 * 16 * MS * 4 <= 9 * 32 * RS * 2, "merge area must fit the Q and K/V buffers");
   static_assert(9 * 32 * RS * 2 <= kScratchBytes - 2 * kRopeCacheRows * (HD / 2) * 4, "attention buffers overlap the rope cache");
   const __nv_bfloat16 *kpool = lay.k_pool, *vpool = lay.v_pool;
-  const float scale = rsqrtf((float)HD);
+  const float scale = rsqrtf((float)HD), inv_group = 1.f / (float)group;
   const int n_work = a.n_attn * a.nkv * a.n_splits;
 #pragma unroll 1
   for (int wi = blockIdx.x; wi < n_work; wi += gridDim.x) {
@@ -405,10 +406,12 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
     worker_sync();                                               // previous item's merge area fully read
     // ---- q rows of the item (whole CTA) and this warp's page ids: lane j holds the page of the warp's j-th
     //      sub-tile (re-read every 32 sub-tiles); kept in shared memory across layers when the CTA has one item
-    for (int i = wt; i < nqv * CPR; i += 256) {
-      const int qi = i / CPR, ch = i % CPR;
-      const int r = qi / group, gq = qi % group;
-      cp_async16(shQ + qi * RS + swz(qi, ch) * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + gq) * HD + ch * 8);
+    if (!a.fuse_qkv) {
+      for (int i = wt; i < nqv * CPR; i += 256) {
+        const int qi = i / CPR, ch = i % CPR;
+        const int r = qi / group, gq = qi % group;
+        cp_async16(shQ + qi * RS + swz(qi, ch) * 8, a.q + ((size_t)(row0 + r) * a.nq + kvh * group + gq) * HD + ch * 8);
+      }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
     const bool pages_cached = (pc->tag_item == wi) && n_mine <= 16;
@@ -426,20 +429,117 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
       }
     };
     load_pages(0);
-    auto issue = [&](const __nv_bfloat16 *pool, __nv_bfloat16 *sh, int j, bool zero_pad) {    // one sub-tile, one operand
-      const int kt = key_lo + (first + j * step) * 16, nk = min(16, key_hi - kt);
+    // `key_stop`: keys from there on are not fetched (fused QKV finish: the item's own new keys are written
+    // straight into the buffers of a warp's first sub-tile by the threads that compute them)
+    auto issue = [&](const __nv_bfloat16 *pool, __nv_bfloat16 *sh, int j, bool zero_pad, int key_stop) {    // one sub-tile, one operand
+      const int kt = key_lo + (first + j * step) * 16, nk = min(16, key_hi - kt), nload = min(nk, key_stop - kt);
       const int pg = __shfl_sync(0xFFFFFFFFu, pg_reg, j - pg_base);
       const size_t base = ((((size_t)pg * a.nkv + kvh) << a.page_shift) + (kt & (a.page - 1))) * HD;
 #pragma unroll
       for (int i = 0; i < 16 * CPR / 32; ++i) {
         const int idx = i * 32 + lane, kk = idx / CPR, ch = idx % CPR;
-        if (kk < nk) cp_async16(sh + kk * RS + swz(kk, ch) * 8, pool + base + (size_t)kk * HD + ch * 8);
-        else if (zero_pad) *reinterpret_cast<uint4 *>(sh + kk * RS + ch * 8) = make_uint4(0u, 0u, 0u, 0u);   // P is 0 there, V must be finite
+        if (kk < nload) cp_async16(sh + kk * RS + swz(kk, ch) * 8, pool + base + (size_t)kk * HD + ch * 8);
+        else if (zero_pad && kk >= nk) *reinterpret_cast<uint4 *>(sh + kk * RS + ch * 8) = make_uint4(0u, 0u, 0u, 0u);   // P is 0 there, V must be finite
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    if (n_mine > 0) { issue(kpool, shK, 0, false); issue(vpool, shV, 0, true); }
+    constexpr int kAllKeys = 0x7FFFFFFF;
+    const int first_stop = a.fuse_qkv ? pos0 : kAllKeys;
+    if (n_mine > 0) { issue(kpool, shK, 0, false, first_stop); issue(vpool, shV, 0, true, first_stop); }
     else { asm volatile("cp.async.commit_group;\n\tcp.async.commit_group;" ::: "memory"); }
+    if (a.fuse_qkv) {
+      // ---- QKV finish of the item's own rows: pieces of the projection summed in piece order, rotary embedding,
+      //      q -> the Q buffer, k / v of the rows whose position falls into this key split -> their cache page
+      //      (and the first sub-tile's buffers, when that is where they belong).  A unit = 8 columns of one
+      //      vector plus the 8 columns half a head further on (rotation partners): two 16-byte chunks.
+      // geometry of the QKV projection's pieces (the same in every layer; worked out once at kernel start):
+      // qg[0..6] = first tile of k, first tile of v, parts, pieces_max, U, Gp, KB
+      constexpr int UPV = HD / 16, HALF = HD / 2;
+      const int tile_k = qkv_geom[0], tile_v = qkv_geom[1], g_parts = qkv_geom[2], g_pmax = qkv_geom[3];
+      const int nr_lo = max(0, key_lo - pos0), n_new = max(0, min(nrows, key_hi - pos0) - nr_lo);
+      const int n_units = (nqv + 2 * n_new) * UPV;
+      const bool rope_cached = a.R <= kRopeCacheRows;
+      const size_t pstride = (size_t)NPAD * kTcBlockM;
+#pragma unroll 1
+      for (int u = wt; u < n_units; u += 256) {
+        const int vec = u / UPV, c8 = u % UPV;
+        int kind, rr, n, tile0;
+        if (vec < nqv) { kind = 0; rr = (int)(((float)vec + 0.5f) * inv_group); n = (kvh * group + vec - rr * group) * HD; tile0 = 0; }
+        else {
+          const int v2 = vec - nqv, isv = v2 >= n_new ? 1 : 0;
+          kind = 1 + isv; rr = nr_lo + v2 - isv * n_new; n = kvh * HD; tile0 = isv ? tile_v : tile_k;
+        }
+        n += c8 * 8;
+        const int tile = tile0 + n / kTcBlockM, m = n % kTcBlockM;
+        int n_pieces = g_parts;
+        if (g_parts == 0) {                                      // dealt units: the owners of the tile's first and last k-block
+          const int U = qkv_geom[4], Gp = qkv_geom[5], KB = qkv_geom[6];
+          n_pieces = unit_owner(U, Gp, tile * KB + KB - 1) - unit_owner(U, Gp, tile * KB) + 1;
+        }
+        const float *base = a.pieces + ((size_t)(tile * g_pmax) * NPAD + (row0 + rr)) * kTcBlockM + m;
+        float4 pc4[4][4];                                        // [piece][low 0-3, low 4-7, high 0-3, high 4-7]
+#pragma unroll
+        for (int pp = 0; pp < 4; ++pp) {
+          const float4 *src = reinterpret_cast<const float4 *>(base + pp * pstride);
+          const bool on = pp < n_pieces;
+          pc4[pp][0] = on ? __ldcg(src) : make_float4(0.f, 0.f, 0.f, 0.f);
+          pc4[pp][1] = on ? __ldcg(src + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+          pc4[pp][2] = on ? __ldcg(src + HALF / 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          pc4[pp][3] = on ? __ldcg(src + HALF / 4 + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float cs[8], sn[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { cs[e] = 1.f; sn[e] = 0.f; }
+        if (kind < 2) {
+          const float *ct = rope_cached ? rope_cos_sh + (row0 + rr) * HALF + c8 * 8 : a.cos_tab + (size_t)(pos0 + rr) * HALF + c8 * 8;
+          const float *st = rope_cached ? rope_sin_sh + (row0 + rr) * HALF + c8 * 8 : a.sin_tab + (size_t)(pos0 + rr) * HALF + c8 * 8;
+#pragma unroll
+          for (int e = 0; e < 8; e += 4) {
+            const float4 cv = *reinterpret_cast<const float4 *>(ct + e), sv = *reinterpret_cast<const float4 *>(st + e);
+            cs[e] = cv.x; cs[e + 1] = cv.y; cs[e + 2] = cv.z; cs[e + 3] = cv.w;
+            sn[e] = sv.x; sn[e + 1] = sv.y; sn[e + 2] = sv.z; sn[e + 3] = sv.w;
+          }
+        }
+        float lo[8], hi[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) { lo[e] = 0.f; hi[e] = 0.f; }
+#pragma unroll
+        for (int pp = 0; pp < 4; ++pp) {
+          lo[0] += pc4[pp][0].x; lo[1] += pc4[pp][0].y; lo[2] += pc4[pp][0].z; lo[3] += pc4[pp][0].w;
+          lo[4] += pc4[pp][1].x; lo[5] += pc4[pp][1].y; lo[6] += pc4[pp][1].z; lo[7] += pc4[pp][1].w;
+          hi[0] += pc4[pp][2].x; hi[1] += pc4[pp][2].y; hi[2] += pc4[pp][2].z; hi[3] += pc4[pp][2].w;
+          hi[4] += pc4[pp][3].x; hi[5] += pc4[pp][3].y; hi[6] += pc4[pp][3].z; hi[7] += pc4[pp][3].w;
+        }
+        unsigned wl[4], wh[4];
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+          const __nv_bfloat162 l2 = __floats2bfloat162_rn(lo[e] * cs[e] - hi[e] * sn[e], lo[e + 1] * cs[e + 1] - hi[e + 1] * sn[e + 1]);
+          const __nv_bfloat162 h2 = __floats2bfloat162_rn(hi[e] * cs[e] + lo[e] * sn[e], hi[e + 1] * cs[e + 1] + lo[e + 1] * sn[e + 1]);
+          wl[e >> 1] = *reinterpret_cast<const unsigned *>(&l2);
+          wh[e >> 1] = *reinterpret_cast<const unsigned *>(&h2);
+        }
+        const uint4 vl = make_uint4(wl[0], wl[1], wl[2], wl[3]), vh = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+        if (kind == 0) {
+          *reinterpret_cast<uint4 *>(shQ + vec * RS + swz(vec, c8) * 8) = vl;
+          *reinterpret_cast<uint4 *>(shQ + vec * RS + swz(vec, c8 + CPR / 2) * 8) = vh;
+        } else {
+          const int pos = pos0 + rr;
+          __nv_bfloat16 *pool = kind == 1 ? lay.k_pool : lay.v_pool;
+          const size_t off = (((size_t)row_pg_sh[row0 + rr] * a.nkv + kvh) * a.page + (pos & (a.page - 1))) * HD + c8 * 8;
+          *reinterpret_cast<uint4 *>(pool + off) = vl;
+          *reinterpret_cast<uint4 *>(pool + off + HALF) = vh;
+          const int st = (pos - key_lo) >> 4, kk = (pos - key_lo) & 15;
+          if (st < step) {                                       // a first sub-tile: its warp (pair) is waiting for these rows
+            const int w0 = n_mt == 2 ? 2 * st : st;
+            for (int ww = w0; ww < w0 + (n_mt == 2 ? 2 : 1); ++ww) {
+              __nv_bfloat16 *sh = shQ + 32 * RS + ww * (32 * RS) + (kind == 2 ? 16 * RS : 0);
+              *reinterpret_cast<uint4 *>(sh + kk * RS + swz(kk, c8) * 8) = vl;
+              *reinterpret_cast<uint4 *>(sh + kk * RS + swz(kk, c8 + CPR / 2) * 8) = vh;
+            }
+          }
+        }
+      }
+    }
     float o[NT][4];
 #pragma unroll
     for (int n = 0; n < NT; ++n)
@@ -480,7 +580,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
         }
       }
       __syncwarp();                                              // every lane is done with the K buffer
-      if (j + 1 < n_mine) issue(kpool, shK, j + 1, false);
+      if (j + 1 < n_mine) issue(kpool, shK, j + 1, false, kAllKeys);
       else asm volatile("cp.async.commit_group;" ::: "memory");  // keep the group count uniform
       // ---- online softmax on the accumulator rows (g and g + 8); P re-packed as the A operand of P V
       unsigned ph[4], pl[4];
@@ -542,7 +642,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
         }
       }
       __syncwarp();                                              // every lane is done with the V buffer
-      if (j + 1 < n_mine) issue(vpool, shV, j + 1, true);
+      if (j + 1 < n_mine) issue(vpool, shV, j + 1, true, kAllKeys);
       else asm volatile("cp.async.commit_group;" ::: "memory");
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
@@ -845,6 +945,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   uint32_t *tmem_slot = ctl;
   volatile int *abort_flag = reinterpret_cast<volatile int *>(ctl + 1);
   int *first_item_sh = reinterpret_cast<int *>(ctl + 148);               // [4] this CTA's first attention item
+  int *qkv_geom_sh = reinterpret_cast<int *>(ctl + 152);                 // [7] piece geometry of the QKV projection
   volatile int *wait_ok = reinterpret_cast<volatile int *>(ctl + 4);   // [2]
   float *red = reinterpret_cast<float *>(ctl + 8);                      // [8]
   PageCache *pcache = reinterpret_cast<PageCache *>(ctl + 16);          // 130 words
@@ -1032,6 +1133,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       int4 fi = make_int4(0, 0, 0, 0);
       if ((int)blockIdx.x < n_work) fi = a.attn_items[blockIdx.x / (a.n_splits * a.nkv)];
       first_item_sh[0] = fi.x; first_item_sh[1] = fi.y; first_item_sh[2] = fi.z; first_item_sh[3] = fi.w;
+      const Gemm gq = make_gemm(a, 0);
+      const SplitGeom geo = split_geom(gq, G);
+      qkv_geom_sh[0] = (gq.seg_n[0] + kTcBlockM - 1) / kTcBlockM;
+      qkv_geom_sh[1] = qkv_geom_sh[0] + (gq.seg_n[1] + kTcBlockM - 1) / kTcBlockM;
+      qkv_geom_sh[2] = geo.parts; qkv_geom_sh[3] = geo.pieces_max; qkv_geom_sh[4] = geo.U; qkv_geom_sh[5] = geo.Gp; qkv_geom_sh[6] = gq.KB;
     }
     // One step loop, one call site per phase body: the whole per-layer program has to stay resident in
     // the instruction cache (every phase runs once per layer, so code that does not fit is fetched
@@ -1054,7 +1160,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         const int sstep = (t - 1) % 10, p = 4 * l;
         switch (sstep) {
           case 0: kind = K_EPI; gp = p; break;
-          case 1: kind = K_FIN; gp = p; break;
+          case 1:                                            // folded into the attention phase when every item stands alone
+            if (a.fuse_qkv) { kind = K_NONE; barrier = false; }
+            else { kind = K_FIN; gp = p; }
+            break;
           case 2: kind = K_ATTN_A; if (a.n_splits == 1) ready = p + 1; break;       // a single key split needs no merge phase
           case 3:
             if (a.n_splits == 1) { kind = K_NONE; barrier = false; }
@@ -1074,7 +1183,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       switch (kind) {
         case K_EPI: if (is_epi) gemm_epilogue<NPAD>(a, w, gp); break;
         case K_FIN: gemm_finish<NPAD>(a, w, gp); break;
-        case K_ATTN_A: attn_tiles_phase<HD>(a, layers_sh[l], scratch, pcache, wt, dbg_cy, first_item_sh); break;
+        case K_ATTN_A:
+          attn_tiles_phase<NPAD, HD>(a, layers_sh[l], scratch, pcache, wt, dbg_cy, first_item_sh, qkv_geom_sh, row_pg_sh, rope_cos_sh, rope_sin_sh);
+          break;
         case K_ATTN_B: attn_merge_phase<HD>(a, row_pos_sh, wt); break;
         case K_NORM: {
           const bool first = (t == 0);

@@ -25,6 +25,7 @@ struct FwdArgs {
   // this call
   int R, L, n_attn, attn_rows, n_splits, keys_per_split;
   int a_box_rows;                  // rows of one activation TMA box (<= the row padding)
+  int fuse_qkv;                    // 1: every sequence is one attention item; the item's CTAs finish its q / k / v themselves
   const int *tokens, *page_table, *row_seq, *row_pos, *lrow_src;
   const int4 *attn_items;          // (first packed row, rows, sequence, position of first row)
   const long long *lrow_dst;

@@ -139,6 +139,28 @@ def test_page_size_does_not_change_the_stream(lib):
     assert torch.equal(outs[0], outs[1]) and torch.equal(outs[1], outs[2])
 
 
+@pytest.mark.parametrize("name", ["mini3", "mini4long"])
+def test_folded_qkv_finish_gives_the_stream_of_the_separate_phase(lib, name, monkeypatch):
+    """Decode passes fold the QKV finish (piece sum, rotary embedding, cache write) into the attention phase;
+    HSD_NO_FUSE_QKV keeps the separate phase.  Same sums in the same order: the token streams are equal."""
+    wl = inputs.WORKLOADS[name]
+    cfg = wl["model"]
+    w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
+    batch = wl.get("batch", 1)
+    prompts = inputs.make_prompts(cfg["vocab"], batch, wl["prompt"], wl["prompt_seed"]).cuda()
+    max_seq = wl["prompt"] + wl["n_new"] + sum(wl["T"]) + len(wl["exits"]) + 8
+    outs = []
+    for separate in (False, True):
+        if separate:
+            monkeypatch.setenv("HSD_NO_FUSE_QKV", "1")
+        else:
+            monkeypatch.delenv("HSD_NO_FUSE_QKV", raising=False)
+        eng = lib.Hsd(cfg, w, wl["exits"], wl["T"], max_batch=batch, max_seq=max_seq, page_size=wl["page"])
+        outs.append(eng.generate(prompts, wl["n_new"], 1)[0].cpu())
+        eng.close()
+    assert torch.equal(outs[0], outs[1])
+
+
 def test_mini_bf16_decisions_follow_the_oracle_on_the_same_logits(lib, tmp_path):
     """bf16: the two forwards differ by rounding, so the stream is checked call by call: given the
     library's own stored logits, the oracle's decision arithmetic must reproduce every token and accept
