@@ -39,7 +39,7 @@ size_t elem_size(int dtype) { return dtype == HSD_BF16 ? 2 : 4; }
 // Workspace layout, shared by hsd_workspace_bytes and hsd_create.
 struct Layout {
   size_t tokens, cos_tab, sin_tab, page_table, k_pool, v_pool, pool_layer_stride, x, h, qkv, q, att, act, partials, hf,
-      vscratch, n_acc, ring, tc_scratch, tc_pieces_bytes, wmaps_dev, layers_dev, attn_counters, grid_counter, prof, total;
+      vscratch, n_acc, ring, tc_scratch, tc_pieces_bytes, tc_pieces2, wmaps_dev, layers_dev, attn_counters, grid_counter, prof, total;
   std::vector<size_t> logits;
   std::vector<int> slots;
   int max_rows, pages_per_seq, n_pages, partial_rows;
@@ -128,6 +128,7 @@ Layout make_layout(const hsd_model_desc *m, int n_levels, const int32_t *T) {
       }
   }
   L.tc_scratch = take(kTcCtrlBytes + L.tc_pieces_bytes);
+  L.tc_pieces2 = take(L.tc_pieces_bytes);       // second piece buffer (down projection of passes with few rows)
   L.wmaps_dev = take(((size_t)m->n_layers * 7 + 1) * sizeof(CUtensorMap));
   L.layers_dev = take((size_t)m->n_layers * sizeof(FwdLayerDev));
   L.attn_counters = take(16384);
@@ -181,6 +182,7 @@ struct hsd_ctx {
   bool use_tc, use_persist;
   int attn_single_max = 0;                    // contexts up to this many keys use one attention key split
   bool no_fuse_qkv = false;                   // debugging aid (HSD_NO_FUSE_QKV): keep the QKV finish phase in every pass
+  bool no_fuse_gu = false;                    // debugging aid (HSD_NO_FUSE_GU): keep the gate / up finish phase in every pass
   int sm_count;
   std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + 1]: wq wk wv wo wg wu wd per layer, then lm_head
   CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
@@ -447,6 +449,9 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     a.a_box_rows = box_rows;
     // the new keys of an attention item are then its own rows only: the QKV finish phase folds into attention
     a.fuse_qkv = (one_item_per_seq && !c->no_fuse_qkv) ? 1 : 0;
+    // few rows: the SwiGLU finish folds into the down projection (its CTAs build their activation tiles)
+    a.fuse_gu = (R <= 4 && !c->no_fuse_gu) ? 1 : 0;
+    a.pieces2 = (float *)(c->ws + L.tc_pieces2);
     for (int b = 0; b < 4; ++b) a.amap[b] = box_rows <= 16 ? c->amaps_rows[b][box_rows - 1] : c->amaps[b][pi];
     // debugging aid: HSD_PROFILE=<file> dumps the barrier timeline of the latest top-level pass
     const char *prof_path = getenv("HSD_PROFILE");
@@ -811,6 +816,7 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
                        getenv("HSD_NO_PERSIST") == nullptr;
       if (const char *e = getenv("HSD_ATTN_SINGLE_MAX")) c->attn_single_max = atoi(e);
       c->no_fuse_qkv = getenv("HSD_NO_FUSE_QKV") != nullptr;
+      c->no_fuse_gu = getenv("HSD_NO_FUSE_GU") != nullptr;
     }
     if (!st && cudaMallocHost(&c->status_host, 4) != cudaSuccess) st = HSD_E_CUDA;
     if (st) {

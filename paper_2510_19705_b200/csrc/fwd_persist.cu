@@ -160,6 +160,10 @@ __device__ __forceinline__ void tile_pieces(const Gemm &g, const SplitGeom &geo,
   first_owner = unit_owner(geo.U, geo.Gp, tile * g.KB);
   n = unit_owner(geo.U, geo.Gp, tile * g.KB + g.KB - 1) - first_owner + 1;
 }
+// Phase p is a down projection whose activation tiles are built in place from the gate / up pieces: its own
+// pieces then go to the second buffer (the first is still being read by slower CTAs).
+__device__ __forceinline__ bool built_down(const FwdArgs &a, int p) { return a.fuse_gu && (p & 3) == 3 && p < 4 * a.n_run; }
+__device__ __forceinline__ float *pieces_of(const FwdArgs &a, int p) { return built_down(a, p) ? a.pieces2 : a.pieces; }
 __device__ __forceinline__ void worker_sync() { asm volatile("bar.sync 2, 256;" ::: "memory"); }
 __device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 // barrier of one 128-thread worker group (id 1 = warps 4..7, the epilogue group; id 3 = warps 8..11)
@@ -230,8 +234,8 @@ __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, 
 // Requires d % 4 == 0 and d <= 4096.
 template <int NPAD>
 __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const int *row_list, bool src_embed,
-                                           const Gemm *pend, const __nv_bfloat16 *gain, __nv_bfloat16 *dst, float *red,
-                                           int wt) {
+                                           const Gemm *pend, const float *pend_pieces, const __nv_bfloat16 *gain, __nv_bfloat16 *dst,
+                                           float *red, int wt) {
   constexpr int MAXV = 4;                                  // float4 slots per thread
   constexpr int PB = 4;                                    // pieces loaded at a time per slot
   const int d = a.d, nvec = d >> 2;
@@ -276,7 +280,7 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
 #pragma unroll
       for (int j = 0; j < MAXV; ++j) {
         const int iv = wt + 256 * j, k = iv << 2, tile = k >> 7, mm = k & 127;
-        const float *base = a.pieces + ((size_t)tile * np * NPAD + row) * kTcBlockM + mm;
+        const float *base = pend_pieces + ((size_t)tile * np * NPAD + row) * kTcBlockM + mm;
 #pragma unroll
         for (int pp = 0; pp < PB; ++pp)
           t[j][pp] = (iv < nvec && pp < np) ? __ldcg(reinterpret_cast<const float4 *>(base + (size_t)pp * NPAD * kTcBlockM))
@@ -775,7 +779,7 @@ __device__ __forceinline__ void final_store(const FwdArgs &a, const Gemm &g, con
       const int r = c0 + i, col = ti.row0 + cc;
       if (r < rows && col < g.seg_n[0]) {
         const float gt = staging[cc * (CH + 1) + i], up = staging[(cc + kTcBoxRows) * (CH + 1) + i];
-        a.act[(size_t)r * a.ff + col] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * up);
+        a.act[(size_t)r * a.ff + col] = __float2bfloat16_rn(silu_mul(gt, up));
       }
     }
     group_sync(bar_id);
@@ -840,7 +844,7 @@ __device__ __forceinline__ void gemm_epilogue(const FwdArgs &a, WorkerCtx &w, in
       int fo, np_tile;
       tile_pieces(g, geo, sg.tile, fo, np_tile);
       const int piece = w.c - fo;
-      float *mine = a.pieces + ((size_t)sg.tile * geo.pieces_max + piece) * NPAD * kTcBlockM;
+      float *mine = pieces_of(a, p) + ((size_t)sg.tile * geo.pieces_max + piece) * NPAD * kTcBlockM;
       if (w.wt == 0) w.wait_ok[w.seg_idx & 1] = mbar_wait((w.accf_bar0 + 8u * ab), (uint32_t)((w.seg_idx >> 1) & 1), w.abort_flag) ? 1 : 0;
       epi_sync();
       if (!w.wait_ok[w.seg_idx & 1]) return;
@@ -865,6 +869,103 @@ __device__ __forceinline__ void gemm_epilogue(const FwdArgs &a, WorkerCtx &w, in
       }
     }
   }
+
+// Down projection p of a pass with at most four rows: the worker warps build its activation tiles straight into
+// the ring slots (SwiGLU of the gate / up pieces, summed in piece order; k-block kb of the down projection is tile
+// kb of gate / up), in the layout the activation TMA box would have had (128-byte rows, 16-byte chunk index XOR
+// row & 7).  Builder warp i of four takes the CTA's stages i, i + 4, ...; a lane covers one row x 8 columns.  Under the weight
+// stream a load from L2 takes longer than a ring slot's turn-around, so with at most two pieces per tile (PB = 2)
+// a warp keeps the loads of its next two stages in flight (DEPTH = 2).
+template <int NPAD, int PB, int DEPTH>
+__device__ __forceinline__ void build_act_stages(const FwdArgs &a, WorkerCtx &w, int p, uint8_t *ring, uint32_t full_bar0,
+                                                 uint32_t empty_bar0, volatile unsigned *ring_pos, const int *bgeom) {
+  constexpr int STAGES = PCfg<NPAD>::kStages;
+  // geometry worked out once at kernel start (the same in every layer): this CTA's k-blocks of the down projection
+  // (residual projections: one segment per CTA) and how the gate / up tiles are cut into pieces
+  SegIter it;
+  it.tile = 0; it.kb = bgeom[0]; it.left = bgeom[1];
+  const int g_parts = bgeom[2], g_pmax = bgeom[3];
+  const int KBg = a.d / kTcBlockK, Ug = ((a.ff + kTcBoxRows - 1) / kTcBoxRows) * KBg, Gpg = min(w.G, Ug);
+  const float inv_U = 1.f / (float)Ug;
+  // unit_owner without an integer division (all quantities < 2^24, so the float quotient is off by one at most)
+  auto owner = [&](int u) {
+    const int x = (u + 1) * Gpg - 1;
+    int q = (int)((float)x * inv_U);
+    const int rem = x - q * Ug;
+    return rem < 0 ? q - 1 : (rem >= Ug ? q + 1 : q);
+  };
+  // builders: the four worker warps that share no scheduler with the weight producer or the MMA issuer (single
+  // threads whose issue rate bounds the phase)
+  if (it.left <= 0 || ((w.wt >> 5) & 1) == 0) return;
+  // ring position (slot, parity of its empty barrier) of the phase's first stage, published by the weight producer
+  ring_pos += (p >> 2) & 15;
+  unsigned rp = *ring_pos;
+  if ((int)(rp >> 16) != p) {
+    const unsigned long long t0 = globaltimer_ns();
+    while ((int)((rp = *ring_pos) >> 16) != p)
+      if (*w.abort_flag || globaltimer_ns() - t0 > kWaitLimitNs) { *w.abort_flag = 1; return; }
+  }
+  const int s0 = (int)(rp & 0xFFu), warp4 = w.wt >> 6, r = w.lane >> 3, c8 = w.lane & 7;
+  const uint32_t par0 = (rp >> 8) & 1u;
+  const bool on = r < a.R;
+  const size_t pstride = (size_t)NPAD * kTcBlockM;
+  const float *lane_base = a.pieces + (size_t)r * kTcBlockM + c8 * 8;
+  float4 t[DEPTH][PB][4];                                      // [stage in flight][piece][gate 0-3, gate 4-7, up 0-3, up 4-7]
+  auto load = [&](float4 (&dst)[PB][4], int i) {               // pieces of the CTA's stage i (this lane's row and columns)
+    const int kb = it.kb + i;
+    int n_pieces = 0;
+    if (i < it.left) n_pieces = g_parts ? g_parts : owner(kb * KBg + KBg - 1) - owner(kb * KBg) + 1;
+    const float *tbase = lane_base + (size_t)kb * g_pmax * pstride;
+#pragma unroll
+    for (int pp = 0; pp < PB; ++pp) {
+      const float4 *src = reinterpret_cast<const float4 *>(tbase + pp * pstride);
+      const bool ld = on && pp < n_pieces;
+      dst[pp][0] = ld ? __ldcg(src) : make_float4(0.f, 0.f, 0.f, 0.f);
+      dst[pp][1] = ld ? __ldcg(src + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+      dst[pp][2] = ld ? __ldcg(src + kTcBoxRows / 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      dst[pp][3] = ld ? __ldcg(src + kTcBoxRows / 4 + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
+#pragma unroll
+  for (int dpt = 0; dpt < DEPTH; ++dpt) load(t[dpt], warp4 + 4 * dpt);
+#pragma unroll 1
+  for (int i0 = warp4; i0 < it.left; i0 += 4 * DEPTH) {
+#pragma unroll
+    for (int dpt = 0; dpt < DEPTH; ++dpt) {
+      const int i = i0 + 4 * dpt;
+      if (i >= it.left) break;
+      const int pos = s0 + i, s = pos % STAGES;
+      const uint32_t par = par0 ^ (uint32_t)((pos / STAGES) & 1);
+      bool ok = true;                                          // the slot is free once its previous MMAs have retired
+      if (w.lane == 0) ok = mbar_wait(empty_bar0 + 8u * s, par, w.abort_flag);
+      if (!__shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0)) return;
+      float gt[8], up[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { gt[e] = 0.f; up[e] = 0.f; }
+#pragma unroll
+      for (int pp = 0; pp < PB; ++pp) {
+        gt[0] += t[dpt][pp][0].x; gt[1] += t[dpt][pp][0].y; gt[2] += t[dpt][pp][0].z; gt[3] += t[dpt][pp][0].w;
+        gt[4] += t[dpt][pp][1].x; gt[5] += t[dpt][pp][1].y; gt[6] += t[dpt][pp][1].z; gt[7] += t[dpt][pp][1].w;
+        up[0] += t[dpt][pp][2].x; up[1] += t[dpt][pp][2].y; up[2] += t[dpt][pp][2].z; up[3] += t[dpt][pp][2].w;
+        up[4] += t[dpt][pp][3].x; up[5] += t[dpt][pp][3].y; up[6] += t[dpt][pp][3].z; up[7] += t[dpt][pp][3].w;
+      }
+      if (on) {
+        unsigned o[4];
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(silu_mul(gt[e], up[e]), silu_mul(gt[e + 1], up[e + 1]));
+          o[e >> 1] = *reinterpret_cast<const unsigned *>(&v2);
+        }
+        uint8_t *slot = ring + (size_t)s * PCfg<NPAD>::kStageBytes + kWBytes;
+        *reinterpret_cast<uint4 *>(slot + r * 128 + ((c8 ^ (r & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads the tile through the async proxy
+      __syncwarp();
+      if (w.lane == 0) mbar_arrive(full_bar0 + 8u * s);
+      load(t[dpt], i + 4 * DEPTH);                               // this buffer's next stage
+    }
+  }
+}
 
 // Finish phase of GEMM p (QKV, gate/up, output head): units of (tile, block of up to 8 token rows)
 // round-robin over the CTAs, two at a time (one per 128-thread group); the pieces of a tile (at most
@@ -946,6 +1047,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   volatile int *abort_flag = reinterpret_cast<volatile int *>(ctl + 1);
   int *first_item_sh = reinterpret_cast<int *>(ctl + 148);               // [4] this CTA's first attention item
   int *qkv_geom_sh = reinterpret_cast<int *>(ctl + 152);                 // [7] piece geometry of the QKV projection
+  // [16] phase << 16 | parity << 8 | slot of the first stage of built down projection number (layer & 15): the
+  // weight producer is at most one ring (8 stages) ahead, so never 16 such phases
+  volatile unsigned *ring_pos_sh = reinterpret_cast<volatile unsigned *>(ctl + 928);
+  int *bgeom_sh = reinterpret_cast<int *>(ctl + 944);                    // [4] geometry of the built down projection
+  static_assert((2 * Cfg::kStages + 6) * 8 + (944 + 4) * 4 <= kCtrlBytes - 128, "control area overflow");
   volatile int *wait_ok = reinterpret_cast<volatile int *>(ctl + 4);   // [2]
   float *red = reinterpret_cast<float *>(ctl + 8);                      // [8]
   PageCache *pcache = reinterpret_cast<PageCache *>(ctl + 16);          // 130 words
@@ -972,6 +1078,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); mbar_init(ready_bar(b), 1); }
     *abort_flag = 0;
+    for (int i = 0; i < 16; ++i) ring_pos_sh[i] = 0xFFFFFFFFu;
     for (int i = 0; i < 16; ++i) dbg_cy[i] = 0;
     pcache->tag_item = -1;
     pcache->tag_tile = -1;
@@ -1005,6 +1112,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         const Gemm g = make_gemm(a, p);
         SegIter it = seg_begin(g, G, c);
         Seg sg;
+        if (built_down(a, p)) ring_pos_sh[(p >> 2) & 15] = (unsigned)s | (par << 8) | ((unsigned)p << 16);   // where the builders' tiles go
         while (ok && seg_next(g, it, sg)) {
           const Tile ti = tile_of(g, sg.tile);
           const bool second = (g.mode == MODE_SWIGLU) || (ti.row0 + kTcBoxRows < g.seg_n[ti.seg]);
@@ -1049,12 +1157,15 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         bool have = seg_next(g, it, sg);
         // the operand of phase p is complete once the workers have passed the barrier before it
         if (!mbar_wait(ready_bar(p & 1), (uint32_t)((p >> 1) & 1), abort_flag)) { ok = false; break; }
+        const bool built = built_down(a, p);
         while (ok && have) {
           for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
             if (s % WGS == 0 && !mbar_wait(empty_bar(s / WGS), par, abort_flag)) { ok = false; break; }
             const uint32_t dst = smem_u32(ring) + (uint32_t)(s * Cfg::kStageBytes) + kWBytes;
-            mbar_expect_tx(full_bar(s), a_bytes);
-            tma_load_2d(dst, g.amap, kb * kTcBlockK, 0, full_bar(s));
+            if (!built) {                                // built down projection: the workers fill the tile and arrive
+              mbar_expect_tx(full_bar(s), a_bytes);
+              tma_load_2d(dst, g.amap, kb * kTcBlockK, 0, full_bar(s));
+            }
             if (++s == STAGES) { s = 0; par ^= 1u; }
           }
           have = seg_next(g, it, sg);
@@ -1138,6 +1249,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       qkv_geom_sh[0] = (gq.seg_n[0] + kTcBlockM - 1) / kTcBlockM;
       qkv_geom_sh[1] = qkv_geom_sh[0] + (gq.seg_n[1] + kTcBlockM - 1) / kTcBlockM;
       qkv_geom_sh[2] = geo.parts; qkv_geom_sh[3] = geo.pieces_max; qkv_geom_sh[4] = geo.U; qkv_geom_sh[5] = geo.Gp; qkv_geom_sh[6] = gq.KB;
+      const Gemm gdn = make_gemm(a, 3);
+      const SplitGeom geo_gu = split_geom(make_gemm(a, 2), G);
+      const SegIter itd = seg_begin(gdn, G, c);
+      bgeom_sh[0] = itd.kb; bgeom_sh[1] = itd.left; bgeom_sh[2] = geo_gu.parts; bgeom_sh[3] = geo_gu.pieces_max;
     }
     // One step loop, one call site per phase body: the whole per-layer program has to stay resident in
     // the instruction cache (every phase runs once per layer, so code that does not fit is fetched
@@ -1171,8 +1286,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
             break;
           case 4: kind = K_EPI; gp = p + 1; break;
           case 5: kind = K_NORM; gp = p + 1; ready = p + 2; break;
-          case 6: kind = K_EPI; gp = p + 2; break;
-          case 7: kind = K_FIN; gp = p + 2; ready = p + 3; break;
+          case 6: kind = K_EPI; gp = p + 2; if (a.fuse_gu) ready = p + 3; break;
+          case 7:                                            // folded into the down projection in passes with few rows
+            if (a.fuse_gu) { kind = K_NONE; barrier = false; }
+            else { kind = K_FIN; gp = p + 2; ready = p + 3; }
+            break;
           case 8: kind = K_EPI; gp = p + 3; barrier = (l + 1 < a.n_run || a.L > 0); break;
           default:
             kind = (l + 1 < a.n_run || a.L > 0) ? K_NORM : K_NONE; gp = p + 3; ready = p + 4;
@@ -1181,7 +1299,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         }
       }
       switch (kind) {
-        case K_EPI: if (is_epi) gemm_epilogue<NPAD>(a, w, gp); break;
+        case K_EPI:
+          if (built_down(a, gp)) {
+            if (a.gu_pieces_max <= 2) build_act_stages<NPAD, 2, 2>(a, w, gp, ring, full_bar(0), empty_bar(0), ring_pos_sh, bgeom_sh);
+            else build_act_stages<NPAD, 4, 1>(a, w, gp, ring, full_bar(0), empty_bar(0), ring_pos_sh, bgeom_sh);
+          }
+          if (is_epi) gemm_epilogue<NPAD>(a, w, gp);
+          break;
         case K_FIN: gemm_finish<NPAD>(a, w, gp); break;
         case K_ATTN_A:
           attn_tiles_phase<NPAD, HD>(a, layers_sh[l], scratch, pcache, wt, dbg_cy, first_item_sh, qkv_geom_sh, row_pg_sh, rope_cos_sh, rope_sin_sh);
@@ -1194,7 +1318,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
           const Gemm pend = make_gemm(a, first ? 0 : gp);
           const __nv_bfloat16 *gain = first ? a.layers[0].attn_norm
                                             : (last ? a.final_norm : (mid ? layers_sh[l].mlp_norm : layers_sh[l + 1].attn_norm));
-          norm_phase<NPAD>(a, last ? a.L : a.R, last ? a.lrow_src : nullptr, first, first ? nullptr : &pend, gain,
+          norm_phase<NPAD>(a, last ? a.L : a.R, last ? a.lrow_src : nullptr, first, first ? nullptr : &pend, pieces_of(a, gp), gain,
                            last ? a.hf : a.h, red, wt);
           break;
         }
@@ -1253,10 +1377,20 @@ int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaS
     long long kb = std::max(args.ff, std::max(args.d, args.nq * args.hd)) / kTcBlockK;
     if (tiles * kb * sm_count >= (1ll << 31)) return HSD_E_UNSUPPORTED;
   }
-  switch (args.hd) {
-    case 128: return launch_hd<128>(args, npad, sm_count, s);
-    case 64: return launch_hd<64>(args, npad, sm_count, s);
-    case 32: return launch_hd<32>(args, npad, sm_count, s);
+  FwdArgs a = args;
+  {  // pieces per gate / up tile (the device's split_geom, for a grid of sm_count CTAs)
+    const int n_tiles = (a.ff + kTcBoxRows - 1) / kTcBoxRows, KB = a.d / kTcBlockK;
+    if (n_tiles * 2 <= sm_count) a.gu_pieces_max = std::min(std::min(4, sm_count / n_tiles), KB);
+    else {
+      const int U = n_tiles * KB, Gp = std::min(sm_count, U), per = U / Gp;
+      a.gu_pieces_max = (KB + per - 1) / per + 1;
+    }
+    if (a.gu_pieces_max > 4) a.fuse_gu = 0;
+  }
+  switch (a.hd) {
+    case 128: return launch_hd<128>(a, npad, sm_count, s);
+    case 64: return launch_hd<64>(a, npad, sm_count, s);
+    case 32: return launch_hd<32>(a, npad, sm_count, s);
     default: return HSD_E_UNSUPPORTED;
   }
 }

@@ -26,6 +26,9 @@ struct FwdArgs {
   int R, L, n_attn, attn_rows, n_splits, keys_per_split;
   int a_box_rows;                  // rows of one activation TMA box (<= the row padding)
   int fuse_qkv;                    // 1: every sequence is one attention item; the item's CTAs finish its q / k / v themselves
+  int fuse_gu;                     // 1: at most 4 rows; the down projection's CTAs build their activation tiles from the gate / up pieces
+  int gu_pieces_max;               // pieces per gate / up tile at most (its split geometry; filled in by the launcher)
+  float *pieces2;                  // split pieces of the down projection while `pieces` still holds gate / up (fuse_gu)
   const int *tokens, *page_table, *row_seq, *row_pos, *lrow_src;
   const int4 *attn_items;          // (first packed row, rows, sequence, position of first row)
   const long long *lrow_dst;

@@ -229,7 +229,7 @@ gemm_tc_kernel(const __grid_constant__ TcGemmArgs args, int n_tiles, int KB, int
             int col = ti.row0 + cc;
             if (col < args.seg_n[0]) {
               float g = staging[cc * (NPAD + 1) + r], up = staging[(cc + kTcBoxRows) * (NPAD + 1) + r];
-              args.out_bf16[(size_t)(args.row0 + r) * args.ldo + col] = __float2bfloat16_rn(g / (1.f + __expf(-g)) * up);
+              args.out_bf16[(size_t)(args.row0 + r) * args.ldo + col] = __float2bfloat16_rn(ptx::silu_mul(g, up));
             }
           }
           asm volatile("bar.sync 1, 128;" ::: "memory");

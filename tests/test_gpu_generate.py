@@ -140,9 +140,11 @@ def test_page_size_does_not_change_the_stream(lib):
 
 
 @pytest.mark.parametrize("name", ["mini3", "mini4long"])
-def test_folded_qkv_finish_gives_the_stream_of_the_separate_phase(lib, name, monkeypatch):
-    """Decode passes fold the QKV finish (piece sum, rotary embedding, cache write) into the attention phase;
-    HSD_NO_FUSE_QKV keeps the separate phase.  Same sums in the same order: the token streams are equal."""
+def test_folded_finish_phases_give_the_stream_of_the_separate_phases(lib, name, monkeypatch):
+    """Decode passes fold the QKV finish (piece sum, rotary embedding, cache write) into the attention phase and,
+    with at most four rows, the gate / up finish (piece sum, SwiGLU) into the down projection, whose CTAs build
+    their activation tiles in shared memory.  HSD_NO_FUSE_QKV / HSD_NO_FUSE_GU keep the separate phases.  Same
+    sums in the same order: all four combinations give the same token stream."""
     wl = inputs.WORKLOADS[name]
     cfg = wl["model"]
     w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
@@ -150,15 +152,17 @@ def test_folded_qkv_finish_gives_the_stream_of_the_separate_phase(lib, name, mon
     prompts = inputs.make_prompts(cfg["vocab"], batch, wl["prompt"], wl["prompt_seed"]).cuda()
     max_seq = wl["prompt"] + wl["n_new"] + sum(wl["T"]) + len(wl["exits"]) + 8
     outs = []
-    for separate in (False, True):
-        if separate:
-            monkeypatch.setenv("HSD_NO_FUSE_QKV", "1")
-        else:
-            monkeypatch.delenv("HSD_NO_FUSE_QKV", raising=False)
+    for keep in ((), ("HSD_NO_FUSE_QKV",), ("HSD_NO_FUSE_GU",), ("HSD_NO_FUSE_QKV", "HSD_NO_FUSE_GU")):
+        for k in ("HSD_NO_FUSE_QKV", "HSD_NO_FUSE_GU"):
+            if k in keep:
+                monkeypatch.setenv(k, "1")
+            else:
+                monkeypatch.delenv(k, raising=False)
         eng = lib.Hsd(cfg, w, wl["exits"], wl["T"], max_batch=batch, max_seq=max_seq, page_size=wl["page"])
         outs.append(eng.generate(prompts, wl["n_new"], 1)[0].cpu())
         eng.close()
-    assert torch.equal(outs[0], outs[1])
+    for o in outs[1:]:
+        assert torch.equal(outs[0], o)
 
 
 def test_mini_bf16_decisions_follow_the_oracle_on_the_same_logits(lib, tmp_path):
