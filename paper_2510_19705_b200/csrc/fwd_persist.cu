@@ -26,7 +26,6 @@ constexpr int kBoxBytes = kTcBoxRows * kTcBlockK * 2;  // 8 KiB TMA box
 constexpr int kScratchBytes = 78 * 1024;               // union: epilogue staging / attention buffers, + rope cache
 constexpr int kCtrlBytes = 4096;                       // barriers, flags, page-id cache, per-row info
 constexpr int kSmemTotal = 232448;
-constexpr int kKeyTile = 32;
 constexpr int kMaxLayersSh = 64;                       // layers whose pointer table fits the control area
 
 enum { MODE_QKV = 0, MODE_ADD = 1, MODE_SWIGLU = 2, MODE_LOGITS = 3 };
@@ -172,13 +171,6 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
-}
-__device__ __forceinline__ float bf(const __nv_bfloat16 v) { return __bfloat162float(v); }
-
-// Debug timeline: CTA 0's first worker thread adds the time to slot 960 + k (only when profiling is on;
-// differences of two slots hit equally often give summed intervals).
-__device__ __forceinline__ void prof_mark(const FwdArgs &a, int wt, int k) {
-  if (a.prof && wt == 0 && blockIdx.x == 0) a.prof[960 + k] += globaltimer_ns();
 }
 
 // Grid-wide barrier of the worker threads.  `epoch` counts barriers; the counter only grows.
@@ -333,11 +325,6 @@ constexpr int kAttnMaxSplits = 20;
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gsrc) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all() {
-  asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
-}
-__device__ __forceinline__ float bf_lo(unsigned w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf_hi(unsigned w) { return __uint_as_float(w & 0xFFFF0000u); }
 
 struct PageCache { int tag_item, tag_tile; int pg[128]; };   // pg[warp * 16 + j]: page of the warp's j-th sub-tile
 
@@ -1035,7 +1022,6 @@ template <int NPAD, int HD>
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __grid_constant__ FwdArgs a) {
   using Cfg = PCfg<NPAD>;
   constexpr int STAGES = Cfg::kStages;
-  constexpr int CH = Cfg::kChunk;
   extern __shared__ uint8_t smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   uint8_t *ring = smem;
@@ -1210,10 +1196,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     // ------------------------------------------------------------ workers (+ epilogue: warps 4..7)
     const int wt = threadIdx.x - 128;              // 0..255
     const bool is_epi = warp < 8;
-    const int q = warp & 3, m = q * 32 + lane;
+    const int q = warp & 3;
     float *staging = reinterpret_cast<float *>(scratch);
     unsigned epoch = 0;
-    int seg_idx = 0;
     bool alive = true;
 
     WorkerCtx w;
