@@ -1,7 +1,11 @@
 """The model abstraction M_i(context) -> next-token distribution (Section 3.1), for the
 early-exit family of Section 5.1: M_i is the first e_i layers of one decoder-only
 transformer followed by the shared final norm and the shared output head (the
-LayerSkip setting, where "the same LM head" serves every layer).
+LayerSkip setting, where "the same LM head" serves every layer).  The other setting of
+Section 5.1 (one trained output head per exit layer, a linear map from the embedding
+dimension to the vocabulary; memory grows with the number of levels) is the optional
+`exit_heads` entry of the weights: level i then uses its own head matrix, and its own
+norm gain if one is given, in place of the shared ones.
 
 The paper uses pretrained checkpoints and does not describe the network; the
 architecture below is the benchmark contract's Llama-style decoder:
@@ -40,7 +44,8 @@ class Transformer:
     """cfg: dict(n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab, dtype,
     rms_eps, rope_theta); weights: dict(embed, final_norm, lm_head, layers=[dict(attn_norm, wq,
     wk, wv, wo, mlp_norm, wg, wu, wd)]) of fp32 arrays (dtype 'fp32') or uint16 bf16 bit
-    patterns (dtype 'bf16'), matrices stored [out_features, in_features]."""
+    patterns (dtype 'bf16'), matrices stored [out_features, in_features].  Optional
+    weights['exit_heads']: list over levels of None (shared head) or dict(lm_head[, final_norm])."""
 
     def __init__(self, cfg, weights, exits, cache_bytes=8 << 30):
         self.cfg, self.w, self.exits = dict(cfg), weights, list(exits)
@@ -62,6 +67,20 @@ class Transformer:
             self._wide[key] = wide
             self._wide_bytes += wide.nbytes
         return wide
+
+    def _head(self, level, name):
+        """The level's own output head / norm gain if it has one (Section 5.1, per-exit heads), else the shared one."""
+        heads = self.w.get("exit_heads")
+        own = heads[level] if heads is not None else None
+        if own is None or own.get(name) is None:
+            return self._mat(None, name)
+        key = (("head", level), name)
+        hit = self._wide.get(key)
+        if hit is None:
+            raw = own[name]
+            hit = bf16_bits_to_f64(raw) if self.bf16 else raw.astype(np.float64)
+            self._wide[key] = hit
+        return hit
 
     def _rnd(self, x):
         return bf16_round(x) if self.bf16 else x
@@ -139,8 +158,8 @@ class Transformer:
             act = self._rnd(gte / (1.0 + np.exp(-gte)) * up)
             x = x + act @ self._mat(l, "wd").T
         xo = x[first_out - start:]
-        hf = self._rnd(self._rmsnorm(xo, self._mat(None, "final_norm")))
-        logits = hf @ self._mat(None, "lm_head").T
+        hf = self._rnd(self._rmsnorm(xo, self._head(level, "final_norm")))
+        logits = hf @ self._head(level, "lm_head").T
         self.last_logits64 = logits
         stored = self._rnd(logits) if self.bf16 else logits.astype(np.float32).astype(np.float64)
         return [stored[j].astype(np.float32) for j in range(stored.shape[0])]

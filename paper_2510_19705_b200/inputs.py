@@ -72,13 +72,32 @@ def make_weights(cfg, seed, device="cpu", std=0.02):
     return w
 
 
+def make_exit_heads(cfg, n_levels, seed, device="cpu", std=0.02, with_norm=True):
+    """One output head per drafting level (Section 5.1, the setting with a trained head per exit layer):
+    list over levels of dict(lm_head [vocab, d] ~ N(0, std^2), final_norm [d] ~ 1 + 0.1 N(0, 1) if with_norm);
+    the last level (the target) keeps the shared head (None).  Stand-in for trained heads: random-init."""
+    dt = torch.float32 if cfg["dtype"] == "fp32" else torch.bfloat16
+    g = _gen(seed, device)
+    d, V = cfg["d_model"], cfg["vocab"]
+    heads = []
+    for _ in range(n_levels - 1):
+        h = dict(lm_head=(torch.randn(V, d, generator=g, device=device, dtype=torch.float32) * std).to(dt))
+        if with_norm:
+            h["final_norm"] = (1.0 + 0.1 * torch.randn(d, generator=g, device=device, dtype=torch.float32)).to(dt)
+        heads.append(h)
+    heads.append(None)
+    return heads
+
+
 def weights_to_numpy(w):
     """fp32 tensors -> float32 arrays; bf16 tensors -> uint16 bit patterns (host copies)."""
     def conv(t):
         t = t.detach().cpu().contiguous()
         return t.view(torch.uint16).numpy() if t.dtype == torch.bfloat16 else t.numpy()
-    out = {k: conv(v) for k, v in w.items() if k != "layers"}
+    out = {k: conv(v) for k, v in w.items() if k not in ("layers", "exit_heads")}
     out["layers"] = [{k: conv(v) for k, v in layer.items()} for layer in w["layers"]]
+    if w.get("exit_heads") is not None:
+        out["exit_heads"] = [None if h is None else {k: conv(v) for k, v in h.items()} for h in w["exit_heads"]]
     return out
 
 

@@ -78,6 +78,32 @@ def test_bf16_model_matches_library_ops_with_the_same_rounding_points():
     assert np.array_equal(stored, bf16_round(got).astype(np.float32))
 
 
+def test_per_exit_heads_replace_the_shared_head_at_their_level_only():
+    """Section 5.1, one trained head per exit layer: level i's logits = own head x RMSNorm(hidden state at e_i, own
+    gain); a level without an own head (here the target) and a head without an own gain use the shared ones."""
+    w, _ = _setup(CFG32)
+    heads = inputs.make_exit_heads(CFG32, 3, seed=21, std=0.2)
+    del heads[1]["final_norm"]                        # level 1: own matrix, shared norm gain
+    w["exit_heads"] = heads
+    m = Transformer(CFG32, inputs.weights_to_numpy(w), exits=(1, 2, 3))
+    toks = inputs.make_prompts(CFG32["vocab"], 1, 12, seed=3)[0].tolist()
+    for level, e in enumerate((1, 2, 3)):
+        own = heads[level] or {}
+        w_level = dict(w, lm_head=own.get("lm_head", w["lm_head"]), final_norm=own.get("final_norm", w["final_norm"]))
+        ref = library_forward(CFG32, w_level, e, toks, bf16=False)
+        shared = library_forward(CFG32, w, e, toks, bf16=False)
+        m.rows_from_scratch(level, toks[:8], toks[8:])
+        got = m.last_logits64
+        assert np.abs(got - ref[7:]).max() < 1e-6 * max(1.0, np.abs(ref).max())
+        if level < 2:
+            assert np.abs(ref - shared).max() > 0.05   # the own head matters
+    # heads equal to the shared one change nothing
+    w["exit_heads"] = [dict(lm_head=w["lm_head"], final_norm=w["final_norm"]), None, None]
+    m2 = Transformer(CFG32, inputs.weights_to_numpy(w), exits=(1, 2, 3))
+    m2.rows_from_scratch(0, toks[:8], toks[8:])
+    assert np.abs(m2.last_logits64 - library_forward(CFG32, w, 1, toks, bf16=False)[7:]).max() < 1e-6
+
+
 def test_bf16_round_is_nearest_even():
     x = torch.randn(4096, dtype=torch.float32) * 3
     x[:4] = torch.tensor([1.00390625, 1.01171875, -1.00390625, 0.0])     # exact ties
