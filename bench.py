@@ -202,6 +202,8 @@ def run_ours(args):
     else:
         T, calib = list(wl["T"]), None
     eng = binding.Hsd(cfg, weights, wl["exits"], T, max_batch=B, max_seq=P + n_new + sum(T) + 16, page_size=wl["page"])
+    if args.exit_heads:                                  # Section 5.1's other setting: one (random-init) head per drafting level
+        eng.set_exit_heads(inputs.make_exit_heads(cfg, len(wl["exits"]), seed=4242, device="cuda"))
 
     def barrier():
         torch.cuda.synchronize()
@@ -270,7 +272,7 @@ def run_ours(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dec_ms_step, 3), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": cfg["dtype"], "data": "synthetic",
         "config": {"workload": args.workload, "batch": B, "prompt_len": P, "n_new": n_new, "exits": list(wl["exits"]),
-                   "T": T, "T_search": calib, "hierarchy_search": hier, "l2": "inputs larger than L2 (weights %.1f GB per target pass)"
+                   "T": T, "T_search": calib, "hierarchy_search": hier, "exit_heads": bool(args.exit_heads), "l2": "inputs larger than L2 (weights %.1f GB per target pass)"
                    % (weight_bytes(cfg, cfg["n_layers"]) / 1e9), "replicas": "independent sequence per GPU"},
         "prefill_ms": round(pre_ms_step, 3), "step_ms_with_prefill": round(step_ms, 3),
         "e2e": {"value": round(aggregate_tokens_per_s(world, B * n_new, e2e_ms), 2), "unit": UNIT, "h2d_bytes_per_step": B * P * 4,
@@ -431,6 +433,8 @@ def main():
     ap.add_argument("--batch", type=int, default=1, help="sequences per GPU (the metric is quoted at 1)")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length (development runs)")
     ap.add_argument("--T", default="", help="fix T (comma separated) instead of calibrating / using the workload's")
+    ap.add_argument("--exit-heads", action="store_true",
+                    help="give every drafting level its own output head and norm gain (not the default config)")
     ap.add_argument("--search-hierarchy", action="store_true",
                     help="choose the exit layers and T by the latency-optimal hierarchy search over all layers (not the default config)")
     args = ap.parse_args()

@@ -156,6 +156,19 @@ size_t hsd_workspace_bytes(const hsd_model_desc *model, const int32_t *exit_laye
 int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_levels, const int32_t *T,
                void *workspace, size_t workspace_bytes, hsd_ctx **out);
 
+/* One output head per level instead of the shared one (Section 5.1: the setting in which every exit
+ * layer has its own trained head, a linear map from the embedding dimension to the vocabulary, so that
+ * memory grows with the number of levels; the shared head of the descriptor is the other setting).
+ * Level i then computes its logits as lm_heads[i] x RMSNorm(hidden state after exit_layers[i]; gain
+ * final_norms[i]).
+ *   final_norms  host [n_levels] of device pointers [d_model] in the model's dtype, or NULL
+ *   lm_heads     host [n_levels] of device pointers [vocab, d_model] row-major in the model's dtype,
+ *                16-byte aligned, or NULL
+ * A NULL array or entry keeps (or restores) the descriptor's shared tensor for that level.  The tensors
+ * are not copied and must outlive the context.  Waits for the context's stream; must not overlap a
+ * generation.  hsd_layer_logits keeps using the shared head.  Errors: INVALID_ARG, CUDA. */
+int hsd_set_exit_heads(hsd_ctx *ctx, const void *const *final_norms, const void *const *lm_heads);
+
 /* Generate n_new tokens per sequence with Algorithm 1 called at idx = K until enough tokens exist
  * (the first n_new are returned).  Sequence b produces exactly the tokens it would produce alone
  * with the same seed (uniforms are keyed by b).

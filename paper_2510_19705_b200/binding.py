@@ -153,6 +153,8 @@ def _declare_engine(lib):
     lib.hsd_generate.argtypes = [vp, vp, i32, i32, i32, u64, vp, vp, c.POINTER(LevelStats), c.POINTER(c.c_double)]
     lib.hsd_set_trace.restype = i32
     lib.hsd_set_trace.argtypes = [vp, c.c_char_p, i32]
+    lib.hsd_set_exit_heads.restype = i32
+    lib.hsd_set_exit_heads.argtypes = [vp, c.POINTER(vp), c.POINTER(vp)]
     lib.hsd_destroy.restype = None
     lib.hsd_destroy.argtypes = [vp]
     lib.hsd_expected_latency.restype = i32
@@ -218,6 +220,22 @@ class Hsd:
         self._ctx = ctx
         self.n_levels = n_levels
         self.workspace_bytes = need
+
+    def set_exit_heads(self, heads):
+        """heads: list over levels of None (shared head) or dict(lm_head[, final_norm]) of CUDA tensors in the
+        model's dtype (hsd_set_exit_heads); None restores the shared head everywhere."""
+        n = self.n_levels
+        norms = (ctypes.c_void_p * n)()
+        mats = (ctypes.c_void_p * n)()
+        for i in range(n):
+            h = heads[i] if heads is not None else None
+            if h is not None:
+                assert h["lm_head"].is_cuda and h["lm_head"].is_contiguous()
+                mats[i] = h["lm_head"].data_ptr()
+                if h.get("final_norm") is not None:
+                    norms[i] = h["final_norm"].data_ptr()
+        self._exit_heads = heads                    # keep the device buffers alive
+        _check(self._lib.hsd_set_exit_heads(self._ctx, norms, mats))
 
     def set_trace(self, path, logit_calls=0):
         _check(self._lib.hsd_set_trace(self._ctx, path.encode() if path else None, logit_calls))

@@ -25,6 +25,7 @@ constexpr int kPrefillRows = 128;
 constexpr uint32_t kTraceMagic = 0x48534454u;
 
 constexpr size_t kTcCtrlBytes = 16384 + 256;    // status word (first 256 bytes) + per-tile counters
+constexpr int kHeadMaps = 17;                   // output-head tensor maps: one per level (<= 16), then the shared head
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 int device_sm_count() {
@@ -129,7 +130,7 @@ Layout make_layout(const hsd_model_desc *m, int n_levels, const int32_t *T) {
   }
   L.tc_scratch = take(kTcCtrlBytes + L.tc_pieces_bytes);
   L.tc_pieces2 = take(L.tc_pieces_bytes);       // second piece buffer (down projection of passes with few rows)
-  L.wmaps_dev = take(((size_t)m->n_layers * 7 + 1) * sizeof(CUtensorMap));
+  L.wmaps_dev = take(((size_t)m->n_layers * 7 + kHeadMaps) * sizeof(CUtensorMap));
   L.layers_dev = take((size_t)m->n_layers * sizeof(FwdLayerDev));
   L.attn_counters = take(16384);
   L.grid_counter = take(256);
@@ -184,7 +185,8 @@ struct hsd_ctx {
   bool no_fuse_qkv = false;                   // debugging aid (HSD_NO_FUSE_QKV): keep the QKV finish phase in every pass
   bool no_fuse_gu = false;                    // debugging aid (HSD_NO_FUSE_GU): keep the gate / up finish phase in every pass
   int sm_count;
-  std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + 1]: wq wk wv wo wg wu wd per layer, then lm_head
+  std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + kHeadMaps]: wq wk wv wo wg wu wd per layer, then the levels' heads, the shared head
+  std::vector<const void *> level_head, level_norm;   // output head and final norm gain of each level (shared unless set)
   CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
   CUtensorMap amaps_rows[4][16];              // the same buffers with a box of exactly 1..16 rows (persistent forward, few rows)
   int *status_host;
@@ -423,13 +425,13 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     // one cooperative launch runs the whole pass
     FwdArgs a;
     a.d = md.d; a.nq = md.nq; a.nkv = md.nkv; a.hd = md.hd; a.ff = md.ff; a.V = md.V;
-    a.n_run = c->exits[level]; a.lm_map = md.n_layers * 7; a.max_seq = md.max_seq; a.page = md.page;
+    a.n_run = c->exits[level]; a.lm_map = md.n_layers * 7 + level; a.max_seq = md.max_seq; a.page = md.page;
     a.page_shift = 0;
     while ((1 << a.page_shift) < md.page) ++a.page_shift;
     a.pages_per_seq = md.pages_per_seq; a.eps = md.eps;
     a.wmaps = c->dev<CUtensorMap>(L.wmaps_dev);
     a.layers = c->dev<FwdLayerDev>(L.layers_dev);
-    a.embed = (const __nv_bfloat16 *)c->embed; a.final_norm = (const __nv_bfloat16 *)c->final_norm;
+    a.embed = (const __nv_bfloat16 *)c->embed; a.final_norm = (const __nv_bfloat16 *)c->level_norm[level];
     a.cos_tab = c->dev<float>(L.cos_tab); a.sin_tab = c->dev<float>(L.sin_tab);
     a.R = R; a.L = n_logit; a.n_attn = n_attn; a.attn_rows = arows; a.n_splits = n_splits; a.keys_per_split = keys_per_split;
     a.tokens = c->dev<int>(L.tokens); a.page_table = c->dev<int>(L.page_table);
@@ -509,9 +511,9 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   }
   if (n_logit > 0) {
     void *hf = c->dev<void>(L.hf);
-    HSD_TRY(launch_rmsnorm(md, x, c->final_norm, rb.lrow_src, n_logit, hf, s));
-    GemmSegs lm_segs = {{c->lm_head, nullptr, nullptr}, {md.V, 0, 0}, 1};
-    HSD_TRY(gemm(c, 3, hf, n_logit, md.d, lm_segs, md.n_layers * 7, GEMM_STORE_T_SCATTER, nullptr, c->ws + L.logits[level],
+    HSD_TRY(launch_rmsnorm(md, x, c->level_norm[level], rb.lrow_src, n_logit, hf, s));
+    GemmSegs lm_segs = {{c->level_head[level], nullptr, nullptr}, {md.V, 0, 0}, 1};
+    HSD_TRY(gemm(c, 3, hf, n_logit, md.d, lm_segs, md.n_layers * 7 + level, GEMM_STORE_T_SCATTER, nullptr, c->ws + L.logits[level],
                  rb.lrow_dst));
   }
   if (tp) cudaEventRecord(tp->b, s);
@@ -741,6 +743,8 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
   c->lay = lay;
   c->ws = (char *)workspace;
   c->embed = model->embed; c->final_norm = model->final_norm; c->lm_head = model->lm_head;
+  c->level_head.assign(n_levels, model->lm_head);
+  c->level_norm.assign(n_levels, model->final_norm);
   c->lw.assign(model->layer_weights, model->layer_weights + (size_t)model->n_layers * 9);
   c->ring_host = nullptr; c->n_acc_host = nullptr; c->page_table_host = nullptr; c->status_host = nullptr;
   c->use_tc = false; c->use_persist = false; c->sm_count = 148;
@@ -777,14 +781,14 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
   if (c->use_tc) {
     const ModelDims &md = c->md;
     int st = HSD_OK;
-    c->wmaps.resize((size_t)md.n_layers * 7 + 1);
+    c->wmaps.resize((size_t)md.n_layers * 7 + kHeadMaps);
     const long long rows7[7] = {(long long)md.nq * md.hd, (long long)md.nkv * md.hd, (long long)md.nkv * md.hd, md.d, md.ff, md.ff, md.d};
     const long long cols7[7] = {md.d, md.d, md.d, (long long)md.nq * md.hd, md.d, md.d, md.ff};
     const int widx[7] = {1, 2, 3, 4, 6, 7, 8};
     for (int l = 0; l < md.n_layers && !st; ++l)
       for (int k = 0; k < 7 && !st; ++k)
         st = tc_make_map(&c->wmaps[(size_t)l * 7 + k], c->lw[(size_t)l * 9 + widx[k]], rows7[k], cols7[k], kTcBoxRows);
-    if (!st) st = tc_make_map(&c->wmaps[(size_t)md.n_layers * 7], c->lm_head, md.V, md.d, kTcBoxRows);
+    for (int i = 0; i < kHeadMaps && !st; ++i) st = tc_make_map(&c->wmaps[(size_t)md.n_layers * 7 + i], c->lm_head, md.V, md.d, kTcBoxRows);
     const size_t abuf_off[4] = {lay.h, lay.att, lay.act, lay.hf};
     const long long acols[4] = {md.d, (long long)md.nq * md.hd, md.ff, md.d};
     int max_logit_rows = 0;
@@ -958,12 +962,32 @@ int hsd_layer_logits(hsd_ctx *c, const int32_t *token_ids, int n_tokens, const i
       // buffer of the generation path's final norm holds the few logit rows of a verification only)
       HSD_TRY(launch_rmsnorm(md, x, c->final_norm, rb.lrow_src, R, h, s));
       GemmSegs lm_segs = {{c->lm_head, nullptr, nullptr}, {md.V, 0, 0}, 1};
-      HSD_TRY(gemm(c, 0, h, R, md.d, lm_segs, md.n_layers * 7, GEMM_STORE_T_SCATTER, nullptr,
+      HSD_TRY(gemm(c, 0, h, R, md.d, lm_segs, md.n_layers * 7 + kHeadMaps - 1, GEMM_STORE_T_SCATTER, nullptr,
                    (char *)out_logits + (size_t)next * R * md.V * es, rb.lrow_dst));
       ++next;
     }
   }
   return sync_stream(c);
+}
+
+int hsd_set_exit_heads(hsd_ctx *c, const void *const *final_norms, const void *const *lm_heads) {
+  if (!c) return HSD_E_INVALID_ARG;
+  const ModelDims &md = c->md;
+  int st = sync_stream(c);                      // no pass of this context may be in flight
+  if (st) return st;
+  for (int i = 0; i < c->n_levels; ++i) {
+    c->level_norm[i] = (final_norms && final_norms[i]) ? final_norms[i] : c->final_norm;
+    c->level_head[i] = (lm_heads && lm_heads[i]) ? lm_heads[i] : c->lm_head;
+    if (((uintptr_t)c->level_head[i] & 15) != 0) return HSD_E_INVALID_ARG;
+  }
+  if (!c->use_tc) return HSD_OK;
+  for (int i = 0; i < c->n_levels && !st; ++i)
+    st = tc_make_map(&c->wmaps[(size_t)md.n_layers * 7 + i], c->level_head[i], md.V, md.d, kTcBoxRows);
+  if (!st && cudaMemcpy(c->ws + c->lay.wmaps_dev + (size_t)md.n_layers * 7 * sizeof(CUtensorMap),
+                        &c->wmaps[(size_t)md.n_layers * 7], (size_t)c->n_levels * sizeof(CUtensorMap),
+                        cudaMemcpyHostToDevice) != cudaSuccess)
+    st = HSD_E_CUDA;
+  return st;
 }
 
 int hsd_set_trace(hsd_ctx *c, const char *path, int logit_calls) {

@@ -170,6 +170,10 @@ def test_mini_bf16_decisions_follow_the_oracle_on_the_same_logits(lib, tmp_path)
     library's own stored logits, the oracle's decision arithmetic must reproduce every token and accept
     count; the logits themselves must match the oracle's forward within 2e-2."""
     wl, cfg, eng, om, prompts, T = _setup("mini3", lib)
+    _bf16_trace_check(lib, wl, eng, om, prompts, tmp_path)
+
+
+def _bf16_trace_check(lib, wl, eng, om, prompts, tmp_path):
     path = str(tmp_path / "trace.bin")
     eng.set_trace(path, logit_calls=10 ** 6)
     toks, stats, _ = eng.generate(prompts.cuda(), wl["n_new"], 0)
@@ -215,3 +219,38 @@ def test_mini_bf16_decisions_follow_the_oracle_on_the_same_logits(lib, tmp_path)
     # the emitted stream is what the log says
     final = _context_of(recs, None, prompt)
     assert final[len(prompt):len(prompt) + wl["n_new"]] == toks[0].cpu().tolist()
+
+
+def _with_exit_heads(name, lib, with_norm=True):
+    wl, cfg, eng, om, prompts, T = _setup(name, lib)
+    heads = inputs.make_exit_heads(cfg, len(wl["exits"]), seed=77, with_norm=with_norm)
+    eng.set_exit_heads([None if h is None else {k: v.cuda() for k, v in h.items()} for h in heads])
+    w_cpu = inputs.make_weights(cfg, wl["weight_seed"])
+    w_cpu["exit_heads"] = heads
+    om = Transformer(cfg, inputs.weights_to_numpy(w_cpu), wl["exits"])
+    return wl, cfg, eng, om, prompts, T
+
+
+def test_per_exit_heads_fp32_streams_match_oracle_bit_exact(lib):
+    """Section 5.1, one head per exit layer (hsd_set_exit_heads): every drafting level has its own head matrix and
+    norm gain; the stream still equals the oracle's, and it differs from the shared-head stream."""
+    wl, cfg, eng, om, prompts, T = _with_exit_heads("tiny3", lib)
+    p_gpu = prompts.cuda()
+    for seed in range(3):
+        toks, stats, _ = eng.generate(p_gpu, wl["n_new"], seed)
+        want, run = _oracle_run(om, T, prompts[0].tolist(), wl["n_new"], seed)
+        assert np.array_equal(toks[0].cpu().numpy(), want), seed
+        _check_stats(stats, run)
+    with_heads = [dict(s) for s in stats]
+    eng.set_exit_heads(None)                       # back to the shared head: the plain model's stream and counters
+    wl2, _, _, om2, _, _ = _setup("tiny3", lib)
+    toks, stats, _ = eng.generate(p_gpu, wl["n_new"], 2)
+    want, run = _oracle_run(om2, T, prompts[0].tolist(), wl["n_new"], 2)
+    assert np.array_equal(toks[0].cpu().numpy(), want)
+    assert [s["accepted"] for s in stats] != [s["accepted"] for s in with_heads]
+
+
+def test_per_exit_heads_bf16_decisions_and_logits(lib, tmp_path):
+    """The same on the tensor-core path (persistent forward: the level's own head map and norm gain)."""
+    wl, cfg, eng, om, prompts, T = _with_exit_heads("mini3", lib)
+    _bf16_trace_check(lib, wl, eng, om, prompts, tmp_path)
