@@ -286,9 +286,36 @@ def run_ours(args):
                      "traffic": traffic, "ms_per_launch": round(tgt_ms, 4), "bytes_per_launch": int(tgt_bytes)},
         "levels": levels,
     }
+    if args.ablation and world == 1 and K >= 1:
+        line["config"]["ablation"] = ablation_table(binding, eng, prompts, n_new, args.steps, agg, dec_ms, T)
     if not args.no_cpu_baseline and world == 1:
         line["cpu_baseline"] = cpu_baseline(args.workload, T, weights)
     print(json.dumps(line))
+
+
+def ablation_table(binding, eng, prompts, n_new, steps, real_stats, real_ms, T):
+    """The paper's check of its two assumptions (appendix "Examining the assumptions of HSD"): latency per token with
+    real or IID-coin acceptance (coin probability = the measured rate of each level), and with the measured time
+    or a fixed artificial cost per forward (= the level's mean measured forward time, so it leaves out the sampling
+    kernels and the host round trip).  ms per generated token (whole top-level rounds)."""
+    def per_token(stats, ms, costs):
+        toks = max(1, stats[-1]["emitted"])
+        return ms / toks, sum(s["forwards"] * c for s, c in zip(stats, costs)) / toks
+    costs = [s["ms"] / max(1, s["forwards"]) for s in real_stats]
+    alphas = [s["accepted"] / max(1, s["tested"]) for s in real_stats[1:]]
+    eng.set_iid_acceptance(alphas)
+    iid_stats, iid_ms = None, 0.0
+    for i in range(steps):
+        _, st, (_, t_dec) = eng.generate(prompts, n_new, i)
+        iid_ms += t_dec
+        iid_stats = st if iid_stats is None else [{k: a[k] + b[k] for k in a} for a, b in zip(iid_stats, st)]
+    eng.set_iid_acceptance(None)
+    rr, ra = per_token(real_stats, real_ms, costs)
+    ir, ia = per_token(iid_stats, iid_ms, costs)
+    return {"ms_per_token": {"real_acceptance_real_cost": round(rr, 4), "iid_acceptance_real_cost": round(ir, 4),
+                             "real_acceptance_artificial_cost": round(ra, 4), "iid_acceptance_artificial_cost": round(ia, 4)},
+            "theorem_3_2_ms_per_token": round(binding.hsd_expected_latency(costs, alphas, T), 4),
+            "alphas": [round(a, 4) for a in alphas], "costs_ms": [round(c, 4) for c in costs]}
 
 
 def run_accept(args):
@@ -433,6 +460,8 @@ def main():
     ap.add_argument("--batch", type=int, default=1, help="sequences per GPU (the metric is quoted at 1)")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length (development runs)")
     ap.add_argument("--T", default="", help="fix T (comma separated) instead of calibrating / using the workload's")
+    ap.add_argument("--ablation", action="store_true",
+                    help="add the four-way latency table (real / IID-coin acceptance x measured / artificial cost)")
     ap.add_argument("--exit-heads", action="store_true",
                     help="give every drafting level its own output head and norm gain (not the default config)")
     ap.add_argument("--search-hierarchy", action="store_true",

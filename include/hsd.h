@@ -169,6 +169,16 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
  * generation.  hsd_layer_logits keeps using the shared head.  Errors: INVALID_ARG, CUDA. */
 int hsd_set_exit_heads(hsd_ctx *ctx, const void *const *final_norms, const void *const *lm_heads);
 
+/* Ablation of the appendix "Examining the assumptions of HSD": the verification rule of Algorithm 2 is
+ * replaced by a biased coin per drafted token.  Level i+1 then accepts a draft iff the 24-bit uniform of that
+ * accept test is below round(alphas[i] * 2^24) (the same counter-addressed uniform the real test uses; logits
+ * play no part in the test).  The token drawn after the last accepted draft is still Algorithm 2's (residual of
+ * the first rejected position, or the target row after t acceptances), so the output is no longer distributed as
+ * the target's: a measurement mode, not a decoding mode.  The other half of that ablation, a fixed artificial
+ * cost per forward, needs no kernel: it is the sum over levels of hsd_level_stats.forwards times a cost.
+ *   alphas host [n_levels - 1], each in [0, 1]; NULL restores the real rule.  Errors: INVALID_ARG. */
+int hsd_set_iid_acceptance(hsd_ctx *ctx, const double *alphas);
+
 /* Generate n_new tokens per sequence with Algorithm 1 called at idx = K until enough tokens exist
  * (the first n_new are returned).  Sequence b produces exactly the tokens it would produce alone
  * with the same seed (uniforms are keyed by b).

@@ -58,6 +58,27 @@ class SpecDecisions:
         return sampling.residual_sample(p_row, q_row, U)
 
 
+class CoinDecisions(SpecDecisions):
+    """The ablation of the appendix "Examining the assumptions of HSD": Algorithm 2's accept test is replaced by
+    a biased coin per drafted token, level i+1 accepting with probability alphas[i].  The coin is the accept
+    test's own uniform compared with round(alpha * 2^24); drafting and the final draw are unchanged."""
+
+    def __init__(self, seed, alphas, seq=0, log=None):
+        super().__init__(seed, seq, log)
+        self.thr = [int(a * 16777216.0 + 0.5) for a in alphas]
+
+    def accept(self, p_row, q_row, x, j, serial, level):
+        U = philox.uniform24(self.seed, j, serial, level, philox.PURPOSE_ACCEPT, self.seq)
+        return U < self.thr[level - 1]
+
+
+def artificial_latency(stats, costs, n_tokens):
+    """The same ablation's fixed artificial cost: every forward of level i costs costs[i] (level 0 runs one
+    forward per drafted token, a verifier one per call); total cost per generated token."""
+    total = stats[0].rows * costs[0] + sum(st.calls * c for st, c in zip(stats[1:], costs[1:]))
+    return total / n_tokens
+
+
 class HSD:
     """One sequence's run of Algorithm 1 over ``model`` with parameters ``T``.
 

@@ -153,6 +153,8 @@ def _declare_engine(lib):
     lib.hsd_generate.argtypes = [vp, vp, i32, i32, i32, u64, vp, vp, c.POINTER(LevelStats), c.POINTER(c.c_double)]
     lib.hsd_set_trace.restype = i32
     lib.hsd_set_trace.argtypes = [vp, c.c_char_p, i32]
+    lib.hsd_set_iid_acceptance.restype = i32
+    lib.hsd_set_iid_acceptance.argtypes = [vp, c.POINTER(c.c_double)]
     lib.hsd_set_exit_heads.restype = i32
     lib.hsd_set_exit_heads.argtypes = [vp, c.POINTER(vp), c.POINTER(vp)]
     lib.hsd_destroy.restype = None
@@ -236,6 +238,15 @@ class Hsd:
                     norms[i] = h["final_norm"].data_ptr()
         self._exit_heads = heads                    # keep the device buffers alive
         _check(self._lib.hsd_set_exit_heads(self._ctx, norms, mats))
+
+    def set_iid_acceptance(self, alphas):
+        """Ablation mode (hsd_set_iid_acceptance): alphas[i] = coin probability of level i+1's accept tests; None
+        restores Algorithm 2's rule."""
+        if alphas is None:
+            _check(self._lib.hsd_set_iid_acceptance(self._ctx, None))
+        else:
+            assert len(alphas) == self.n_levels - 1
+            _check(self._lib.hsd_set_iid_acceptance(self._ctx, (ctypes.c_double * max(1, len(alphas)))(*alphas)))
 
     def set_trace(self, path, logit_calls=0):
         _check(self._lib.hsd_set_trace(self._ctx, path.encode() if path else None, logit_calls))

@@ -187,6 +187,7 @@ struct hsd_ctx {
   int sm_count;
   std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + kHeadMaps]: wq wk wv wo wg wu wd per layer, then the levels' heads, the shared head
   std::vector<const void *> level_head, level_norm;   // output head and final norm gain of each level (shared unless set)
+  std::vector<uint32_t> coin24;               // per level: kNoCoin, or the IID acceptance probability x 2^24 (ablation)
   CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
   CUtensorMap amaps_rows[4][16];              // the same buffers with a box of exactly 1..16 rows (persistent forward, few rows)
   int *status_host;
@@ -636,7 +637,7 @@ int run_verify(hsd_ctx *c, int level, const std::vector<int> &act, const std::ve
   for (size_t i = 0; i < drafts.size(); ++i) HSD_TRY(fetch_tokens(c, act[i], ctx[act[i]], c->buf_len[act[i]] - ctx[act[i]], drafts[i]));
   HSD_TRY(launch_verify(c->ws + L.logits[level], c->ws + L.logits[level - 1], c->dev<int>(L.tokens), c->md.dtype, c->md.V,
                         (int)act.size(), t_max, (const VerifySeq *)devp, 0, 0, 0, c->ws + L.vscratch, c->seed, nullptr,
-                        c->dev<int>(L.n_acc), 1, c->stream));
+                        c->dev<int>(L.n_acc), 1, c->stream, c->coin24[level]));
   HSD_CUDA_OK(cudaMemcpyAsync(c->n_acc_host, c->dev<int>(L.n_acc), act.size() * 4, cudaMemcpyDeviceToHost, c->stream));
   HSD_TRY(sync_stream(c));
   hsd_level_stats &st = c->stats[level];
@@ -745,6 +746,7 @@ int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_le
   c->embed = model->embed; c->final_norm = model->final_norm; c->lm_head = model->lm_head;
   c->level_head.assign(n_levels, model->lm_head);
   c->level_norm.assign(n_levels, model->final_norm);
+  c->coin24.assign(n_levels, kNoCoin);
   c->lw.assign(model->layer_weights, model->layer_weights + (size_t)model->n_layers * 9);
   c->ring_host = nullptr; c->n_acc_host = nullptr; c->page_table_host = nullptr; c->status_host = nullptr;
   c->use_tc = false; c->use_persist = false; c->sm_count = 148;
@@ -988,6 +990,16 @@ int hsd_set_exit_heads(hsd_ctx *c, const void *const *final_norms, const void *c
                         cudaMemcpyHostToDevice) != cudaSuccess)
     st = HSD_E_CUDA;
   return st;
+}
+
+int hsd_set_iid_acceptance(hsd_ctx *c, const double *alphas) {
+  if (!c) return HSD_E_INVALID_ARG;
+  if (alphas)
+    for (int i = 0; i + 1 < c->n_levels; ++i)
+      if (!(alphas[i] >= 0.0 && alphas[i] <= 1.0)) return HSD_E_INVALID_ARG;
+  for (int i = 1; i < c->n_levels; ++i)
+    c->coin24[i] = alphas ? (uint32_t)(alphas[i - 1] * 16777216.0 + 0.5) : kNoCoin;
+  return HSD_OK;
 }
 
 int hsd_set_trace(hsd_ctx *c, const char *path, int logit_calls) {

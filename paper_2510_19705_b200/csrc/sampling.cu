@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(kSampleThreads)
 decide_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, int32_t *__restrict__ tokens, int V,
               int t_max, const VerifySeq *__restrict__ desc, int regular_t, u32 regular_serial, u32 regular_level,
               const RowStat *__restrict__ stats, u64 seed, int32_t *__restrict__ out_tokens /*[B, t_max+1] or null*/,
-              int32_t *__restrict__ out_n /*[B]*/, int write_in_place) {
+              int32_t *__restrict__ out_n /*[B]*/, int write_in_place, u32 coin24) {
   __shared__ u64 sh64[34];
   __shared__ int sh_first_reject;
   int b = blockIdx.x;
@@ -194,6 +194,7 @@ decide_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, in
     u64 Pq = fixed_prob(sq.Ex, prob_scale(sq.S));
     u32 U = uniform24(seed, j, d.serial, d.level, PURPOSE_ACCEPT, d.seq);
     bool ok = (((u64)U * Pq) >> 24) < Pp;                 // u < p(x) / q(x)
+    if (coin24 != kNoCoin) ok = U < coin24;               // ablation: IID acceptance with a fixed probability
     if (!ok) atomicMin(&sh_first_reject, j);
   }
   __syncthreads();
@@ -267,7 +268,7 @@ int launch_draft_sample(const void *logits, int dtype, int V, const SampleRow *d
 template <typename T>
 static int launch_verify_t(const void *p, const void *q, int32_t *tokens, int V, int batch, int t_max,
                            const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch,
-                           u64 seed, int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s) {
+                           u64 seed, int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s, u32 coin24) {
   RowStat *stats = (RowStat *)scratch;
   dim3 grid(2 * t_max + 1, batch);
   constexpr int VN = StatVec<T>::N;
@@ -280,19 +281,19 @@ static int launch_verify_t(const void *p, const void *q, int32_t *tokens, int V,
   if (cudaGetLastError() != cudaSuccess) return HSD_E_CUDA;
   decide_kernel<T><<<batch, kSampleThreads, 0, s>>>((const T *)p, (const T *)q, tokens, V, t_max, desc, regular_t,
                                                    regular_serial, regular_level, stats, seed, out_tokens, out_n,
-                                                   write_in_place);
+                                                   write_in_place, coin24);
   hsd_count_launches(2);
   return hsd_launch_status();
 }
 
 int launch_verify(const void *p, const void *q, int32_t *tokens, int dtype, int V, int batch, int t_max,
                   const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch, u64 seed,
-                  int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s) {
+                  int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s, u32 coin24) {
   if (batch == 0) return HSD_OK;
   return dtype == HSD_BF16 ? launch_verify_t<__nv_bfloat16>(p, q, tokens, V, batch, t_max, desc, regular_t, regular_serial,
-                                                            regular_level, scratch, seed, out_tokens, out_n, write_in_place, s)
+                                                            regular_level, scratch, seed, out_tokens, out_n, write_in_place, s, coin24)
                            : launch_verify_t<float>(p, q, tokens, V, batch, t_max, desc, regular_t, regular_serial,
-                                                    regular_level, scratch, seed, out_tokens, out_n, write_in_place, s);
+                                                    regular_level, scratch, seed, out_tokens, out_n, write_in_place, s, coin24);
 }
 
 // ------------------------------------------------------------------------------ static scratch

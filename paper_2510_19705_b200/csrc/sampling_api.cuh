@@ -34,8 +34,11 @@ size_t verify_scratch_bytes(int batch, int t_max);
 int launch_draft_sample(const void *logits, int dtype, int V, const SampleRow *desc, int n_rows, int regular_rows,
                         u32 regular_serial, u64 seed, int32_t *out, cudaStream_t s);
 
+// coin24 != kNoCoin: the ablation of Appendix "Examining the assumptions": every accept test becomes a biased
+// coin, accepted iff the test's own 24-bit uniform is below coin24 (= acceptance probability x 2^24).
+constexpr u32 kNoCoin = 0xFFFFFFFFu;
 int launch_verify(const void *p, const void *q, int32_t *tokens, int dtype, int V, int batch, int t_max,
                   const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch, u64 seed,
-                  int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s);
+                  int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s, u32 coin24 = kNoCoin);
 
 }  // namespace hsd

@@ -6,7 +6,7 @@ import pytest
 import torch
 
 from oracle import philox, sampling
-from oracle.hsd import HSD, SpecDecisions
+from oracle.hsd import HSD, CoinDecisions, SpecDecisions
 from oracle.transformer import Transformer
 from paper_2510_19705_b200 import inputs
 
@@ -254,3 +254,26 @@ def test_per_exit_heads_bf16_decisions_and_logits(lib, tmp_path):
     """The same on the tensor-core path (persistent forward: the level's own head map and norm gain)."""
     wl, cfg, eng, om, prompts, T = _with_exit_heads("mini3", lib)
     _bf16_trace_check(lib, wl, eng, om, prompts, tmp_path)
+
+
+def test_iid_coin_acceptance_streams_match_oracle(lib):
+    """Ablation mode (hsd_set_iid_acceptance): accept tests are biased coins; stream and counters equal the
+    oracle's run with the same coins, the observed rates are the coins' and not the model's."""
+    wl, cfg, eng, om, prompts, T = _setup("tiny3", lib)
+    alphas = (0.35, 0.8)
+    eng.set_iid_acceptance(list(alphas))
+    p_gpu = prompts.cuda()
+    for seed in range(3):
+        toks, stats, _ = eng.generate(p_gpu, wl["n_new"], seed)
+        om.reset()
+        run = HSD(om, T, CoinDecisions(seed, alphas))
+        want = np.asarray(run.generate(prompts[0].tolist(), wl["n_new"]), dtype=np.int32)
+        assert np.array_equal(toks[0].cpu().numpy(), want), seed
+        _check_stats(stats, run)
+    eng.set_iid_acceptance([1.0, 1.0])
+    toks, stats, _ = eng.generate(p_gpu, wl["n_new"], 0)
+    assert all(s["accepted"] == s["drafted"] for s in stats[1:])      # every draft accepted
+    eng.set_iid_acceptance(None)                                      # back to Algorithm 2's rule
+    toks, stats, _ = eng.generate(p_gpu, wl["n_new"], 0)
+    want, run = _oracle_run(om, T, prompts[0].tolist(), wl["n_new"], 0)
+    assert np.array_equal(toks[0].cpu().numpy(), want)

@@ -251,3 +251,63 @@ def test_stats_and_trace_bookkeeping():
     # serials count calls per level from zero
     for lvl in range(3):
         assert [t[1] for t in run.trace if t[0] == lvl] == list(range(run.stats[lvl].calls))
+
+
+class FlatModel:
+    """Three context-free levels over 5 tokens (stored logits)."""
+    n_levels = 3
+    tab = np.log(np.array([[.3, .3, .2, .1, .1], [.25, .35, .2, .1, .1], [.2, .4, .2, .1, .1]])).astype(np.float32)
+
+    def rows(self, level, context, draft_tokens):
+        return [self.tab[level]] * (len(draft_tokens) + 1)
+
+
+def test_coin_acceptance_extremes_and_frequency():
+    from oracle.hsd import CoinDecisions
+    m = FlatModel()
+    run = HSD(m, (2, 3), CoinDecisions(1, (1.0, 1.0)))
+    run.generate([0], 60)
+    assert all(t[4] == t[3] for t in run.trace if t[0] > 0)           # every draft accepted
+    run = HSD(m, (2, 3), CoinDecisions(1, (0.0, 0.0)))
+    run.generate([0], 30)
+    assert all(t[4] == 0 for t in run.trace if t[0] > 0)              # every first draft rejected
+    run = HSD(m, (2, 3), CoinDecisions(7, (0.6, 0.8)))
+    run.generate([0], 3000)
+    for st, a in zip(run.stats[1:], (0.6, 0.8)):
+        assert st.tested > 1500
+        assert abs(st.accepted / st.tested - a) < 4 * (a * (1 - a) / st.tested) ** 0.5
+
+
+class FlatModel2(FlatModel):
+    n_levels = 2
+
+
+def _coin_cost_per_token(model, costs, alphas, T, n_new=2500, seeds=4):
+    from oracle.hsd import CoinDecisions, artificial_latency
+    total, n_tok = 0.0, 0
+    for seed in range(seeds):
+        run = HSD(model, T, CoinDecisions(seed, alphas))
+        run.generate([0], n_new)
+        emitted = run.stats[-1].emitted                                # whole rounds: nothing cut off
+        total += artificial_latency(run.stats, costs, emitted) * emitted
+        n_tok += emitted
+    return total / n_tok
+
+
+def test_coin_acceptance_with_artificial_costs_reproduces_theorem_3_2():
+    """The fully simplified setting of the ablation (IID acceptance, constant costs) is the model behind
+    Theorem 3.2.  Two levels: the closed form (1 - a) / (1 - a^(T+1)) (T c_0 + c_1) is exact, the simulation
+    converges to it.  Three levels: the theorem lets the top verifier see exactly T_1 drafts per round, the
+    literal Algorithm 1 hands it everything the level below collected (T_1 .. T_1 + T_0), so the simulated
+    cost lies a little below the closed form."""
+    from oracle import latency
+    sim2 = _coin_cost_per_token(FlatModel2(), (1.0, 10.0), (0.7,), (3,))
+    want2 = latency.expected_latency((1.0, 10.0), (0.7,), (3,))
+    assert abs(want2 - (1 - 0.7) / (1 - 0.7 ** 4) * 13.0) < 1e-12
+    assert abs(sim2 - want2) < 0.02 * want2, (sim2, want2)
+    costs, alphas, T = (1.0, 3.0, 10.0), (0.6, 0.8), (2, 3)
+    sim3 = _coin_cost_per_token(FlatModel(), costs, alphas, T)
+    want3 = latency.expected_latency(costs, alphas, T)
+    assert 0.88 * want3 < sim3 < 1.01 * want3, (sim3, want3)
+    # and the coins matter: another rate gives another cost
+    assert abs(_coin_cost_per_token(FlatModel2(), (1.0, 10.0), (0.4,), (3,), seeds=2) - want2) > 0.1 * want2
