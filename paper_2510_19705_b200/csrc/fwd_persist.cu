@@ -10,6 +10,9 @@
 // waits for the barrier that completes its operand.  GEMM work is split evenly over the CTAs in
 // (tile, k-block) units; each segment's partial sums go to a piece buffer and the following phase
 // (the next RMSNorm for the residual projections, a short finish phase otherwise) adds them up.
+// In decode passes two finish phases fold into their consumer: the attention phase finishes the
+// q / k / v of its own rows, and with at most four rows the down projection's CTAs build their
+// activation tiles from the gate / up pieces in shared memory (warps 5, 7, 9, 11).
 // Every wait (mbarrier, grid barrier) is bounded by wall time and raises a status word.
 #include "fwd_persist.cuh"
 #include "forward.cuh"
@@ -1247,6 +1250,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     //                           4 O pieces | 5 norm (+O pieces) -> ready(gate/up) | 6 gate/up pieces
     //                           7 gate/up finish -> ready(down) | 8 down pieces | 9 norm (+down pieces) -> ready(next)
     //   t = 1 + 10 n, + 1    output-head pieces | output-head finish
+    // Steps 1 and 7 are empty (no barrier) when the finish is folded into the phase after it.
     const int n_steps = 1 + 10 * a.n_run + (a.L > 0 ? 2 : 0);
     enum { K_EPI, K_FIN, K_ATTN_A, K_ATTN_B, K_NORM, K_NONE };
 #pragma unroll 1
