@@ -32,3 +32,13 @@ def test_strerror_and_argument_validation_need_no_gpu():
     assert lib.hsd_verify_level(0, None, None, None, 1, 1, 8, 0, 0, 0, None, 0, None, None, None) == -1
     assert lib.hsd_verify_workspace_bytes(0, 3) == 0
     assert lib.hsd_verify_workspace_bytes(4, 3) == 4 * 7 * 16
+
+
+def test_context_setters_reject_a_null_context_without_a_gpu():
+    from paper_2510_19705_b200 import binding
+    lib = binding.library()
+    binding._declare_engine(lib)
+    alphas = (ctypes.c_double * 2)(0.5, 0.5)
+    assert lib.hsd_set_iid_acceptance(None, alphas) == -1
+    assert lib.hsd_set_exit_heads(None, None, None) == -1
+    assert lib.hsd_set_trace(None, None, 0) == -1
