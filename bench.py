@@ -198,7 +198,8 @@ def run_ours(args):
     elif wl["T"] is None:
         T, costs, alphas, lat = choose_T(binding, cfg, weights, wl, prompts)
         calib = {"costs_ms": [round(c, 4) for c in costs], "alphas": [round(a, 4) for a in alphas],
-                 "expected_ms_per_token": round(lat, 4)}
+                 "expected_ms_per_token": round(lat, 4),
+                 "literal_algorithm_ms_per_token": round(binding.hsd_expected_latency_literal(costs, alphas, T), 4)}
     else:
         T, calib = list(wl["T"]), None
     eng = binding.Hsd(cfg, weights, wl["exits"], T, max_batch=B, max_seq=P + n_new + sum(T) + 16, page_size=wl["page"])
@@ -315,6 +316,7 @@ def ablation_table(binding, eng, prompts, n_new, steps, real_stats, real_ms, T):
     return {"ms_per_token": {"real_acceptance_real_cost": round(rr, 4), "iid_acceptance_real_cost": round(ir, 4),
                              "real_acceptance_artificial_cost": round(ra, 4), "iid_acceptance_artificial_cost": round(ia, 4)},
             "theorem_3_2_ms_per_token": round(binding.hsd_expected_latency(costs, alphas, T), 4),
+            "literal_algorithm_ms_per_token": round(binding.hsd_expected_latency_literal(costs, alphas, T), 4),
             "alphas": [round(a, 4) for a in alphas], "costs_ms": [round(c, 4) for c in costs]}
 
 

@@ -212,6 +212,13 @@ void hsd_destroy(hsd_ctx *ctx);
  * graph's constraint T_k >= T_{k-1} (Section 4.2, edge list).  Ties keep the lexicographically
  * first T.  Host-only; Errors: INVALID_ARG. */
 int hsd_expected_latency(const double *costs, const double *alphas, int n_levels, const int32_t *T, double *out);
+/* The same quantity for Algorithm 1 run as printed, under the same assumptions (IID acceptance, constant costs):
+ * Theorem 3.2 lets every verifier see exactly T_{k-1} drafts per round, the algorithm hands it everything the
+ * level below collected (T_{k-1} up to T_{k-1} + that level's last batch).  Exact renewal computation: the
+ * distribution of the number of tokens each level returns is carried upward, cost_k = E[rounds] (cost_{k-1} + c_k)
+ * (Wald), L = (cost_{K-1} + c_K) / E[tokens per target verification].  Equal to Theorem 3.2 for n_levels <= 2,
+ * below it otherwise.  Same arguments and errors as hsd_expected_latency (T[i] <= 4096). */
+int hsd_expected_latency_literal(const double *costs, const double *alphas, int n_levels, const int32_t *T, double *out);
 int hsd_search_T(const double *costs, const double *alphas, int n_levels, int T_max, int monotone, int32_t *out_T,
                  double *out_latency);
 

@@ -52,6 +52,47 @@ def expected_latency(costs, alphas, T):
     return top_multiplier(alphas[K - 1], T[K - 1]) * (cost + costs[K])
 
 
+def literal_latency(costs, alphas, T):
+    """Expected cost per token of Algorithm 1 run literally, under the same two assumptions (IID acceptance,
+    constant costs).  Theorem 3.2 lets every verifier see exactly T_{k-1} drafts; the algorithm as printed hands
+    a verifier everything the level below collected, between T_{k-1} and T_{k-1} + (its own batch) tokens.  This
+    is the exact renewal computation for that process:
+      level 0 returns t = T_0 tokens at cost T_0 c_0;
+      level k, 0 < k < K, repeats (call level k-1, verify: n accepted of t with P(n = j) = a^j (1 - a) for
+        j < t and a^t for j = t, yield n + 1) until it holds >= T_k tokens: cost_k = E[rounds] (cost_{k-1} + c_k)
+        by Wald's identity, and the distribution of the number it returns feeds level k + 1;
+      the target does one such round per call: L = (cost_{K-1} + c_K) / E[yield]  (renewal-reward).
+    Equal to Theorem 3.2 for one drafter (K = 1)."""
+    K = len(costs) - 1
+    assert len(alphas) == K and len(T) == K
+    if K == 0:
+        return costs[0]
+    dist = {T[0]: 1.0}                     # number of tokens the level below returns
+    cost = T[0] * costs[0]
+    for k in range(1, K + 1):
+        a = alphas[k - 1]
+        yld = {}
+        for t, pt in dist.items():
+            for j in range(t):
+                yld[j + 1] = yld.get(j + 1, 0.0) + pt * a ** j * (1.0 - a)
+            yld[t + 1] = yld.get(t + 1, 0.0) + pt * a ** t
+        if k == K:
+            return (cost + costs[K]) / sum(y * p for y, p in yld.items())
+        need = T[k]
+        mass = {0: 1.0}                    # probability of holding c < need tokens before a round
+        rounds, out = 0.0, {}
+        for c in range(need):
+            m = mass.get(c, 0.0)
+            if m == 0.0:
+                continue
+            rounds += m
+            for y, p in yld.items():
+                tgt = out if c + y >= need else mass
+                tgt[c + y] = tgt.get(c + y, 0.0) + m * p
+        cost = rounds * (cost + costs[k])
+        dist = out
+
+
 def subset_latency(costs, alpha, sigma, T):
     """Corollary 4.1: L(sigma, T); alpha[i][j] = acceptance rate drafter i -> verifier j."""
     c = [costs[i] for i in sigma]

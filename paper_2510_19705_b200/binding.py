@@ -162,6 +162,8 @@ def _declare_engine(lib):
     lib.hsd_expected_latency.restype = i32
     lib.hsd_expected_latency.argtypes = [c.POINTER(c.c_double), c.POINTER(c.c_double), i32, c.POINTER(c.c_int32),
                                          c.POINTER(c.c_double)]
+    lib.hsd_expected_latency_literal.restype = i32
+    lib.hsd_expected_latency_literal.argtypes = lib.hsd_expected_latency.argtypes
     lib.hsd_search_T.restype = i32
     lib.hsd_search_T.argtypes = [c.POINTER(c.c_double), c.POINTER(c.c_double), i32, i32, i32, c.POINTER(c.c_int32),
                                  c.POINTER(c.c_double)]
@@ -315,6 +317,17 @@ def hsd_expected_latency(costs, alphas, T):
     out = ctypes.c_double()
     _check(lib.hsd_expected_latency((ctypes.c_double * n)(*costs), (ctypes.c_double * max(1, n - 1))(*(alphas or [0])), n,
                                     (ctypes.c_int32 * max(1, n - 1))(*(T or [1])), ctypes.byref(out)))
+    return out.value
+
+
+def hsd_expected_latency_literal(costs, alphas, T):
+    """Expected cost per token of Algorithm 1 as printed (verifiers see everything the level below collected)."""
+    lib = library()
+    _declare_engine(lib)
+    n = len(costs)
+    out = ctypes.c_double()
+    _check(lib.hsd_expected_latency_literal((ctypes.c_double * n)(*costs), (ctypes.c_double * max(1, n - 1))(*(alphas or [0])),
+                                            n, (ctypes.c_int32 * max(1, n - 1))(*(T or [1])), ctypes.byref(out)))
     return out.value
 
 

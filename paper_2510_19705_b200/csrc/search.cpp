@@ -47,6 +47,53 @@ int hsd_expected_latency(const double *costs, const double *alphas, int n_levels
   return HSD_OK;
 }
 
+int hsd_expected_latency_literal(const double *costs, const double *alphas, int n_levels, const int32_t *T, double *out) {
+  if (!costs || !out || n_levels < 1 || n_levels > 16) return HSD_E_INVALID_ARG;
+  if (n_levels > 1 && (!alphas || !T)) return HSD_E_INVALID_ARG;
+  const int K = n_levels - 1;
+  long long span = 2;
+  for (int i = 0; i < K; ++i) {
+    if (T[i] < 1 || T[i] > 4096 || alphas[i] < 0.0 || alphas[i] > 1.0) return HSD_E_INVALID_ARG;
+    span += T[i];
+  }
+  if (K == 0) { *out = costs[0]; return HSD_OK; }
+  // dist[t]: probability that the level below returns t tokens; yld[y]: probability that a round yields y
+  std::vector<double> dist((size_t)span + 1, 0.0), yld, mass, next;
+  dist[T[0]] = 1.0;
+  double cost = T[0] * costs[0];
+  for (int k = 1; k <= K; ++k) {
+    const double a = alphas[k - 1];
+    yld.assign((size_t)span + 2, 0.0);
+    for (size_t t = 1; t < dist.size(); ++t) {
+      if (dist[t] == 0.0) continue;
+      double aj = 1.0;                                  // a^j
+      for (size_t j = 0; j < t; ++j) { yld[j + 1] += dist[t] * aj * (1.0 - a); aj *= a; }
+      yld[t + 1] += dist[t] * aj;
+    }
+    if (k == K) {
+      double mean = 0.0;
+      for (size_t y = 1; y < yld.size(); ++y) mean += (double)y * yld[y];
+      *out = (cost + costs[K]) / mean;
+      return HSD_OK;
+    }
+    const int need = T[k];
+    mass.assign((size_t)need + yld.size(), 0.0);        // mass[c]: probability of holding c tokens (c < need: before a round)
+    mass[0] = 1.0;
+    double rounds = 0.0;
+    for (int c = 0; c < need; ++c) {
+      const double m = mass[c];
+      if (m == 0.0) continue;
+      rounds += m;
+      for (size_t y = 1; y < yld.size(); ++y) mass[c + y] += m * yld[y];
+    }
+    cost = rounds * (cost + costs[k]);
+    next.assign((size_t)span + 1, 0.0);
+    for (size_t c = need; c < mass.size() && c < next.size(); ++c) next[c] = mass[c];
+    dist.swap(next);
+  }
+  return HSD_E_INVALID_ARG;
+}
+
 int hsd_search_T(const double *costs, const double *alphas, int n_levels, int T_max, int monotone, int32_t *out_T,
                  double *out_latency) {
   if (!costs || n_levels < 1 || n_levels > 8 || T_max < 1 || T_max > 64) return HSD_E_INVALID_ARG;

@@ -311,3 +311,24 @@ def test_coin_acceptance_with_artificial_costs_reproduces_theorem_3_2():
     assert 0.88 * want3 < sim3 < 1.01 * want3, (sim3, want3)
     # and the coins matter: another rate gives another cost
     assert abs(_coin_cost_per_token(FlatModel2(), (1.0, 10.0), (0.4,), (3,), seeds=2) - want2) > 0.1 * want2
+
+
+def test_literal_latency_model_matches_the_simulated_algorithm():
+    """oracle/latency.py: literal_latency is the exact expected cost per token of Algorithm 1 as printed under IID
+    acceptance and constant costs: the coin simulation converges to it for three and four levels, and it equals
+    Theorem 3.2's closed form for one drafter."""
+    from oracle import latency
+    assert abs(latency.literal_latency((1.0, 10.0), (0.7,), (3,)) - latency.expected_latency((1.0, 10.0), (0.7,), (3,))) < 1e-12
+    costs, alphas, T = (1.0, 3.0, 10.0), (0.6, 0.8), (2, 3)
+    sim3 = _coin_cost_per_token(FlatModel(), costs, alphas, T)
+    lit3 = latency.literal_latency(costs, alphas, T)
+    assert abs(sim3 - lit3) < 0.02 * lit3, (sim3, lit3)
+    assert lit3 < latency.expected_latency(costs, alphas, T)          # more drafts per target pass than the theorem grants
+
+    class Flat4(FlatModel):
+        n_levels = 4
+        tab = np.concatenate([FlatModel.tab, FlatModel.tab[-1:]])
+    costs, alphas, T = (1.0, 2.0, 5.0, 20.0), (0.5, 0.7, 0.6), (1, 2, 2)
+    sim4 = _coin_cost_per_token(Flat4(), costs, alphas, T)
+    lit4 = latency.literal_latency(costs, alphas, T)
+    assert abs(sim4 - lit4) < 0.02 * lit4, (sim4, lit4)

@@ -1,6 +1,8 @@
 """The library's host-side latency model and T search against the oracle's (no GPU needed)."""
 import itertools
 
+import numpy as np
+
 from oracle import latency as L
 from paper_2510_19705_b200 import binding
 
@@ -96,3 +98,24 @@ def test_search_hierarchy_rejects_bad_arguments():
         binding.hsd_search_hierarchy([1.0, 2.0], [[0.0, 1.5], [0.0, 0.0]], 4)
     with pytest.raises(binding.HsdError):
         binding.hsd_search_hierarchy([1.0, 2.0], [[0.0, 0.5], [0.0, 0.0]], 0)
+
+
+def test_literal_latency_matches_the_oracle():
+    from oracle import latency
+    from paper_2510_19705_b200 import binding
+    rng = np.random.default_rng(5)
+    for _ in range(40):
+        n = int(rng.integers(1, 6))
+        costs = sorted(rng.uniform(0.1, 10.0, n).tolist())
+        alphas = rng.uniform(0.0, 1.0, n - 1).tolist()
+        T = [int(t) for t in rng.integers(1, 9, n - 1)]
+        want = latency.literal_latency(tuple(costs), tuple(alphas), tuple(T))
+        got = binding.hsd_expected_latency_literal(costs, alphas, T)
+        assert abs(got - want) <= 1e-12 * max(1.0, abs(want)), (costs, alphas, T)
+        if n <= 2:
+            assert abs(got - binding.hsd_expected_latency(costs, alphas, T)) <= 1e-12 * max(1.0, got)
+        else:
+            assert got <= binding.hsd_expected_latency(costs, alphas, T) * (1 + 1e-12)
+    # extremes: every draft accepted / every first draft rejected
+    assert abs(binding.hsd_expected_latency_literal([1.0, 2.0, 4.0], [1.0, 1.0], [2, 3]) - (1 * (2 * 1.0 + 2.0) + 4.0) / 4.0) < 1e-12   # one round of 3 tokens below, 3 + 1 at the target
+    assert abs(binding.hsd_expected_latency_literal([1.0, 2.0, 4.0], [0.0, 0.0], [2, 3]) - (3 * (2 * 1.0 + 2.0) + 4.0) / 1.0) < 1e-12
