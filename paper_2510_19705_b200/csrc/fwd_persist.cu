@@ -973,6 +973,38 @@ __device__ __forceinline__ void gemm_finish(const FwdArgs &a, WorkerCtx &w, int 
   float *gstage = w.staging + gidx * (kTcBlockM * (RG + 1));
   const int n_rb = (g.rows + RB - 1) / RB, n_units = g.n_tiles * n_rb;
   const bool rope_cached = a.R <= kRopeCacheRows;
+  if (g.mode == MODE_SWIGLU) {
+    // gate / up: a thread owns one of the tile's 64 columns (gate in tile row c, up in tile row c + 64) and four of
+    // the unit's eight token rows; all its loads are in flight at once, no staging and no barrier
+    const int cc = gm & (kTcBoxRows - 1), rh = (gm >> 6) * (RB / 2);
+#pragma unroll 1
+    for (int u = w.c + gidx * w.G; u < n_units; u += 2 * w.G) {
+      const int tile = u / n_rb, r0 = (u - tile * n_rb) * RB + rh, col = tile * kTcBoxRows + cc;
+      int fo, n_pieces;
+      tile_pieces(g, geo, tile, fo, n_pieces);
+      const float *base = a.pieces + (size_t)tile * geo.pieces_max * NPAD * kTcBlockM + cc;
+      float tg[PBF][RB / 2], tu[PBF][RB / 2];
+#pragma unroll
+      for (int pp = 0; pp < PBF; ++pp)
+#pragma unroll
+        for (int i = 0; i < RB / 2; ++i) {
+          const bool on = pp < n_pieces && r0 + i < g.rows;
+          const float *src = base + ((size_t)pp * NPAD + r0 + i) * kTcBlockM;
+          tg[pp][i] = on ? __ldcg(src) : 0.f;
+          tu[pp][i] = on ? __ldcg(src + kTcBoxRows) : 0.f;
+        }
+      if (col < g.seg_n[0]) {
+#pragma unroll
+        for (int i = 0; i < RB / 2; ++i) {
+          float gt = 0.f, up = 0.f;
+#pragma unroll
+          for (int pp = 0; pp < PBF; ++pp) { gt += tg[pp][i]; up += tu[pp][i]; }
+          if (r0 + i < g.rows) a.act[(size_t)(r0 + i) * a.ff + col] = __float2bfloat16_rn(silu_mul(gt, up));
+        }
+      }
+    }
+    return;
+  }
 #pragma unroll 1
   for (int u = w.c + gidx * w.G; u < n_units; u += 2 * w.G) {
     const int tile = u / n_rb, r_lo = (u - tile * n_rb) * RB, r_hi = min(g.rows, r_lo + RB);
