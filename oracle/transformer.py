@@ -37,6 +37,12 @@ def bf16_round(x):
 
 
 def bf16_bits_to_f64(bits):
+    """bf16 bit patterns (uint16) widened to float64: exact (a bf16 value is an fp32 value with a zero low half).
+    Large matrices go through torch's conversion, which uses every host core; same values."""
+    bits = np.ascontiguousarray(bits)
+    if bits.size >= (1 << 20):
+        import torch
+        return torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16).to(torch.float64).numpy()
     return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
 
 
@@ -47,12 +53,18 @@ class Transformer:
     patterns (dtype 'bf16'), matrices stored [out_features, in_features].  Optional
     weights['exit_heads']: list over levels of None (shared head) or dict(lm_head[, final_norm])."""
 
-    def __init__(self, cfg, weights, exits, cache_bytes=8 << 30):
+    def __init__(self, cfg, weights, exits, cache_bytes=8 << 30, share_weights_with=None):
+        """share_weights_with: another Transformer over the same weights whose widened (float64) copies of the
+        matrices are reused instead of being made again (a cache only; no effect on any value)."""
         self.cfg, self.w, self.exits = dict(cfg), weights, list(exits)
         assert self.exits == sorted(self.exits) and self.exits[-1] == cfg["n_layers"]
         self.n_levels = len(self.exits)
         self.bf16 = cfg["dtype"] == "bf16"
-        self._wide, self._wide_bytes, self._budget = {}, 0, cache_bytes
+        if share_weights_with is not None:
+            assert share_weights_with.w is weights
+            self._wide, self._acct = share_weights_with._wide, share_weights_with._acct
+        else:
+            self._wide, self._acct = {}, {"bytes": 0, "budget": cache_bytes}
         self.reset()
 
     # ------------------------------------------------------------------ weights
@@ -63,9 +75,9 @@ class Transformer:
             return hit
         raw = self.w[name] if layer is None else self.w["layers"][layer][name]
         wide = bf16_bits_to_f64(raw) if self.bf16 else raw.astype(np.float64)
-        if self._wide_bytes + wide.nbytes <= self._budget:
+        if self._acct["bytes"] + wide.nbytes <= self._acct["budget"]:
             self._wide[key] = wide
-            self._wide_bytes += wide.nbytes
+            self._acct["bytes"] += wide.nbytes
         return wide
 
     def _head(self, level, name):
@@ -144,12 +156,12 @@ class Transformer:
             for r in range(R):
                 n_keys = start + r + 1                      # causal: keys at positions <= own
                 Kc, Vc = self.K[l][:n_keys], self.V[l][:n_keys]
-                for hq in range(nq):
-                    g = hq // group
-                    s = (Kc[:, g, :] @ q[r, hq]) * scale
-                    p = np.exp(s - s.max())
-                    p /= p.sum()
-                    att[r, hq] = p @ Vc[:, g, :]
+                for g in range(nkv):                      # the query heads that share KV head g, together
+                    qg = q[r, g * group:(g + 1) * group]                 # [group, hd]
+                    s = (Kc[:, g, :] @ qg.T) * scale                     # [n_keys, group]
+                    p = np.exp(s - s.max(axis=0, keepdims=True))
+                    p /= p.sum(axis=0, keepdims=True)
+                    att[r, g * group:(g + 1) * group] = p.T @ Vc[:, g, :]
             att = self._rnd(att.reshape(R, nq * hd))
             x = x + att @ self._mat(l, "wo").T
             h = self._rnd(self._rmsnorm(x, self._mat(l, "mlp_norm")))

@@ -4,6 +4,9 @@ The oracle cannot replay a whole 8B-shape generation in reasonable time, so: (a)
 re-taken by the oracle's decision arithmetic on the library's own stored logits (bit-exact), (b) the logits of
 sampled calls (one per level) are compared with the oracle's own forward, (c) properties that hold at any size
 (yield bounds, counters, determinism) are checked on the whole run."""
+import json
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -60,19 +63,29 @@ def _context_of(recs, rec, prompt, b=0):
     return buf if rec is None else buf[:rec["ctx_len"]]
 
 
-def _perturbed_oracle_logits(cfg, w_np, exits, level, context, drafts, eps=2e-6):
+def _perturbed_oracle_logits(cfg, w_np, exits, level, context, drafts, eps=2e-6, share=None):
     """The oracle's logits for the same call when every value is nudged by eps (the size of fp32 accumulation
-    error) before each bf16 rounding point."""
+    error) before each bf16 rounding point.  `share`: a Transformer over the same weights whose widened copies
+    of the matrices are reused."""
     from oracle import transformer as T
     orig = T.bf16_round
     rng = np.random.default_rng(0)
     T.bf16_round = lambda x: orig(np.asarray(x, dtype=np.float64) * (1.0 + eps * rng.standard_normal(np.shape(x))))
     try:
-        m = T.Transformer(cfg, w_np, exits, cache_bytes=24 << 30)
+        m = T.Transformer(cfg, w_np, exits, cache_bytes=24 << 30, share_weights_with=share)
         m.rows(level, context, drafts)
         return m.last_logits64.copy()
     finally:
         T.bf16_round = orig
+
+
+_FIGURES = []           # what the tolerance checks measured; written to $HSD_PARITY_REPORT (a JSON file) if set
+
+
+def _softmax64(x):
+    x = np.asarray(x, dtype=np.float64)
+    e = np.exp(x - x.max(axis=-1, keepdims=True))
+    return e / e.sum(axis=-1, keepdims=True)
 
 
 def _assert_bf16_logits_close(got, ref, ref_perturbed, what):
@@ -80,13 +93,45 @@ def _assert_bf16_logits_close(got, ref, ref_perturbed, what):
     rounding step: nudging every value by 2e-6 before rounding moves the oracle's own logits by 0.005 rms
     (1B shape, 4 layers) to 0.012 rms (8B shape, 4 layers) and it grows with depth, so a fixed 2e-2 bound per
     entry cannot hold for any fp32-accumulating implementation.  The library must stay within twice the
-    oracle's own sensitivity (rms and 99th percentile), measured for the same call."""
-    d = np.abs(np.asarray(got, dtype=np.float64) - np.asarray(ref, dtype=np.float64))
-    d0 = np.abs(np.asarray(ref_perturbed, dtype=np.float64) - np.asarray(ref, dtype=np.float64))
+    oracle's own sensitivity, measured for the same call (d0 = |perturbed oracle - oracle|), in every respect:
+    rms, 99th percentile, the largest entry, and the share of entries beyond each threshold (2e-2 among them)
+    against the share of 2 d0 + 2e-3 beyond it.  Probabilities (softmax of the rows) must agree within 2e-2
+    absolute per entry, and in total variation within twice the perturbed oracle's + 5e-3."""
+    got, ref, ref_perturbed = (np.asarray(a, dtype=np.float64) for a in (got, ref, ref_perturbed))
+    d, d0 = np.abs(got - ref), np.abs(ref_perturbed - ref)
     rms, rms0 = float(np.sqrt((d ** 2).mean())), float(np.sqrt((d0 ** 2).mean()))
-    assert rms <= 2.0 * rms0 + 2e-3, (what, rms, rms0)
-    assert np.percentile(d, 99) <= 2.0 * np.percentile(d0, 99) + 4e-3, (what, float(np.percentile(d, 99)))
-    assert rms < 0.05 * float(np.std(ref)), what           # and never more than a few percent of the logit scale
+    fig = {"what": str(what), "rows": int(d.shape[0]), "rms": rms, "rms_perturbed_oracle": rms0,
+           "max": float(d.max()), "max_perturbed_oracle": float(d0.max()),
+           "frac_beyond_2e-2": float((d > 2e-2).mean()), "frac_beyond_2e-2_perturbed_oracle": float((d0 > 2e-2).mean()),
+           "logit_std": float(np.std(ref))}
+    pg, pr, pp = _softmax64(got), _softmax64(ref), _softmax64(ref_perturbed)
+    fig["prob_max_abs"] = float(np.abs(pg - pr).max())
+    fig["prob_tv"] = float(0.5 * np.abs(pg - pr).sum(axis=-1).max())
+    fig["prob_tv_perturbed_oracle"] = float(0.5 * np.abs(pp - pr).sum(axis=-1).max())
+    _FIGURES.append(fig)
+    path = os.environ.get("HSD_PARITY_REPORT")
+    if path:
+        with open(path, "w") as f:
+            json.dump(_FIGURES, f, indent=1)
+    assert rms <= 2.0 * rms0 + 2e-3, fig
+    assert np.percentile(d, 99) <= 2.0 * np.percentile(d0, 99) + 4e-3, fig
+    assert rms < 0.05 * float(np.std(ref)), fig            # and never more than a few percent of the logit scale
+    assert d.max() <= 2.5 * d0.max() + 1e-2, fig           # no single entry far outside the band
+    for tau in (1e-2, 2e-2, 4e-2, 8e-2):
+        assert (d > tau).mean() <= (2.0 * d0 + 2e-3 > tau).mean() + 2e-3, (tau, fig)
+    assert fig["prob_max_abs"] <= 2e-2, fig
+    assert fig["prob_tv"] <= 2.0 * fig["prob_tv_perturbed_oracle"] + 5e-3, fig
+    return fig
+
+
+def _oracle_check(om, cfg, w_np, exits, rec, context, what):
+    """One logged call against the oracle's own forward (and the perturbed oracle's, for the band)."""
+    drafts = [] if rec["level"] == 0 else rec["tokens"][:-1].tolist()
+    om.rows(rec["level"], context, drafts)
+    ref = om.last_logits64.copy()
+    ref_p = _perturbed_oracle_logits(cfg, w_np, exits, rec["level"], context, drafts, share=om)
+    got = rec["logits"][:1] if rec["level"] == 0 else rec["logits"]
+    return _assert_bf16_logits_close(got, ref, ref_p, what)
 
 
 def _check_run_properties(stats, T, n_new):
@@ -217,3 +262,127 @@ def test_long_context_four_levels_paged_batch(lib, tmp_path):
             ref = om.last_logits64.copy()
             ref_p = _perturbed_oracle_logits(cfg, w_np, wl["exits"], lvl, ctx_b, drafts_b)
             _assert_bf16_logits_close(rec["logits"], ref, ref_p, ("mini4long", b, lvl))
+
+
+def _run_traced(lib, cfg, w, exits, T, prompts, n_new, seed, page, tmp_path, tag="trace"):
+    B, P = prompts.shape
+    eng = lib.Hsd(cfg, w, exits, T, max_batch=B, max_seq=P + n_new + sum(T) + 16, page_size=page)
+    path = str(tmp_path / (tag + ".bin"))
+    eng.set_trace(path, logit_calls=10 ** 6)
+    toks, stats, _ = eng.generate(prompts.cuda(), n_new, seed)
+    eng.set_trace(None)
+    eng.close()
+    return toks.cpu(), stats, lib.read_trace(path)
+
+
+@pytest.mark.parametrize("name,T,P,n_new", [("1b3", (4, 2), 96, 24), ("8b3", (1, 1), 96, 12)])
+def test_every_level_first_call_matches_oracle_forward(lib, tmp_path, name, T, P, n_new):
+    """The model shapes of the benchmark with a short prompt, so that the oracle can follow EVERY level: the first
+    call of each level -- the 16- / 32-layer target verification with its two or three rows among them, over the
+    keys and values the 95-row prompt pass wrote -- against the oracle's own forward.  8B shape: T = (1, 1), the
+    value the latency search returns in the benchmark run."""
+    wl = inputs.WORKLOADS[name]
+    cfg, exits = wl["model"], wl["exits"]
+    w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
+    prompts = inputs.make_prompts(cfg["vocab"], 1, P, wl["prompt_seed"])
+    toks, stats, recs = _run_traced(lib, cfg, w, exits, list(T), prompts, n_new, 0, wl["page"], tmp_path)
+    _check_run_properties(stats, list(T), n_new)
+    assert _replay_decisions(recs, 0) == sum(s["calls"] for s in stats[1:])
+    prompt = prompts[0].tolist()
+    assert _context_of(recs, None, prompt)[P:P + n_new] == toks[0].tolist()
+    w_np = inputs.weights_to_numpy(w)
+    om = Transformer(cfg, w_np, exits, cache_bytes=24 << 30)
+    for level in range(len(exits)):
+        rec = next(r for r in recs if r["level"] == level)
+        _oracle_check(om, cfg, w_np, exits, rec, _context_of(recs, rec, prompt), (name, "P=%d" % P, "level", level))
+
+
+@pytest.mark.parametrize("P,n_new,with_oracle", [(160, 24, True), (1024, 32, False)])
+def test_8b_shape_batch_of_eight(lib, tmp_path, P, n_new, with_oracle):
+    """The 8B-shape hierarchy with eight sequences in one batch (passes of 17-32 rows, prompt chunks that span
+    sequences): every decision of every sequence follows the oracle on the logged logits; with the short prompt,
+    sequence 0's first target verification (32 layers) also matches the oracle's forward."""
+    wl = inputs.WORKLOADS["8b3"]
+    cfg, exits, T, B = wl["model"], wl["exits"], [1, 2], 8
+    w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
+    prompts = inputs.make_prompts(cfg["vocab"], B, P, wl["prompt_seed"])
+    toks, stats, recs = _run_traced(lib, cfg, w, exits, T, prompts, n_new, 2, wl["page"], tmp_path)
+    _check_run_properties(stats, T, n_new * B)
+    assert _replay_decisions(recs, 2, n_seq=B) == sum(s["calls"] for s in stats[1:])
+    for b in range(B):
+        prompt = prompts[b].tolist()
+        assert _context_of(recs, None, prompt, b)[P:P + n_new] == toks[b].tolist()
+    if with_oracle:
+        w_np = inputs.weights_to_numpy(w)
+        om = Transformer(cfg, w_np, exits, cache_bytes=24 << 30)
+        rec = next(r for r in recs if r["seq"] == 0 and r["level"] == 2)
+        _oracle_check(om, cfg, w_np, exits, rec, _context_of(recs, rec, prompts[0].tolist()), ("8b3 batch 8", "target"))
+
+
+def test_long_context_config_full_size(lib, tmp_path):
+    """The long-context configuration at its own size: 8B shape, exits (2, 6, 16, 32), T = (2, 2, 3), sixteen
+    sequences with 8192-token prompts in 16-token pages.  The oracle cannot follow a forward over 8192 tokens in
+    test time, so (a) every decision of all sixteen sequences is re-taken by the oracle on the logged logits,
+    (b) sequences 0 and 15 of the batch give the logits that a batch of one gives for the same prompt (same
+    calls, as long as the two runs draw the same tokens) within the rounding band, which ties paging and batch
+    indexing at this size to the single-sequence path, and (c) the same batch shape with 2304-token prompts (the
+    key-split model of long contexts, several pages and sub-tiles per split) is checked against the oracle's own
+    forward at level 1 (six layers, catch-up row + drafts)."""
+    wl = inputs.WORKLOADS["8b4long"]
+    cfg, exits, T, B = wl["model"], wl["exits"], list(wl["T"]), wl["batch"]
+    w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
+    P, n_new, seed = wl["prompt"], 8, 1
+    prompts = inputs.make_prompts(cfg["vocab"], B, P, wl["prompt_seed"])
+    toks, stats, recs = _run_traced(lib, cfg, w, exits, T, prompts, n_new, seed, wl["page"], tmp_path)
+    _check_run_properties(stats, T, n_new * B)
+    assert _replay_decisions(recs, seed, n_seq=B) == sum(s["calls"] for s in stats[1:])
+    for b in range(B):
+        assert _context_of(recs, None, prompts[b].tolist(), b)[P:P + n_new] == toks[b].tolist()
+    for b in (0, B - 1):
+        # a batch of one has sequence index 0, so its random numbers differ from sequence b's: only calls made
+        # before the first draw differs can be compared (the first level-0 row always is)
+        _, _, recs1 = _run_traced(lib, cfg, w, exits, T, prompts[b:b + 1], n_new, seed, wl["page"], tmp_path, "single%d" % b)
+        first_a = next(r for r in recs if r["seq"] == b)
+        first_b = recs1[0]
+        assert first_a["level"] == first_b["level"] == 0 and first_a["ctx_len"] == first_b["ctx_len"] == P
+        d = first_a["logits"][0].astype(np.float64) - first_b["logits"][0].astype(np.float64)
+        rms = float(np.sqrt((d ** 2).mean()))
+        _FIGURES.append({"what": "8b4long batch 16 vs batch 1, sequence %d, first level-0 row" % b, "rms": rms,
+                         "max": float(np.abs(d).max())})
+        assert rms <= 0.02 and np.abs(d).max() <= 0.15, (b, rms, float(np.abs(d).max()))
+    # (c) the oracle's forward at a context the oracle can follow
+    P2 = 2304
+    prompts2 = inputs.make_prompts(cfg["vocab"], B, P2, wl["prompt_seed"] + 1)
+    toks2, stats2, recs2 = _run_traced(lib, cfg, w, exits, T, prompts2, n_new, seed, wl["page"], tmp_path, "mid")
+    assert _replay_decisions(recs2, seed, n_seq=B) == sum(s["calls"] for s in stats2[1:])
+    w_np = inputs.weights_to_numpy(w)
+    om = Transformer(cfg, w_np, exits, cache_bytes=24 << 30)
+    rec = next(r for r in recs2 if r["seq"] == 0 and r["level"] == 1)
+    _oracle_check(om, cfg, w_np, exits, rec, _context_of(recs2, rec, prompts2[0].tolist()), ("8b4long P=2304 batch 16", "level 1"))
+
+
+def test_long_context_config_level0_against_oracle_at_8192_tokens(lib, tmp_path):
+    """The long-context configuration's first drafting step at its own context length against the oracle's own
+    forward: sixteen 8192-token prompts in 16-token pages, sequence 0's first level-0 row (two layers over all
+    8192 positions: every key split, page and sub-tile of the prompt's keys is read).  The band comes from the
+    perturbed oracle on the first 256 tokens of the same prompt (the full-length perturbed pass would double
+    the test's minutes; the sensitivity of a two-layer forward does not grow with the context: the measured
+    figures are in the parity report)."""
+    wl = inputs.WORKLOADS["8b4long"]
+    cfg, exits, T, B = wl["model"], wl["exits"], list(wl["T"]), wl["batch"]
+    w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
+    P = wl["prompt"]
+    prompts = inputs.make_prompts(cfg["vocab"], B, P, wl["prompt_seed"])
+    _, _, recs = _run_traced(lib, cfg, w, exits, T, prompts, 2, 1, wl["page"], tmp_path)
+    rec = next(r for r in recs if r["seq"] == 0 and r["level"] == 0)
+    assert rec["ctx_len"] == P
+    w_np = inputs.weights_to_numpy(w)
+    om = Transformer(cfg, w_np, exits, cache_bytes=24 << 30)
+    prompt = prompts[0].tolist()
+    om.rows(0, prompt[:256], [])
+    short = om.last_logits64.copy()
+    short_p = _perturbed_oracle_logits(cfg, w_np, exits, 0, prompt[:256], [], share=om)
+    om.reset()
+    om.rows(0, prompt, [])
+    ref = om.last_logits64.copy()
+    _assert_bf16_logits_close(rec["logits"][:1], ref, ref + (short_p - short), ("8b4long P=8192 batch 16", "level 0"))
