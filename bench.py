@@ -371,7 +371,7 @@ def run_accept(args):
             "e2e": {"value": round(B * t / (e2e_ms / 1e3), 1), "unit": "positions/s", "h2d_bytes_per_step": bytes_alg + B * t * 4,
                     "d2h_bytes_per_step": B * (t + 1) * 4},
             "gpu_launches": int(launches), "clocks": clk.summary(),
-            "roofline": {"bound": "hbm", "kernel": "row_stats_vec_kernel + decide_kernel (one verification call)",
+            "roofline": {"bound": "hbm", "kernel": "verify_fused_kernel (one verification call: row statistics, accept tests, final draw)",
                          "achieved": round(achieved, 1), "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
                          "frac": round(achieved / hbm_peak, 4), "traffic": None, "bytes_per_launch": bytes_alg}}
     if not args.no_cpu_baseline:

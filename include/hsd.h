@@ -49,7 +49,7 @@ enum { HSD_F32 = 0, HSD_BF16 = 1 };
 const char *hsd_strerror(int status);
 
 /* ---------------------------------------------------------------------------------------
- * Level-0 drafting, sampling step (Algorithm 1, base case: "new_token, new_prob <- M_0(...)").
+ * Level-0 drafting, sampling step (Algorithm 1, base case: M_0 emits one token and its distribution at a time).
  * Token (b, j) is drawn from softmax(logits[b, j, :]) by inverse CDF in ascending token id
  * with the uniform addressed (j, call_serial, level 0, purpose 0, b).
  *   logits      device [batch, rows, vocab], dtype as given, row-major, read only
@@ -91,16 +91,19 @@ int hsd_verify_level(int level, const void *target_logits, const void *draft_log
  * allocating call (which may synchronise the whole device) is off limits.  hsd_verify_level
  * makes such callers find scratch memory somewhere; this variant brings its own.
  *
- * Same arguments, outputs and results as hsd_verify_level.  The row statistics live in a fixed
- * 64 KiB device array inside the library image (every GPU that loads the library holds it until
- * the process exits), which bounds the call: batch * (2 t + 1) <= 4096, else HSD_E_TOO_LARGE.
+ * Same arguments, outputs and results as hsd_verify_level.  The scratch (row statistics, counters
+ * and a queue of sequences) lives in a fixed device array of 98,560 bytes inside the library image (every GPU
+ * that loads the library holds it until the process exits), which bounds the call:
+ * batch * (2 t + 1) <= 4096, else HSD_E_TOO_LARGE (exactly 4096 is accepted).
  * The call performs no cudaMalloc / cudaFree and uses no allocating library routine.
- *   - The first call on each device looks up the array's device address; make that first call
- *     outside any stream capture.
- *   - All calls share the one array and it keeps whatever the last call left in it.  Nothing in
- *     it has to start at zero (each call overwrites every entry before reading it), but two
- *     calls that overlap on the GPU -- different streams, or different host threads -- race on it.
- *     Serialise such calls (one stream, or an event between them).
+ *   - The first call on each device looks up the array's device address and keeps it; make that
+ *     first call outside any stream capture.  The kept address does not survive cudaDeviceReset():
+ *     do not use this entry point on a device after resetting it.
+ *   - All calls share the one array and it keeps whatever the last call left in it.  The counters
+ *     and the queue must start at zero and every call clears them on `stream` before its kernel; the statistics
+ *     are overwritten before they are read.  Two calls that overlap on the GPU -- different streams,
+ *     or different host threads -- race on the array: serialise them (one stream, or an event
+ *     between them).
  * Errors: INVALID_ARG, TOO_LARGE, CUDA. */
 int hsd_verify_level_static(int level, const void *target_logits, const void *draft_logits,
                             const int32_t *draft_tokens, int batch, int t, int vocab, int dtype,
@@ -156,6 +159,30 @@ size_t hsd_workspace_bytes(const hsd_model_desc *model, const int32_t *exit_laye
 int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_levels, const int32_t *T,
                void *workspace, size_t workspace_bytes, hsd_ctx **out);
 
+/* The hierarchy as separate models (Section 3.1, "Preliminaries": M_0..M_K are arbitrary models over one
+ * vocabulary, each with its own cost c_i; Section 5.1's early exits are one way to get them).  Level i is ALL
+ * layers of models[i] with that model's own embedding, final norm and output head, and keeps a KV cache of its own:
+ * a level's forward pass processes every position its own cache has not seen (the drafts it verifies plus the
+ * tokens the other levels emitted since its last pass), the prompt pass runs every model over the prompt, and the
+ * rollback after a verification cuts every model's cache to the accepted length.  Algorithm 1 and Algorithm 2 run
+ * unchanged on top (hsd_generate, hsd_set_trace, hsd_set_iid_acceptance, hsd_set_exit_heads, hsd_destroy).
+ *   models  host [n_levels], models[n_levels - 1] = the target.  All must agree on vocab, dtype, max_batch,
+ *           max_seq and page_size; layer counts, widths, head counts and d_ff are free per model.
+ *   T       host [n_levels - 1], each >= 1.
+ * hsd_layer_logits on such a context runs the target model.
+ * Errors: INVALID_ARG (also: the models disagree on a shared quantity), WORKSPACE_TOO_SMALL, UNSUPPORTED, CUDA. */
+size_t hsd_models_workspace_bytes(const hsd_model_desc *models, int n_levels, const int32_t *T);
+int hsd_create_models(const hsd_model_desc *models, int n_levels, const int32_t *T, void *workspace,
+                      size_t workspace_bytes, hsd_ctx **out);
+
+/* Decode passes of bf16 models fold two finish phases of the verification forward (Algorithm 2's multi-row pass)
+ * into their consumers: the q / k / v finish into the attention phase, the gate / up finish into the down
+ * projection; and the RMSNorm after each residual projection starts, on CTAs that hold no tile of that
+ * projection, as soon as its partial sums are stored instead of after a grid-wide barrier.  fold_qkv = 0 /
+ * fold_gate_up = 0 / early_norm = 0 keeps the separate phase or the barrier; the results are the same sums in
+ * the same order either way (a test hook and a tuning knob; all on by default).  Errors: INVALID_ARG. */
+int hsd_set_phase_folding(hsd_ctx *ctx, int fold_qkv, int fold_gate_up, int early_norm);
+
 /* One output head per level instead of the shared one (Section 5.1: the setting in which every exit
  * layer has its own trained head, a linear map from the embedding dimension to the vocabulary, so that
  * memory grows with the number of levels; the shared head of the descriptor is the other setting).
@@ -188,7 +215,9 @@ int hsd_set_iid_acceptance(hsd_ctx *ctx, const double *alphas);
  *   timing_ms   host [2] or NULL: device time of the prompt pass and of the generation loop
  * Blocks until done (the host reads one accept count per verification).  Requires
  * prompt_len + n_new + sum(T) + n_levels + 1 <= max_seq and batch <= max_batch.
- * Errors: INVALID_ARG, OUT_OF_PAGES, CUDA, IO (trace file). */
+ * Errors: INVALID_ARG, OUT_OF_PAGES, CUDA, IO (trace file), DEVICE_TIMEOUT (a kernel gave up one of its
+ * bounded waits: it raises a status word in the workspace that every later call of the context reports too;
+ * the word is sticky, so a context that has returned DEVICE_TIMEOUT must be destroyed). */
 int hsd_generate(hsd_ctx *ctx, const int32_t *prompt_ids, int batch, int prompt_len, int n_new, uint64_t seed,
                  void *stream, int32_t *out_tokens, hsd_level_stats *stats, double *timing_ms);
 

@@ -1,15 +1,17 @@
-"""Algorithm 1 (Hierarchical Speculative Decoding), step by step, and the outer loop.
+"""Algorithm 1 (Hierarchical Speculative Decoding) and the outer generation loop.
 
-Models M_0..M_K (M_K the target), parameters T_0..T_{K-1}.
-  idx = 0      M_0 samples T_0 tokens autoregressively, keeping each full row.
-  0 < idx < K  repeat { draft = HSD(idx-1, context+tokens); Verify(idx, draft) }
-               until count >= T_idx; everything collected is returned (the count
-               may overshoot T_idx: Algorithm 1 returns tokens, probs untruncated).
-  idx = K      one draft from HSD(K-1) and one Verify.
-Generation (Section 3.2, "begins with a call with idx = K"): call HSD(K, prompt +
-output) until at least n_new tokens exist, keep the first n_new (the paper does
-not say how generation stops; truncation is this project's reading).  K = 0 is
-this project's degenerate case: one sample from M_0 per round.
+Models M_0..M_K (M_K the target), parameters T_0..T_{K-1}.  What each level does:
+  bottom (0)     M_0 extends the context by T_0 tokens, one forward per token,
+                 and keeps the full distribution row behind every token.
+  middle (i)     asks the level below for drafts after everything it has collected
+                 so far, verifies them with M_i (Algorithm 2), and repeats until it
+                 holds at least T_i tokens; ALL collected tokens and rows go up (the
+                 count may exceed T_i: Algorithm 1 hands back what it has, uncut).
+  top (K)        one draft request to level K-1, one verification by the target.
+Generation (Section 3.2 starts every round at the top level): rounds are run on
+prompt + output until at least n_new tokens exist and the first n_new are kept
+(the paper does not say how generation stops; truncation is this project's
+reading).  K = 0 is this project's degenerate case: one sample from M_0 per round.
 
 Random numbers are addressed by (purpose, level, per-level call serial, position
 in the call, sequence) -- see oracle/philox.py -- so a decision's uniform does
@@ -100,35 +102,40 @@ class HSD:
         return s
 
     def hsd(self, idx, context):
-        tokens, rows = [], []
-        st = self.stats[idx]
+        """Tokens and rows that level idx hands to the level above for this context."""
         if idx == 0:
-            serial = self._next_serial(0)
-            n_draft = self.T[0] if self.K > 0 else 1
-            count = 0
-            while count < n_draft:
-                row = self.model.rows(0, context + tokens, [])[0]
-                tok = self.dec.draft_sample(row, count, serial, 0)
-                tokens.append(tok)
-                rows.append(row)
-                count += 1
-                st.rows += 1
-            st.calls += 1
-            st.emitted += n_draft
-            self.trace.append((0, serial, len(context), 0, n_draft, tuple(tokens)))
-        elif idx == self.K:
+            return self._bottom(context)
+        if idx == self.K:
             d_tok, d_rows = self.hsd(idx - 1, context)
-            tokens, rows = self._verify(idx, d_tok, d_rows, context)
-        else:
-            count = 0
-            while count < self.T[idx]:
-                ctx = context + tokens
-                d_tok, d_rows = self.hsd(idx - 1, ctx)
-                v_tok, v_rows = self._verify(idx, d_tok, d_rows, ctx)
-                tokens.extend(v_tok)
-                rows.extend(v_rows)
-                count += len(v_tok)
+            return self._verify(idx, d_tok, d_rows, context)
+        return self._middle(idx, context)
+
+    def _bottom(self, context):
+        # M_0 on its own: one forward per token, each token drawn from the row just computed
+        st = self.stats[0]
+        serial = self._next_serial(0)
+        n_draft = self.T[0] if self.K > 0 else 1
+        tokens, rows = [], []
+        for j in range(n_draft):
+            row = self.model.rows(0, context + tokens, [])[0]
+            tokens.append(self.dec.draft_sample(row, j, serial, 0))
+            rows.append(row)
+            st.rows += 1
+        st.calls += 1
+        st.emitted += n_draft
+        self.trace.append((0, serial, len(context), 0, n_draft, tuple(tokens)))
         return tokens, rows
+
+    def _middle(self, idx, context):
+        # keep drafting (below) and verifying (here) behind what has been collected, until T_idx tokens are in hand
+        held_tokens, held_rows = [], []
+        while len(held_tokens) < self.T[idx]:
+            ctx = context + held_tokens
+            d_tok, d_rows = self.hsd(idx - 1, ctx)
+            v_tok, v_rows = self._verify(idx, d_tok, d_rows, ctx)
+            held_tokens += v_tok
+            held_rows += v_rows
+        return held_tokens, held_rows
 
     def _verify(self, idx, d_tok, d_rows, ctx):
         serial = self._next_serial(idx)

@@ -7,10 +7,10 @@ with a dummy alpha_{-1,0}; the corollary sums to |sigma|): the proof's recursion
     cost(k) = gamma(alpha_{k-1,k}, T_{k-1}, T_k) * (cost(k-1) + c_k)       0 < k < K
     L       = (1 - a) / (1 - a^(T_{K-1}+1)) * (cost(K-1) + c_K),  a = alpha_{K-1,K}
 
-gamma(alpha, T_in, T_out) is "the expected number of draft and verification
-rounds" until a level that needs T_out tokens has them when each round offers
-T_in drafts; the paper gives no formula ("we estimate ... empirically").  Reading
-used here: acceptances are IID with rate alpha (the paper's standing assumption),
+gamma(alpha, T_in, T_out) counts, in expectation, the draft-and-verify rounds a
+level goes through until it holds the T_out tokens it needs when each round offers
+T_in drafts; the paper gives no formula for it (it says the value was measured).
+Reading used here: acceptances are IID with rate alpha (the paper's standing assumption),
 a round yields Y = k tokens with probability alpha^(k-1) (1 - alpha) for
 k = 1..T_in and T_in + 1 with probability alpha^T_in, and gamma is the expected
 number of rounds until the yields sum to at least T_out.

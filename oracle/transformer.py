@@ -180,3 +180,26 @@ class Transformer:
         """Same rows with every cache dropped first (the definition)."""
         self.reset()
         return self.rows(level, context, draft_tokens)
+
+
+class ModelStack:
+    """M_0..M_K as separate models over one vocabulary (Section 3.1: the hierarchy is any list of models with
+    costs c_i; early exits of one decoder, as in Section 5.1, are one way to get such a list).  Level i is the
+    whole of models[i] (a Transformer whose last exit is its full depth), with its own memoised keys / values.
+    Same interface as Transformer towards Algorithm 1 / Algorithm 2: n_levels, rows(level, context, drafts)."""
+
+    def __init__(self, models):
+        self.models = list(models)
+        self.n_levels = len(self.models)
+        self.last_logits64 = None
+
+    def reset(self):
+        for m in self.models:
+            m.reset()
+        self.last_logits64 = None
+
+    def rows(self, level, context, draft_tokens):
+        m = self.models[level]
+        out = m.rows(m.n_levels - 1, context, draft_tokens)
+        self.last_logits64 = m.last_logits64
+        return out

@@ -149,6 +149,12 @@ def _declare_engine(lib):
     lib.hsd_create.restype = i32
     lib.hsd_create.argtypes = [c.POINTER(_ModelDesc), c.POINTER(c.c_int32), i32, c.POINTER(c.c_int32), vp, sz,
                                c.POINTER(vp)]
+    lib.hsd_models_workspace_bytes.restype = sz
+    lib.hsd_models_workspace_bytes.argtypes = [c.POINTER(_ModelDesc), i32, c.POINTER(c.c_int32)]
+    lib.hsd_create_models.restype = i32
+    lib.hsd_create_models.argtypes = [c.POINTER(_ModelDesc), i32, c.POINTER(c.c_int32), vp, sz, c.POINTER(vp)]
+    lib.hsd_set_phase_folding.restype = i32
+    lib.hsd_set_phase_folding.argtypes = [vp, i32, i32, i32]
     lib.hsd_generate.restype = i32
     lib.hsd_generate.argtypes = [vp, vp, i32, i32, i32, u64, vp, vp, c.POINTER(LevelStats), c.POINTER(c.c_double)]
     lib.hsd_set_trace.restype = i32
@@ -186,44 +192,74 @@ def _declare_engine(lib):
     lib.hsd_gemm_status.argtypes = [vp, vp]
 
 
-class Hsd:
-    """A hierarchy M_0..M_K of early exits of one decoder (hsd_create / hsd_generate / hsd_destroy).
+def _model_desc(cfg, weights, max_batch, max_seq, page_size):
+    """(hsd_model_desc, the host pointer array it refers to) for one decoder."""
+    n_layers = cfg["n_layers"]
+    ptrs = (ctypes.c_void_p * (n_layers * 9))()
+    for l, layer in enumerate(weights["layers"]):
+        for k, name in enumerate(_LAYER_KEYS):
+            t = layer[name]
+            assert t.is_cuda and t.is_contiguous()
+            ptrs[l * 9 + k] = t.data_ptr()
+    d = _ModelDesc(n_layers, cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"],
+                   cfg["vocab"], HSD_BF16 if cfg["dtype"] == "bf16" else HSD_F32, cfg["rms_eps"],
+                   cfg["rope_theta"], max_batch, max_seq, page_size, weights["embed"].data_ptr(),
+                   weights["final_norm"].data_ptr(), weights["lm_head"].data_ptr(), ptrs)
+    return d, ptrs
 
-    cfg: dict as produced by inputs.model_cfg; weights: dict of CUDA tensors (inputs.make_weights);
-    exits: exit layer per level (last == n_layers); T: T_0..T_{K-1}."""
+
+class Hsd:
+    """A hierarchy M_0..M_K (hsd_create / hsd_create_models, hsd_generate, hsd_destroy).
+
+    Early exits of one decoder: cfg = dict as produced by inputs.model_cfg, weights = dict of CUDA tensors
+    (inputs.make_weights), exits = exit layer per level (last == n_layers).
+    Separate models: cfg and weights are LISTS with one entry per level (the last is the target), exits = None.
+    T: T_0..T_{K-1}."""
 
     def __init__(self, cfg, weights, exits, T, max_batch, max_seq, page_size=16):
         lib = library()
         _declare_engine(lib)
         self._lib = lib
-        self.cfg, self.exits, self.T = dict(cfg), list(exits), list(T)
+        self.T = list(T)
         self.weights = weights                      # keep the device buffers alive
-        n_layers = cfg["n_layers"]
-        ptrs = (ctypes.c_void_p * (n_layers * 9))()
-        for l, layer in enumerate(weights["layers"]):
-            for k, name in enumerate(_LAYER_KEYS):
-                t = layer[name]
-                assert t.is_cuda and t.is_contiguous()
-                ptrs[l * 9 + k] = t.data_ptr()
-        self._ptrs = ptrs
-        d = _ModelDesc(n_layers, cfg["d_model"], cfg["n_q_heads"], cfg["n_kv_heads"], cfg["head_dim"], cfg["d_ff"],
-                       cfg["vocab"], HSD_BF16 if cfg["dtype"] == "bf16" else HSD_F32, cfg["rms_eps"],
-                       cfg["rope_theta"], max_batch, max_seq, page_size, weights["embed"].data_ptr(),
-                       weights["final_norm"].data_ptr(), weights["lm_head"].data_ptr(), ptrs)
-        self._desc = d
-        n_levels = len(self.exits)
-        ex = (ctypes.c_int32 * n_levels)(*self.exits)
-        tt = (ctypes.c_int32 * max(1, n_levels - 1))(*(self.T or [1]))
-        need = lib.hsd_workspace_bytes(ctypes.byref(d), ex, n_levels, tt)
-        if need == 0:
-            raise HsdError("hsd_workspace_bytes rejected the configuration")
-        self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=weights["embed"].device)
-        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        tt = (ctypes.c_int32 * max(1, len(self.T)))(*(self.T or [1]))
         ctx = ctypes.c_void_p()
-        _check(lib.hsd_create(ctypes.byref(d), ex, n_levels, tt, ctypes.c_void_p(base), need, ctypes.byref(ctx)))
+        if exits is None:
+            cfgs, ws = list(cfg), list(weights)
+            n_levels = len(cfgs)
+            descs = (_ModelDesc * n_levels)()
+            self._ptrs = []
+            for i in range(n_levels):
+                descs[i], ptrs = _model_desc(cfgs[i], ws[i], max_batch, max_seq, page_size)
+                self._ptrs.append(ptrs)
+            self._desc = descs
+            self.cfg, self.exits = dict(cfgs[-1]), [c["n_layers"] for c in cfgs]
+            need = lib.hsd_models_workspace_bytes(descs, n_levels, tt)
+            dev = ws[-1]["embed"].device
+        else:
+            self.cfg, self.exits = dict(cfg), list(exits)
+            n_levels = len(self.exits)
+            d, self._ptrs = _model_desc(cfg, weights, max_batch, max_seq, page_size)
+            self._desc = d
+            ex = (ctypes.c_int32 * n_levels)(*self.exits)
+            need = lib.hsd_workspace_bytes(ctypes.byref(d), ex, n_levels, tt)
+            dev = weights["embed"].device
+        if need == 0:
+            raise HsdError("the workspace-size call rejected the configuration")
+        self.workspace = torch.empty(need + 256, dtype=torch.uint8, device=dev)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        if exits is None:
+            _check(lib.hsd_create_models(self._desc, n_levels, tt, ctypes.c_void_p(base), need, ctypes.byref(ctx)))
+        else:
+            _check(lib.hsd_create(ctypes.byref(self._desc), ex, n_levels, tt, ctypes.c_void_p(base), need, ctypes.byref(ctx)))
         self._ctx = ctx
         self.n_levels = n_levels
         self.workspace_bytes = need
+
+    def set_phase_folding(self, fold_qkv=True, fold_gate_up=True, early_norm=True):
+        """hsd_set_phase_folding: keep (False) or fold (True) the two finish phases of decode passes; keep (False) or
+        drop (True) the grid barrier between a residual projection and its norm."""
+        _check(self._lib.hsd_set_phase_folding(self._ctx, int(bool(fold_qkv)), int(bool(fold_gate_up)), int(bool(early_norm))))
 
     def set_exit_heads(self, heads):
         """heads: list over levels of None (shared head) or dict(lm_head[, final_norm]) of CUDA tensors in the

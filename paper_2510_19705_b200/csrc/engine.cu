@@ -37,104 +37,137 @@ int device_sm_count() {
 }
 size_t elem_size(int dtype) { return dtype == HSD_BF16 ? 2 : 4; }
 
-// Workspace layout, shared by hsd_workspace_bytes and hsd_create.
+// Workspace layout, shared by the workspace-size calls and the create calls.  One part per model (its KV
+// pools, activations, rotary tables, tensor-core scratch) and one part that all levels share (token buffer,
+// page table, per-level logits rows, decision scratch, descriptor ring).
+struct ModelLayout {
+  size_t cos_tab, sin_tab, k_pool, v_pool, pool_layer_stride, x, h, qkv, q, att, act, partials, hf, tc_scratch,
+      tc_pieces_bytes, tc_pieces2, wmaps_dev, layers_dev, attn_counters, prof;
+  int partial_rows;
+};
 struct Layout {
-  size_t tokens, cos_tab, sin_tab, page_table, k_pool, v_pool, pool_layer_stride, x, h, qkv, q, att, act, partials, hf,
-      vscratch, n_acc, ring, tc_scratch, tc_pieces_bytes, tc_pieces2, wmaps_dev, layers_dev, attn_counters, grid_counter, prof, total;
+  size_t tokens, page_table, vscratch, n_acc, ring, grid_counter, total;
   std::vector<size_t> logits;
   std::vector<int> slots;
-  int max_rows, pages_per_seq, n_pages, partial_rows;
+  std::vector<ModelLayout> model;
+  int max_rows, pages_per_seq, n_pages, max_logit_rows;
   size_t ring_slot;
 };
 
-bool valid_model(const hsd_model_desc *m, const int32_t *exits, int n_levels, const int32_t *T) {
-  if (!m || !exits || n_levels < 1 || n_levels > 16) return false;
-  if (n_levels > 1 && !T) return false;
+bool valid_dims(const hsd_model_desc *m) {
+  if (!m) return false;
   if (m->n_layers < 1 || m->d_model < 8 || m->n_q_heads < 1 || m->n_kv_heads < 1 || m->head_dim < 2 || m->d_ff < 8 ||
       m->vocab < 2)
     return false;
   if (m->dtype != HSD_F32 && m->dtype != HSD_BF16) return false;
   if (m->max_batch < 1 || m->max_seq < 4 || m->page_size < 0) return false;
   if (m->n_q_heads % m->n_kv_heads != 0 || (m->head_dim & 1)) return false;
-  for (int i = 0; i < n_levels; ++i) {
-    if (exits[i] < 1 || exits[i] > m->n_layers) return false;
-    if (i > 0 && exits[i] <= exits[i - 1]) return false;
-  }
-  if (exits[n_levels - 1] != m->n_layers) return false;
+  return true;
+}
+bool valid_T(int n_levels, const int32_t *T) {
+  if (n_levels < 1 || n_levels > 16) return false;
+  if (n_levels > 1 && !T) return false;
   for (int i = 0; i + 1 < n_levels; ++i)
     if (T[i] < 1 || T[i] > 64) return false;
   return true;
 }
+// One decoder, levels = early exits.
+bool valid_model(const hsd_model_desc *m, const int32_t *exits, int n_levels, const int32_t *T) {
+  if (!valid_dims(m) || !exits || !valid_T(n_levels, T)) return false;
+  for (int i = 0; i < n_levels; ++i) {
+    if (exits[i] < 1 || exits[i] > m->n_layers) return false;
+    if (i > 0 && exits[i] <= exits[i - 1]) return false;
+  }
+  return exits[n_levels - 1] == m->n_layers;
+}
+// One model per level: what the levels must have in common (vocabulary, storage type, capacity, page size).
+bool valid_models(const hsd_model_desc *ms, int n_levels, const int32_t *T) {
+  if (!ms || !valid_T(n_levels, T)) return false;
+  for (int i = 0; i < n_levels; ++i) {
+    if (!valid_dims(&ms[i])) return false;
+    if (ms[i].vocab != ms[0].vocab || ms[i].dtype != ms[0].dtype || ms[i].max_batch != ms[0].max_batch ||
+        ms[i].max_seq != ms[0].max_seq || ms[i].page_size != ms[0].page_size)
+      return false;
+  }
+  return true;
+}
 
-Layout make_layout(const hsd_model_desc *m, int n_levels, const int32_t *T) {
+Layout make_layout(const hsd_model_desc *models, int n_models, int n_levels, const int32_t *T) {
   Layout L;
-  const size_t es = elem_size(m->dtype);
-  const int page = m->page_size ? m->page_size : 16;
-  const int B = m->max_batch, d = m->d_model, hd = m->head_dim, nq = m->n_q_heads, nkv = m->n_kv_heads;
+  const hsd_model_desc *m0 = &models[0];
+  const size_t es = elem_size(m0->dtype);
+  const int page = m0->page_size ? m0->page_size : 16;
+  const int B = m0->max_batch;
   int sumT = 0;
   L.slots.resize(n_levels);
   for (int i = 0; i < n_levels; ++i) {
     if (i + 1 < n_levels) sumT += T[i];
-    L.slots[i] = (i + 1 < n_levels ? sumT : sumT) + 1;      // level i keeps at most sum_{j<=i} T_j (+1) rows
+    L.slots[i] = sumT + 1;                                  // level i keeps at most sum_{j<=i} T_j (+1) rows
   }
   if (n_levels == 1) L.slots[0] = 1;
   // rows of one forward: drafts of the level below + catch-up rows (<= n_levels), per sequence
   int decode_rows = B * (sumT + n_levels + 1);
   L.max_rows = std::max(kPrefillRows, decode_rows);
-  L.pages_per_seq = (m->max_seq + page - 1) / page;
+  L.pages_per_seq = (m0->max_seq + page - 1) / page;
   L.n_pages = B * L.pages_per_seq;
-  L.partial_rows = std::max(L.max_rows + kAttnRows * kAttnBlocksTarget / nkv + kAttnRows * kMaxSplits,
-                            L.max_rows * 20);   // the persistent forward may cut every row's keys into up to 20 splits
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  L.tokens = take((size_t)B * m->max_seq * 4);
-  L.cos_tab = take((size_t)m->max_seq * (hd / 2) * 4);
-  L.sin_tab = take((size_t)m->max_seq * (hd / 2) * 4);
+  L.tokens = take((size_t)B * m0->max_seq * 4);
   L.page_table = take((size_t)B * L.pages_per_seq * 4);
-  L.pool_layer_stride = align_up((size_t)L.n_pages * nkv * page * hd * es, 256);
-  L.k_pool = take(L.pool_layer_stride * m->n_layers);
-  L.v_pool = take(L.pool_layer_stride * m->n_layers);
-  L.x = take((size_t)L.max_rows * d * 4);
-  L.h = take((size_t)L.max_rows * d * es);
-  L.qkv = take((size_t)L.max_rows * (nq + 2 * nkv) * hd * 4);
-  L.q = take((size_t)L.max_rows * nq * hd * es);
-  L.att = take((size_t)L.max_rows * nq * hd * es);
-  L.act = take((size_t)L.max_rows * m->d_ff * es);
-  L.partials = take((size_t)L.partial_rows * nq * (hd + 2) * 4);
-  int max_logit_rows = 0;
+  L.max_logit_rows = 0;
   L.logits.resize(n_levels);
   for (int i = 0; i < n_levels; ++i) {
-    L.logits[i] = take((size_t)B * L.slots[i] * m->vocab * es);
-    max_logit_rows = std::max(max_logit_rows, B * L.slots[i]);
+    L.logits[i] = take((size_t)B * L.slots[i] * m0->vocab * es);
+    L.max_logit_rows = std::max(L.max_logit_rows, B * L.slots[i]);
   }
-  L.hf = take((size_t)max_logit_rows * d * es);
   L.vscratch = take(verify_scratch_bytes(B, sumT + 1));
   L.n_acc = take((size_t)B * 4);
   L.ring_slot = align_up((size_t)L.max_rows * 40 + (size_t)B * 96 + 1024, 256);
   L.ring = take(L.ring_slot * kRingSlots);
-  // tensor-core GEMM scratch: [status word | per-tile counters (16 KiB)] + split pieces (largest plan)
-  L.tc_pieces_bytes = 0;
-  if (m->dtype == HSD_BF16) {
-    const int sms = device_sm_count();
-    const int npads[4] = {16, 32, 64, 128};
-    const int shapes[5][4] = {{nq * hd, nkv * hd, nkv * hd, d}, {d, 0, 0, nq * hd}, {m->d_ff, m->d_ff, 0, d},
-                              {d, 0, 0, m->d_ff}, {m->vocab, 0, 0, d}};
-    const int modes[5] = {GEMM_STORE_F32, GEMM_ADD_F32, GEMM_SWIGLU_T, GEMM_ADD_F32, GEMM_STORE_T_SCATTER};
-    for (int g = 0; g < 5; ++g)
-      for (int np : npads) {
-        if (shapes[g][3] % kTcBlockK) continue;
-        int nsegs = shapes[g][2] ? 3 : (shapes[g][1] ? 2 : 1);
-        TcGemmPlan pl = tc_plan(shapes[g], nsegs, modes[g], shapes[g][3], np, sms);
-        L.tc_pieces_bytes = std::max(L.tc_pieces_bytes, pl.scratch_bytes);
-      }
-  }
-  L.tc_scratch = take(kTcCtrlBytes + L.tc_pieces_bytes);
-  L.tc_pieces2 = take(L.tc_pieces_bytes);       // second piece buffer (down projection of passes with few rows)
-  L.wmaps_dev = take(((size_t)m->n_layers * 7 + kHeadMaps) * sizeof(CUtensorMap));
-  L.layers_dev = take((size_t)m->n_layers * sizeof(FwdLayerDev));
-  L.attn_counters = take(16384);
   L.grid_counter = take(256);
-  L.prof = take((size_t)device_sm_count() * kFwdProfEvents * 8);
+  L.model.resize(n_models);
+  for (int mi = 0; mi < n_models; ++mi) {
+    const hsd_model_desc *m = &models[mi];
+    ModelLayout &M = L.model[mi];
+    const int d = m->d_model, hd = m->head_dim, nq = m->n_q_heads, nkv = m->n_kv_heads;
+    M.partial_rows = std::max(L.max_rows + kAttnRows * kAttnBlocksTarget / nkv + kAttnRows * kMaxSplits,
+                              L.max_rows * 20);   // the persistent forward may cut every row's keys into up to 20 splits
+    M.cos_tab = take((size_t)m->max_seq * (hd / 2) * 4);
+    M.sin_tab = take((size_t)m->max_seq * (hd / 2) * 4);
+    M.pool_layer_stride = align_up((size_t)L.n_pages * nkv * page * hd * es, 256);
+    M.k_pool = take(M.pool_layer_stride * m->n_layers);
+    M.v_pool = take(M.pool_layer_stride * m->n_layers);
+    M.x = take((size_t)L.max_rows * d * 4);
+    M.h = take((size_t)L.max_rows * d * es);
+    M.qkv = take((size_t)L.max_rows * (nq + 2 * nkv) * hd * 4);
+    M.q = take((size_t)L.max_rows * nq * hd * es);
+    M.att = take((size_t)L.max_rows * nq * hd * es);
+    M.act = take((size_t)L.max_rows * m->d_ff * es);
+    M.partials = take((size_t)M.partial_rows * nq * (hd + 2) * 4);
+    M.hf = take((size_t)L.max_logit_rows * d * es);
+    // tensor-core GEMM scratch: [status word | per-tile counters (16 KiB)] + split pieces (largest plan)
+    M.tc_pieces_bytes = 0;
+    if (m->dtype == HSD_BF16) {
+      const int sms = device_sm_count();
+      const int npads[4] = {16, 32, 64, 128};
+      const int shapes[5][4] = {{nq * hd, nkv * hd, nkv * hd, d}, {d, 0, 0, nq * hd}, {m->d_ff, m->d_ff, 0, d},
+                                {d, 0, 0, m->d_ff}, {m->vocab, 0, 0, d}};
+      const int modes[5] = {GEMM_STORE_F32, GEMM_ADD_F32, GEMM_SWIGLU_T, GEMM_ADD_F32, GEMM_STORE_T_SCATTER};
+      for (int g = 0; g < 5; ++g)
+        for (int np : npads) {
+          if (shapes[g][3] % kTcBlockK) continue;
+          int nsegs = shapes[g][2] ? 3 : (shapes[g][1] ? 2 : 1);
+          TcGemmPlan pl = tc_plan(shapes[g], nsegs, modes[g], shapes[g][3], np, sms);
+          M.tc_pieces_bytes = std::max(M.tc_pieces_bytes, pl.scratch_bytes);
+        }
+    }
+    M.tc_scratch = take(kTcCtrlBytes + M.tc_pieces_bytes);
+    M.tc_pieces2 = take(M.tc_pieces_bytes);       // second piece buffer (down projection of passes with few rows)
+    M.wmaps_dev = take(((size_t)m->n_layers * 7 + kHeadMaps) * sizeof(CUtensorMap));
+    M.layers_dev = take((size_t)m->n_layers * sizeof(FwdLayerDev));
+    M.attn_counters = take(16384);
+    M.prof = take((size_t)device_sm_count() * kFwdProfEvents * 8);
+  }
   L.total = off;
   return L;
 }
@@ -149,14 +182,28 @@ struct TimerPair { cudaEvent_t a, b; int level; };
 
 }  // namespace
 
-struct hsd_ctx {
+// One decoder: its geometry, weights, part of the workspace and tensor-core state.  A hierarchy of early exits
+// has one (every level runs its first exits[level] layers); a hierarchy of separate models has one per level.
+struct Model {
   ModelDims md;
-  int n_levels, max_batch;
-  std::vector<int> exits, T;
-  Layout lay;
-  char *ws;
+  ModelLayout lay;
   const void *embed, *final_norm, *lm_head;
   std::vector<const void *> lw;
+  bool use_tc = false, use_persist = false;   // tensor-core GEMMs / the one-launch persistent forward (bf16 models)
+  std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + kHeadMaps]: wq wk wv wo wg wu wd per layer, then the levels' heads, the shared head
+  CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
+  CUtensorMap amaps_rows[4][16];              // the same buffers with a box of exactly 1..16 rows (persistent forward, few rows)
+};
+
+struct hsd_ctx {
+  ModelDims md;                               // what all levels share is read from here: V, dtype, max_seq, page, pages_per_seq
+  int n_levels, max_batch;
+  std::vector<int> exits, T;                  // exits[level] = layers the level runs of its model
+  std::vector<Model> models;
+  std::vector<int> level_model;               // model of each level (all 0 for early exits of one decoder)
+  bool shared_cache = true;                   // early exits: level i's pass also refreshes the KV of the levels below it
+  Layout lay;
+  char *ws;
   // pinned host mirrors
   char *ring_host;
   int *n_acc_host;
@@ -179,18 +226,17 @@ struct hsd_ctx {
   int trace_logit_calls, trace_records;
   cudaStream_t stream;
   uint64_t seed;
-  // tensor-core GEMM state (bf16 models)
-  bool use_tc, use_persist;
-  int attn_single_max = 0;                    // contexts up to this many keys use one attention key split
-  bool no_fuse_qkv = false;                   // debugging aid (HSD_NO_FUSE_QKV): keep the QKV finish phase in every pass
-  bool no_fuse_gu = false;                    // debugging aid (HSD_NO_FUSE_GU): keep the gate / up finish phase in every pass
+  bool any_tc = false;                        // some model runs the tensor-core kernels (their status word is polled)
+  bool no_fuse_qkv = false;                   // keep the QKV finish phase in every pass (hsd_set_phase_folding)
+  bool no_fuse_gu = false;                    // keep the gate / up finish phase in every pass
+  bool no_early_norm = false;                 // keep the grid barrier between a residual projection and its norm
   int sm_count;
-  std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + kHeadMaps]: wq wk wv wo wg wu wd per layer, then the levels' heads, the shared head
-  std::vector<const void *> level_head, level_norm;   // output head and final norm gain of each level (shared unless set)
+  std::vector<const void *> level_head, level_norm;   // output head and final norm gain of each level (the model's own unless set)
   std::vector<uint32_t> coin24;               // per level: kNoCoin, or the IID acceptance probability x 2^24 (ablation)
-  CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
-  CUtensorMap amaps_rows[4][16];              // the same buffers with a box of exactly 1..16 rows (persistent forward, few rows)
   int *status_host;
+  size_t status_off;                          // the one status word every tensor-core kernel of the context raises
+
+  Model &model_of(int level) { return models[level_model[level]]; }
 
   template <typename U> U *dev(size_t off) const { return reinterpret_cast<U *>(ws + off); }
 };
@@ -198,11 +244,11 @@ struct hsd_ctx {
 namespace {
 
 int sync_stream(hsd_ctx *c) {
-  if (c->use_tc &&
-      cudaMemcpyAsync(c->status_host, c->ws + c->lay.tc_scratch, 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
+  if (c->any_tc &&
+      cudaMemcpyAsync(c->status_host, c->ws + c->status_off, 4, cudaMemcpyDeviceToHost, c->stream) != cudaSuccess)
     return HSD_E_CUDA;
   if (cudaStreamSynchronize(c->stream) != cudaSuccess) return HSD_E_CUDA;
-  if (c->use_tc && *c->status_host != 0) return HSD_E_DEVICE_TIMEOUT;
+  if (c->any_tc && *c->status_host != 0) return HSD_E_DEVICE_TIMEOUT;
   c->ring_in_flight = 0;
   for (int i = 0; i < c->timers_used; ++i) {
     float ms = 0.f;
@@ -264,14 +310,14 @@ int upload_page_tables(hsd_ctx *c) {
 // Matrix product of the forward pass: tensor cores for bf16 models, CUDA cores otherwise.
 // abuf names the activation buffer A lives in (0 = h, 1 = att, 2 = act, 3 = hf); wmap0 the index of
 // the first segment's tensor map.
-int gemm(hsd_ctx *c, int abuf, const void *A, int R, int K, const GemmSegs &segs, int wmap0, int mode, float *out_f32,
+int gemm(hsd_ctx *c, Model &M, int abuf, const void *A, int R, int K, const GemmSegs &segs, int wmap0, int mode, float *out_f32,
          void *out_t, const long long *dst) {
-  if (!c->use_tc) return launch_gemm_simt(c->md, A, R, K, segs, mode, out_f32, out_t, dst, c->stream);
+  if (!M.use_tc) return launch_gemm_simt(M.md, A, R, K, segs, mode, out_f32, out_t, dst, c->stream);
   TcGemmArgs a;
   int total = 0;
   for (int i = 0; i < 3; ++i) {
     a.seg_n[i] = i < segs.count ? segs.n[i] : 0;
-    if (i < segs.count) a.w[i] = c->wmaps[wmap0 + i];
+    if (i < segs.count) a.w[i] = M.wmaps[wmap0 + i];
     total += a.seg_n[i];
   }
   a.n_segs = segs.count;
@@ -281,14 +327,14 @@ int gemm(hsd_ctx *c, int abuf, const void *A, int R, int K, const GemmSegs &segs
   a.out_bf16 = (__nv_bfloat16 *)out_t;
   a.dst = dst;
   a.ldo = (mode == GEMM_SWIGLU_T) ? segs.n[0] : total;
-  a.status = (int *)(c->ws + c->lay.tc_scratch);
-  a.counters = (int *)(c->ws + c->lay.tc_scratch + 256);
-  a.pieces = (float *)(c->ws + c->lay.tc_scratch + kTcCtrlBytes);
+  a.status = (int *)(c->ws + c->status_off);
+  a.counters = (int *)(c->ws + M.lay.tc_scratch + 256);
+  a.pieces = (float *)(c->ws + M.lay.tc_scratch + kTcCtrlBytes);
   for (int r0 = 0; r0 < R; r0 += 128) {
     a.R = std::min(128, R - r0);
     a.row0 = r0;
     int np = tc_npad(a.R);
-    a.a = c->amaps[abuf][np == 16 ? 0 : np == 32 ? 1 : np == 64 ? 2 : 3];
+    a.a = M.amaps[abuf][np == 16 ? 0 : np == 32 ? 1 : np == 64 ? 2 : 3];
     int st = launch_gemm_tc(a, c->sm_count, c->stream);
     if (st) return st;
   }
@@ -298,11 +344,13 @@ int gemm(hsd_ctx *c, int abuf, const void *A, int R, int K, const GemmSegs &segs
 // One forward pass of level `level` (layers 1..exit) over the given rows; logits of the wanted
 // rows go to the level's logits buffer.  KV of every processed position is (re)written.
 int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
-  const ModelDims &md = c->md;
+  Model &M = c->model_of(level);
+  const ModelDims &md = M.md;
   const Layout &L = c->lay;
+  const ModelLayout &ML = M.lay;
   int R = 0, n_attn = 0, n_logit = 0, max_kv = 0;
   bool one_item_per_seq = true;
-  const int arows = c->use_persist ? fwd_attn_rows(md.nq / md.nkv, md.hd) : kAttnRows;   // rows per attention item
+  const int arows = M.use_persist ? fwd_attn_rows(md.nq / md.nkv, md.hd) : kAttnRows;   // rows per attention item
   for (const SeqWork &w : work) {
     int rows = w.end - w.start;
     if (rows <= 0 || w.start < 0 || w.end > md.max_seq) return HSD_E_INVALID_ARG;
@@ -351,7 +399,7 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   // 16-row query tiles), so that a CTA's items sample the whole cost range.
   const int qgroup = md.nq / md.nkv;
   auto item_cost = [&](const int4 &it) { return (long long)(it.w + it.y) * ((it.y * qgroup + 15) / 16); };
-  if (c->use_persist && n_attn > 1)
+  if (M.use_persist && n_attn > 1)
     std::stable_sort(attn, attn + n_attn, [&](const int4 &x, const int4 &y) { return item_cost(x) > item_cost(y); });
   HSD_CUDA_OK(cudaMemcpyAsync(devp, host, bytes, cudaMemcpyHostToDevice, c->stream));
   st = upload_page_tables(c);
@@ -368,12 +416,10 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   rb.lrow_dst = (const long long *)(devp + o_dst);
 
   // attention split: enough blocks to fill the GPU, never more partial rows than the buffer holds
-  const int blocks_target = c->use_persist ? c->sm_count : kAttnBlocksTarget;
-  int max_splits = c->use_persist ? 20 : kMaxSplits;      // the persistent merge phase takes <= 20 splits
-  if (c->use_persist) if (const char *e = getenv("HSD_ATTN_SPLITS_MAX")) max_splits = std::max(1, std::min(20, atoi(e)));
+  const int blocks_target = M.use_persist ? c->sm_count : kAttnBlocksTarget;
+  const int max_splits = M.use_persist ? 20 : kMaxSplits;      // the persistent merge phase takes <= 20 splits
   int n_splits = std::max(1, std::min(max_splits, blocks_target / std::max(1, n_attn * md.nkv)));
-  if (c->use_persist && max_kv <= c->attn_single_max) n_splits = 1;   // short contexts: one split, no merge phase
-  if (c->use_persist && max_kv >= 2048) {
+  if (M.use_persist && max_kv >= 2048) {
     // Long contexts: the key loop dominates and the items differ in cost, so the split count is chosen by a
     // small model of the tiles phase: a work unit (item, KV head, split) costs a fixed part plus its keys x
     // query tiles, units go to the CTAs round-robin in item order (as the kernel deals them), the phase lasts
@@ -411,9 +457,9 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     }
     n_splits = best_s;
   }
-  int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, c->use_persist ? 16 : kAttnKeyTile);
+  int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, M.use_persist ? 16 : kAttnKeyTile);
   n_splits = (max_kv + keys_per_split - 1) / keys_per_split;
-  if ((size_t)R * n_splits > (size_t)L.partial_rows) return HSD_E_INVALID_ARG;
+  if ((size_t)R * n_splits > (size_t)ML.partial_rows) return HSD_E_INVALID_ARG;
 
   TimerPair *tp = nullptr;
   if (c->timers_ok && c->timers_used < kTimerPairs) {
@@ -422,7 +468,13 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     cudaEventRecord(tp->a, c->stream);
   }
   cudaStream_t s = c->stream;
-  if (c->use_persist && R <= 128 && n_logit <= 128) {
+  auto mark_valid = [&]() {
+    // the pass (re)wrote the KV of its rows in every layer it ran: with early exits that covers the caches of
+    // the levels below as well (they ARE the first layers); a separate model has a cache of its own
+    for (const SeqWork &w : work)
+      for (int g = c->shared_cache ? 0 : level; g <= level; ++g) c->len_g[w.b][g] = w.end;
+  };
+  if (M.use_persist && R <= 128 && n_logit <= 128) {
     // one cooperative launch runs the whole pass
     FwdArgs a;
     a.d = md.d; a.nq = md.nq; a.nkv = md.nkv; a.hd = md.hd; a.ff = md.ff; a.V = md.V;
@@ -430,20 +482,20 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     a.page_shift = 0;
     while ((1 << a.page_shift) < md.page) ++a.page_shift;
     a.pages_per_seq = md.pages_per_seq; a.eps = md.eps;
-    a.wmaps = c->dev<CUtensorMap>(L.wmaps_dev);
-    a.layers = c->dev<FwdLayerDev>(L.layers_dev);
-    a.embed = (const __nv_bfloat16 *)c->embed; a.final_norm = (const __nv_bfloat16 *)c->level_norm[level];
-    a.cos_tab = c->dev<float>(L.cos_tab); a.sin_tab = c->dev<float>(L.sin_tab);
+    a.wmaps = c->dev<CUtensorMap>(ML.wmaps_dev);
+    a.layers = c->dev<FwdLayerDev>(ML.layers_dev);
+    a.embed = (const __nv_bfloat16 *)M.embed; a.final_norm = (const __nv_bfloat16 *)c->level_norm[level];
+    a.cos_tab = c->dev<float>(ML.cos_tab); a.sin_tab = c->dev<float>(ML.sin_tab);
     a.R = R; a.L = n_logit; a.n_attn = n_attn; a.attn_rows = arows; a.n_splits = n_splits; a.keys_per_split = keys_per_split;
     a.tokens = c->dev<int>(L.tokens); a.page_table = c->dev<int>(L.page_table);
     a.row_seq = rb.row_seq; a.row_pos = rb.row_pos; a.lrow_src = rb.lrow_src; a.attn_items = rb.attn; a.lrow_dst = rb.lrow_dst;
-    a.x = c->dev<float>(L.x);
-    a.h = c->dev<__nv_bfloat16>(L.h); a.q = c->dev<__nv_bfloat16>(L.q); a.att = c->dev<__nv_bfloat16>(L.att);
-    a.act = c->dev<__nv_bfloat16>(L.act); a.hf = c->dev<__nv_bfloat16>(L.hf);
+    a.x = c->dev<float>(ML.x);
+    a.h = c->dev<__nv_bfloat16>(ML.h); a.q = c->dev<__nv_bfloat16>(ML.q); a.att = c->dev<__nv_bfloat16>(ML.att);
+    a.act = c->dev<__nv_bfloat16>(ML.act); a.hf = c->dev<__nv_bfloat16>(ML.hf);
     a.logits = (__nv_bfloat16 *)(c->ws + L.logits[level]);
-    a.attn_partials = c->dev<float>(L.partials); a.attn_counters = c->dev<int>(L.attn_counters);
-    a.pieces = (float *)(c->ws + L.tc_scratch + kTcCtrlBytes); a.tile_counters = (int *)(c->ws + L.tc_scratch + 256);
-    a.grid_counter = c->dev<unsigned>(L.grid_counter); a.status = (int *)(c->ws + L.tc_scratch);
+    a.attn_partials = c->dev<float>(ML.partials); a.attn_counters = c->dev<int>(ML.attn_counters);
+    a.pieces = (float *)(c->ws + ML.tc_scratch + kTcCtrlBytes); a.tile_counters = (int *)(c->ws + ML.tc_scratch + 256);
+    a.grid_counter = c->dev<unsigned>(L.grid_counter); a.status = (int *)(c->ws + c->status_off);
     const int np = tc_npad(std::max(R, n_logit));
     const int pi = np == 16 ? 0 : np == 32 ? 1 : np == 64 ? 2 : 3;
     // few rows: fetch exactly the rows that exist (the MMA still reads `np` rows of the stage; the rest is stale
@@ -454,17 +506,25 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     a.fuse_qkv = (one_item_per_seq && !c->no_fuse_qkv) ? 1 : 0;
     // few rows: the SwiGLU finish folds into the down projection (its CTAs build their activation tiles)
     a.fuse_gu = (R <= 4 && !c->no_fuse_gu) ? 1 : 0;
-    a.pieces2 = (float *)(c->ws + L.tc_pieces2);
-    for (int b = 0; b < 4; ++b) a.amap[b] = box_rows <= 16 ? c->amaps_rows[b][box_rows - 1] : c->amaps[b][pi];
-    // debugging aid: HSD_PROFILE=<file> dumps the barrier timeline of the latest top-level pass
+    // the norms after the residual projections start on otherwise idle CTAs as soon as the pieces are there
+    a.early_norm = c->no_early_norm ? 0 : 1;
+    a.pieces2 = (float *)(c->ws + ML.tc_pieces2);
+    for (int b = 0; b < 4; ++b) a.amap[b] = box_rows <= 16 ? M.amaps_rows[b][box_rows - 1] : M.amaps[b][pi];
+    a.prof = nullptr;
+#ifdef HSD_PROFILE
+    // profiling build (-DHSD_PROFILE): HSD_PROFILE=<file> dumps the barrier timeline of the latest top-level pass
     const char *prof_path = getenv("HSD_PROFILE");
     const char *prof_rows = getenv("HSD_PROFILE_MIN_ROWS");       // e.g. 100: the prompt's chunks instead of decode passes
     const bool prof = prof_path && level == c->n_levels - 1 && (prof_rows ? R >= atoi(prof_rows) : n_logit > 0);
-    a.prof = prof ? c->dev<unsigned long long>(L.prof) : nullptr;
-    if (prof) HSD_CUDA_OK(cudaMemsetAsync(a.prof, 0, (size_t)c->sm_count * kFwdProfEvents * 8, s));
-    HSD_CUDA_OK(cudaMemsetAsync(a.grid_counter, 0, 4, s));
+    if (prof) {
+      a.prof = c->dev<unsigned long long>(ML.prof);
+      HSD_CUDA_OK(cudaMemsetAsync(a.prof, 0, (size_t)c->sm_count * kFwdProfEvents * 8, s));
+    }
+#endif
+    HSD_CUDA_OK(cudaMemsetAsync(a.grid_counter, 0, 128, s));
     int stp = launch_forward_persistent(a, np, c->sm_count, s);
     if (stp) return stp;
+#ifdef HSD_PROFILE
     if (prof) {
       std::vector<unsigned long long> ev((size_t)c->sm_count * kFwdProfEvents);
       if (cudaMemcpyAsync(ev.data(), a.prof, ev.size() * 8, cudaMemcpyDeviceToHost, s) == cudaSuccess &&
@@ -481,47 +541,46 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
         }
       }
     }
+#endif
     if (tp) cudaEventRecord(tp->b, s);
     c->stats[level].forwards++;
     c->stats[level].rows += R;
-    for (const SeqWork &w : work)
-      for (int g = 0; g <= level; ++g) c->len_g[w.b][g] = w.end;
+    mark_valid();
     return HSD_OK;
   }
-  float *x = c->dev<float>(L.x);
-  void *h = c->dev<void>(L.h), *q = c->dev<void>(L.q), *att = c->dev<void>(L.att), *act = c->dev<void>(L.act);
-  float *qkv = c->dev<float>(L.qkv);
+  float *x = c->dev<float>(ML.x);
+  void *h = c->dev<void>(ML.h), *q = c->dev<void>(ML.q), *att = c->dev<void>(ML.att), *act = c->dev<void>(ML.act);
+  float *qkv = c->dev<float>(ML.qkv);
   const int *pt = c->dev<int>(L.page_table);
 #define HSD_TRY(e) do { int st__ = (e); if (st__) return st__; } while (0)
-  HSD_TRY(launch_embed(md, c->embed, c->dev<int>(L.tokens), rb, x, s));
+  HSD_TRY(launch_embed(md, M.embed, c->dev<int>(L.tokens), rb, x, s));
   for (int l = 0; l < c->exits[level]; ++l) {
-    const void *const *w = &c->lw[(size_t)l * 9];
-    void *kp = c->ws + L.k_pool + L.pool_layer_stride * l, *vp = c->ws + L.v_pool + L.pool_layer_stride * l;
+    const void *const *w = &M.lw[(size_t)l * 9];
+    void *kp = c->ws + ML.k_pool + ML.pool_layer_stride * l, *vp = c->ws + ML.v_pool + ML.pool_layer_stride * l;
     HSD_TRY(launch_rmsnorm(md, x, w[0], nullptr, R, h, s));
     GemmSegs qkv_segs = {{w[1], w[2], w[3]}, {md.nq * md.hd, md.nkv * md.hd, md.nkv * md.hd}, 3};
-    HSD_TRY(gemm(c, 0, h, R, md.d, qkv_segs, l * 7 + 0, GEMM_STORE_F32, qkv, nullptr, nullptr));
-    HSD_TRY(launch_rope_kv(md, qkv, rb, c->dev<float>(L.cos_tab), c->dev<float>(L.sin_tab), pt, kp, vp, q, s));
-    HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(L.partials), keys_per_split, n_splits, att, s));
+    HSD_TRY(gemm(c, M, 0, h, R, md.d, qkv_segs, l * 7 + 0, GEMM_STORE_F32, qkv, nullptr, nullptr));
+    HSD_TRY(launch_rope_kv(md, qkv, rb, c->dev<float>(ML.cos_tab), c->dev<float>(ML.sin_tab), pt, kp, vp, q, s));
+    HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(ML.partials), keys_per_split, n_splits, att, s));
     GemmSegs o_segs = {{w[4], nullptr, nullptr}, {md.d, 0, 0}, 1};
-    HSD_TRY(gemm(c, 1, att, R, md.nq * md.hd, o_segs, l * 7 + 3, GEMM_ADD_F32, x, nullptr, nullptr));
+    HSD_TRY(gemm(c, M, 1, att, R, md.nq * md.hd, o_segs, l * 7 + 3, GEMM_ADD_F32, x, nullptr, nullptr));
     HSD_TRY(launch_rmsnorm(md, x, w[5], nullptr, R, h, s));
     GemmSegs gu_segs = {{w[6], w[7], nullptr}, {md.ff, md.ff, 0}, 2};
-    HSD_TRY(gemm(c, 0, h, R, md.d, gu_segs, l * 7 + 4, GEMM_SWIGLU_T, nullptr, act, nullptr));
+    HSD_TRY(gemm(c, M, 0, h, R, md.d, gu_segs, l * 7 + 4, GEMM_SWIGLU_T, nullptr, act, nullptr));
     GemmSegs d_segs = {{w[8], nullptr, nullptr}, {md.d, 0, 0}, 1};
-    HSD_TRY(gemm(c, 2, act, R, md.ff, d_segs, l * 7 + 6, GEMM_ADD_F32, x, nullptr, nullptr));
+    HSD_TRY(gemm(c, M, 2, act, R, md.ff, d_segs, l * 7 + 6, GEMM_ADD_F32, x, nullptr, nullptr));
   }
   if (n_logit > 0) {
-    void *hf = c->dev<void>(L.hf);
+    void *hf = c->dev<void>(ML.hf);
     HSD_TRY(launch_rmsnorm(md, x, c->level_norm[level], rb.lrow_src, n_logit, hf, s));
     GemmSegs lm_segs = {{c->level_head[level], nullptr, nullptr}, {md.V, 0, 0}, 1};
-    HSD_TRY(gemm(c, 3, hf, n_logit, md.d, lm_segs, md.n_layers * 7 + level, GEMM_STORE_T_SCATTER, nullptr, c->ws + L.logits[level],
+    HSD_TRY(gemm(c, M, 3, hf, n_logit, md.d, lm_segs, md.n_layers * 7 + level, GEMM_STORE_T_SCATTER, nullptr, c->ws + L.logits[level],
                  rb.lrow_dst));
   }
   if (tp) cudaEventRecord(tp->b, s);
   c->stats[level].forwards++;
   c->stats[level].rows += R;
-  for (const SeqWork &w : work)
-    for (int g = 0; g <= level; ++g) c->len_g[w.b][g] = w.end;
+  mark_valid();
   return HSD_OK;
 }
 
@@ -703,8 +762,148 @@ int prefill(hsd_ctx *c, int batch, int prompt_len) {
       budget -= rows;
     }
     if (work.empty()) break;
-    HSD_TRY(forward(c, K, work));
+    // early exits: the target's pass fills the one cache; separate models: each fills its own
+    for (int lvl = c->shared_cache ? K : 0; lvl <= K; ++lvl) HSD_TRY(forward(c, lvl, work));
   }
+  return HSD_OK;
+}
+
+// Sets up one model of a context: rotary tables, tensor maps, device-side tables.  `head_levels`: the levels whose
+// output-head tensor map slots are (re)built for this model.
+int init_model(hsd_ctx *c, Model &M, const hsd_model_desc *model, const ModelLayout &ml) {
+  const Layout &lay = c->lay;
+  M.md = ModelDims{model->n_layers, model->d_model, model->n_q_heads, model->n_kv_heads, model->head_dim, model->d_ff,
+                   model->vocab, model->dtype, model->rms_eps, model->rope_theta, model->max_seq,
+                   model->page_size ? model->page_size : 16, lay.pages_per_seq};
+  M.lay = ml;
+  M.embed = model->embed; M.final_norm = model->final_norm; M.lm_head = model->lm_head;
+  M.lw.assign(model->layer_weights, model->layer_weights + (size_t)model->n_layers * 9);
+  const ModelDims &md = M.md;
+  {  // rotary tables: angles in double, rounded to fp32
+    const int half = md.hd / 2;
+    std::vector<float> cs((size_t)md.max_seq * half), sn((size_t)md.max_seq * half);
+    for (int p = 0; p < md.max_seq; ++p)
+      for (int k = 0; k < half; ++k) {
+        double ang = (double)p * pow((double)md.theta, -2.0 * k / (double)md.hd);
+        cs[(size_t)p * half + k] = (float)cos(ang);
+        sn[(size_t)p * half + k] = (float)sin(ang);
+      }
+    if (cudaMemcpy(c->ws + ml.cos_tab, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(c->ws + ml.sin_tab, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess)
+      return HSD_E_CUDA;
+  }
+  // tensor-core path: bf16 model whose contraction sizes are multiples of the 64-element k-block
+  M.use_tc = model->dtype == HSD_BF16 && model->d_model % kTcBlockK == 0 && model->d_ff % kTcBlockK == 0 &&
+             (model->n_q_heads * model->head_dim) % kTcBlockK == 0 && tc_init() == HSD_OK;
+  if (!M.use_tc) return HSD_OK;
+  int st = HSD_OK;
+  M.wmaps.resize((size_t)md.n_layers * 7 + kHeadMaps);
+  const long long rows7[7] = {(long long)md.nq * md.hd, (long long)md.nkv * md.hd, (long long)md.nkv * md.hd, md.d, md.ff, md.ff, md.d};
+  const long long cols7[7] = {md.d, md.d, md.d, (long long)md.nq * md.hd, md.d, md.d, md.ff};
+  const int widx[7] = {1, 2, 3, 4, 6, 7, 8};
+  for (int l = 0; l < md.n_layers && !st; ++l)
+    for (int k = 0; k < 7 && !st; ++k)
+      st = tc_make_map(&M.wmaps[(size_t)l * 7 + k], M.lw[(size_t)l * 9 + widx[k]], rows7[k], cols7[k], kTcBoxRows);
+  for (int i = 0; i < kHeadMaps && !st; ++i) st = tc_make_map(&M.wmaps[(size_t)md.n_layers * 7 + i], M.lm_head, md.V, md.d, kTcBoxRows);
+  const size_t abuf_off[4] = {ml.h, ml.att, ml.act, ml.hf};
+  const long long acols[4] = {md.d, (long long)md.nq * md.hd, md.ff, md.d};
+  const long long arows[4] = {lay.max_rows, lay.max_rows, lay.max_rows, lay.max_logit_rows};
+  const int npads[4] = {16, 32, 64, 128};
+  for (int b = 0; b < 4 && !st; ++b)
+    for (int p = 0; p < 4 && !st; ++p) st = tc_make_map(&M.amaps[b][p], c->ws + abuf_off[b], arows[b], acols[b], npads[p]);
+  for (int b = 0; b < 4 && !st; ++b)
+    for (int r = 1; r <= 16 && !st; ++r) st = tc_make_map(&M.amaps_rows[b][r - 1], c->ws + abuf_off[b], arows[b], acols[b], r);
+  if (!st && cudaMemset(c->ws + ml.tc_scratch, 0, kTcCtrlBytes) != cudaSuccess) st = HSD_E_CUDA;
+  if (st) return st;
+  // tables of the persistent forward: tensor maps and per-layer pointers in device memory
+  std::vector<FwdLayerDev> ld(md.n_layers);
+  for (int l = 0; l < md.n_layers; ++l) {
+    ld[l].attn_norm = (const __nv_bfloat16 *)M.lw[(size_t)l * 9 + 0];
+    ld[l].mlp_norm = (const __nv_bfloat16 *)M.lw[(size_t)l * 9 + 5];
+    ld[l].k_pool = (__nv_bfloat16 *)(c->ws + ml.k_pool + ml.pool_layer_stride * l);
+    ld[l].v_pool = (__nv_bfloat16 *)(c->ws + ml.v_pool + ml.pool_layer_stride * l);
+  }
+  if (cudaMemcpy(c->ws + ml.wmaps_dev, M.wmaps.data(), M.wmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(c->ws + ml.layers_dev, ld.data(), ld.size() * sizeof(FwdLayerDev), cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemset(c->ws + ml.attn_counters, 0, 16384) != cudaSuccess)
+    return HSD_E_CUDA;
+  int coop = 0, dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+  M.use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 &&
+                  (md.d / kTcBlockM) * 2 <= c->sm_count && md.n_layers <= 64 && (md.page & (md.page - 1)) == 0 && md.page >= 16;
+  return HSD_OK;
+}
+
+bool supported_dims(const hsd_model_desc *model) {
+  if (model->head_dim != 32 && model->head_dim != 64 && model->head_dim != 128) return false;
+  if (model->n_q_heads / model->n_kv_heads > 8) return false;
+  const int vec = model->dtype == HSD_BF16 ? 8 : 4;
+  return !(model->d_model % vec || model->d_ff % vec || (model->n_q_heads * model->head_dim) % vec);
+}
+
+// Common part of the two create calls.  models[0 .. n_models): one decoder (early exits) or one per level.
+int create_ctx(const hsd_model_desc *models, int n_models, const int32_t *exit_layers, int n_levels, const int32_t *T,
+                      void *workspace, size_t workspace_bytes, hsd_ctx **out) {
+  for (int mi = 0; mi < n_models; ++mi) {
+    const hsd_model_desc *model = &models[mi];
+    if (!model->embed || !model->final_norm || !model->lm_head || !model->layer_weights) return HSD_E_INVALID_ARG;
+    for (int i = 0; i < model->n_layers * 9; ++i)
+      if (!model->layer_weights[i]) return HSD_E_INVALID_ARG;
+    if (!supported_dims(model)) return HSD_E_UNSUPPORTED;
+  }
+  if (!workspace || ((uintptr_t)workspace & 255) != 0) return HSD_E_INVALID_ARG;
+  Layout lay = make_layout(models, n_models, n_levels, T);
+  if (workspace_bytes < lay.total) return HSD_E_WORKSPACE_TOO_SMALL;
+  hsd_ctx *c = new (std::nothrow) hsd_ctx();
+  if (!c) return HSD_E_INVALID_ARG;
+  c->n_levels = n_levels;
+  c->max_batch = models[0].max_batch;
+  c->shared_cache = exit_layers != nullptr;
+  c->exits.resize(n_levels);
+  c->level_model.resize(n_levels);
+  for (int i = 0; i < n_levels; ++i) {
+    c->level_model[i] = c->shared_cache ? 0 : i;
+    c->exits[i] = c->shared_cache ? exit_layers[i] : models[i].n_layers;
+  }
+  if (n_levels > 1) c->T.assign(T, T + n_levels - 1);
+  c->lay = lay;
+  c->ws = (char *)workspace;
+  c->coin24.assign(n_levels, kNoCoin);
+  c->ring_host = nullptr; c->n_acc_host = nullptr; c->page_table_host = nullptr; c->status_host = nullptr;
+  c->sm_count = device_sm_count();
+  c->trace = nullptr; c->trace_logit_calls = 0; c->trace_records = 0;
+  c->ring_next = 0; c->ring_in_flight = 0; c->timers_used = 0; c->timers_ok = true; c->stream = nullptr; c->seed = 0;
+  c->status_off = lay.model[0].tc_scratch;
+  bool ok = cudaMallocHost(&c->ring_host, lay.ring_slot * kRingSlots) == cudaSuccess &&
+            cudaMallocHost(&c->n_acc_host, (size_t)c->max_batch * 4) == cudaSuccess &&
+            cudaMallocHost(&c->page_table_host, (size_t)c->max_batch * lay.pages_per_seq * 4) == cudaSuccess &&
+            cudaMallocHost(&c->status_host, 4) == cudaSuccess;
+  for (int i = 0; i < kTimerPairs; ++i) { c->timers[i].a = nullptr; c->timers[i].b = nullptr; }
+  for (int i = 0; ok && i < kTimerPairs; ++i)
+    c->timers_ok = c->timers_ok && cudaEventCreate(&c->timers[i].a) == cudaSuccess && cudaEventCreate(&c->timers[i].b) == cudaSuccess;
+  int st = ok ? HSD_OK : HSD_E_CUDA;
+  if (!st && (cudaMemset(c->ws + c->status_off, 0, 256) != cudaSuccess || cudaMemset(c->ws + lay.grid_counter, 0, 256) != cudaSuccess))
+    st = HSD_E_CUDA;
+  c->models.resize(n_models);
+  for (int mi = 0; mi < n_models && !st; ++mi) {
+    st = init_model(c, c->models[mi], &models[mi], lay.model[mi]);
+    c->any_tc = c->any_tc || c->models[mi].use_tc;
+  }
+  if (st) {
+    hsd_destroy(c);
+    return st;
+  }
+  c->md = c->models.back().md;
+  c->level_head.resize(n_levels);
+  c->level_norm.resize(n_levels);
+  for (int i = 0; i < n_levels; ++i) {
+    c->level_head[i] = c->model_of(i).lm_head;
+    c->level_norm[i] = c->model_of(i).final_norm;
+  }
+  c->stats.assign(n_levels, hsd_level_stats{});
+  *c->status_host = 0;
+  *out = c;
   return HSD_OK;
 }
 
@@ -714,124 +913,35 @@ extern "C" {
 
 size_t hsd_workspace_bytes(const hsd_model_desc *model, const int32_t *exit_layers, int n_levels, const int32_t *T) {
   if (!valid_model(model, exit_layers, n_levels, T)) return 0;
-  return make_layout(model, n_levels, T).total;
+  return make_layout(model, 1, n_levels, T).total;
+}
+
+size_t hsd_models_workspace_bytes(const hsd_model_desc *models, int n_levels, const int32_t *T) {
+  if (!valid_models(models, n_levels, T)) return 0;
+  return make_layout(models, n_levels, n_levels, T).total;
 }
 
 int hsd_create(const hsd_model_desc *model, const int32_t *exit_layers, int n_levels, const int32_t *T, void *workspace,
                size_t workspace_bytes, hsd_ctx **out) {
   if (!out) return HSD_E_INVALID_ARG;
   *out = nullptr;
-  if (!valid_model(model, exit_layers, n_levels, T) || !workspace) return HSD_E_INVALID_ARG;
-  if (!model->embed || !model->final_norm || !model->lm_head || !model->layer_weights) return HSD_E_INVALID_ARG;
-  for (int i = 0; i < model->n_layers * 9; ++i)
-    if (!model->layer_weights[i]) return HSD_E_INVALID_ARG;
-  if (((uintptr_t)workspace & 255) != 0) return HSD_E_INVALID_ARG;
-  if (model->head_dim != 32 && model->head_dim != 64 && model->head_dim != 128) return HSD_E_UNSUPPORTED;
-  if (model->n_q_heads / model->n_kv_heads > 8) return HSD_E_UNSUPPORTED;
-  const int vec = model->dtype == HSD_BF16 ? 8 : 4;
-  if (model->d_model % vec || model->d_ff % vec || (model->n_q_heads * model->head_dim) % vec) return HSD_E_UNSUPPORTED;
-  Layout lay = make_layout(model, n_levels, T);
-  if (workspace_bytes < lay.total) return HSD_E_WORKSPACE_TOO_SMALL;
-  hsd_ctx *c = new (std::nothrow) hsd_ctx();
+  if (!valid_model(model, exit_layers, n_levels, T)) return HSD_E_INVALID_ARG;
+  return create_ctx(model, 1, exit_layers, n_levels, T, workspace, workspace_bytes, out);
+}
+
+int hsd_create_models(const hsd_model_desc *models, int n_levels, const int32_t *T, void *workspace, size_t workspace_bytes,
+                      hsd_ctx **out) {
+  if (!out) return HSD_E_INVALID_ARG;
+  *out = nullptr;
+  if (!valid_models(models, n_levels, T)) return HSD_E_INVALID_ARG;
+  return create_ctx(models, n_levels, nullptr, n_levels, T, workspace, workspace_bytes, out);
+}
+
+int hsd_set_phase_folding(hsd_ctx *c, int fold_qkv, int fold_gate_up, int early_norm) {
   if (!c) return HSD_E_INVALID_ARG;
-  c->md = ModelDims{model->n_layers, model->d_model, model->n_q_heads, model->n_kv_heads, model->head_dim, model->d_ff,
-                    model->vocab, model->dtype, model->rms_eps, model->rope_theta, model->max_seq,
-                    model->page_size ? model->page_size : 16, lay.pages_per_seq};
-  c->n_levels = n_levels;
-  c->max_batch = model->max_batch;
-  c->exits.assign(exit_layers, exit_layers + n_levels);
-  if (n_levels > 1) c->T.assign(T, T + n_levels - 1);
-  c->lay = lay;
-  c->ws = (char *)workspace;
-  c->embed = model->embed; c->final_norm = model->final_norm; c->lm_head = model->lm_head;
-  c->level_head.assign(n_levels, model->lm_head);
-  c->level_norm.assign(n_levels, model->final_norm);
-  c->coin24.assign(n_levels, kNoCoin);
-  c->lw.assign(model->layer_weights, model->layer_weights + (size_t)model->n_layers * 9);
-  c->ring_host = nullptr; c->n_acc_host = nullptr; c->page_table_host = nullptr; c->status_host = nullptr;
-  c->use_tc = false; c->use_persist = false; c->sm_count = 148;
-  c->trace = nullptr; c->trace_logit_calls = 0; c->trace_records = 0;
-  c->ring_next = 0; c->ring_in_flight = 0; c->timers_used = 0; c->timers_ok = true; c->stream = nullptr; c->seed = 0;
-  bool ok = cudaMallocHost(&c->ring_host, lay.ring_slot * kRingSlots) == cudaSuccess &&
-            cudaMallocHost(&c->n_acc_host, (size_t)c->max_batch * 4) == cudaSuccess &&
-            cudaMallocHost(&c->page_table_host, (size_t)c->max_batch * lay.pages_per_seq * 4) == cudaSuccess;
-  for (int i = 0; i < kTimerPairs; ++i) { c->timers[i].a = nullptr; c->timers[i].b = nullptr; }
-  for (int i = 0; ok && i < kTimerPairs; ++i)
-    c->timers_ok = c->timers_ok && cudaEventCreate(&c->timers[i].a) == cudaSuccess && cudaEventCreate(&c->timers[i].b) == cudaSuccess;
-  if (ok) {
-    // rotary tables: angles in double, rounded to fp32
-    const int half = c->md.hd / 2;
-    std::vector<float> cs((size_t)c->md.max_seq * half), sn((size_t)c->md.max_seq * half);
-    for (int p = 0; p < c->md.max_seq; ++p)
-      for (int k = 0; k < half; ++k) {
-        double ang = (double)p * pow((double)c->md.theta, -2.0 * k / (double)c->md.hd);
-        cs[(size_t)p * half + k] = (float)cos(ang);
-        sn[(size_t)p * half + k] = (float)sin(ang);
-      }
-    ok = cudaMemcpy(c->ws + lay.cos_tab, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess &&
-         cudaMemcpy(c->ws + lay.sin_tab, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice) == cudaSuccess;
-  }
-  if (!ok) {
-    hsd_destroy(c);
-    return HSD_E_CUDA;
-  }
-  c->stats.assign(n_levels, hsd_level_stats{});
-  // tensor-core path: bf16 model whose contraction sizes are multiples of the 64-element k-block
-  c->sm_count = device_sm_count();
-  c->use_tc = model->dtype == HSD_BF16 && model->d_model % kTcBlockK == 0 && model->d_ff % kTcBlockK == 0 &&
-              (model->n_q_heads * model->head_dim) % kTcBlockK == 0 && tc_init() == HSD_OK;
-  if (c->use_tc) {
-    const ModelDims &md = c->md;
-    int st = HSD_OK;
-    c->wmaps.resize((size_t)md.n_layers * 7 + kHeadMaps);
-    const long long rows7[7] = {(long long)md.nq * md.hd, (long long)md.nkv * md.hd, (long long)md.nkv * md.hd, md.d, md.ff, md.ff, md.d};
-    const long long cols7[7] = {md.d, md.d, md.d, (long long)md.nq * md.hd, md.d, md.d, md.ff};
-    const int widx[7] = {1, 2, 3, 4, 6, 7, 8};
-    for (int l = 0; l < md.n_layers && !st; ++l)
-      for (int k = 0; k < 7 && !st; ++k)
-        st = tc_make_map(&c->wmaps[(size_t)l * 7 + k], c->lw[(size_t)l * 9 + widx[k]], rows7[k], cols7[k], kTcBoxRows);
-    for (int i = 0; i < kHeadMaps && !st; ++i) st = tc_make_map(&c->wmaps[(size_t)md.n_layers * 7 + i], c->lm_head, md.V, md.d, kTcBoxRows);
-    const size_t abuf_off[4] = {lay.h, lay.att, lay.act, lay.hf};
-    const long long acols[4] = {md.d, (long long)md.nq * md.hd, md.ff, md.d};
-    int max_logit_rows = 0;
-    for (int i = 0; i < n_levels; ++i) max_logit_rows = std::max(max_logit_rows, c->max_batch * lay.slots[i]);
-    const long long arows[4] = {lay.max_rows, lay.max_rows, lay.max_rows, max_logit_rows};
-    const int npads[4] = {16, 32, 64, 128};
-    for (int b = 0; b < 4 && !st; ++b)
-      for (int p = 0; p < 4 && !st; ++p) st = tc_make_map(&c->amaps[b][p], c->ws + abuf_off[b], arows[b], acols[b], npads[p]);
-    for (int b = 0; b < 4 && !st; ++b)
-      for (int r = 1; r <= 16 && !st; ++r) st = tc_make_map(&c->amaps_rows[b][r - 1], c->ws + abuf_off[b], arows[b], acols[b], r);
-    if (!st && cudaMemset(c->ws + lay.tc_scratch, 0, kTcCtrlBytes) != cudaSuccess) st = HSD_E_CUDA;
-    // tables of the persistent forward: tensor maps and per-layer pointers in device memory
-    if (!st) {
-      std::vector<FwdLayerDev> ld(md.n_layers);
-      for (int l = 0; l < md.n_layers; ++l) {
-        ld[l].attn_norm = (const __nv_bfloat16 *)c->lw[(size_t)l * 9 + 0];
-        ld[l].mlp_norm = (const __nv_bfloat16 *)c->lw[(size_t)l * 9 + 5];
-        ld[l].k_pool = (__nv_bfloat16 *)(c->ws + lay.k_pool + lay.pool_layer_stride * l);
-        ld[l].v_pool = (__nv_bfloat16 *)(c->ws + lay.v_pool + lay.pool_layer_stride * l);
-      }
-      if (cudaMemcpy(c->ws + lay.wmaps_dev, c->wmaps.data(), c->wmaps.size() * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess ||
-          cudaMemcpy(c->ws + lay.layers_dev, ld.data(), ld.size() * sizeof(FwdLayerDev), cudaMemcpyHostToDevice) != cudaSuccess ||
-          cudaMemset(c->ws + lay.attn_counters, 0, 16384) != cudaSuccess || cudaMemset(c->ws + lay.grid_counter, 0, 256) != cudaSuccess)
-        st = HSD_E_CUDA;
-      int coop = 0, dev = 0;
-      cudaGetDevice(&dev);
-      cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-      c->use_persist = coop != 0 && fwd_persist_supported(md.hd, md.nq / md.nkv) && md.d % 256 == 0 && md.d <= 4096 && (md.d / kTcBlockM) * 2 <= c->sm_count && md.n_layers <= 64 && (md.page & (md.page - 1)) == 0 && md.page >= 16 &&
-                       getenv("HSD_NO_PERSIST") == nullptr;
-      if (const char *e = getenv("HSD_ATTN_SINGLE_MAX")) c->attn_single_max = atoi(e);
-      c->no_fuse_qkv = getenv("HSD_NO_FUSE_QKV") != nullptr;
-      c->no_fuse_gu = getenv("HSD_NO_FUSE_GU") != nullptr;
-    }
-    if (!st && cudaMallocHost(&c->status_host, 4) != cudaSuccess) st = HSD_E_CUDA;
-    if (st) {
-      hsd_destroy(c);
-      return st;
-    }
-    *c->status_host = 0;
-  }
-  *out = c;
+  c->no_fuse_qkv = fold_qkv == 0;
+  c->no_fuse_gu = fold_gate_up == 0;
+  c->no_early_norm = early_norm == 0;
   return HSD_OK;
 }
 
@@ -900,8 +1010,10 @@ int hsd_generate(hsd_ctx *c, const int32_t *prompt_ids, int batch, int prompt_le
 int hsd_layer_logits(hsd_ctx *c, const int32_t *token_ids, int n_tokens, const int32_t *layers, int n_layers_sel,
                      void *out_logits, void *stream) {
   if (!c || !token_ids || !layers || !out_logits || n_tokens < 1 || n_layers_sel < 1) return HSD_E_INVALID_ARG;
-  const ModelDims &md = c->md;
+  Model &M = c->models.back();                  // the target's decoder
+  const ModelDims &md = M.md;
   const Layout &L = c->lay;
+  const ModelLayout &ML = M.lay;
   if (n_tokens > L.max_rows || n_tokens > md.max_seq || n_tokens > 128) return HSD_E_INVALID_ARG;
   for (int i = 0; i < n_layers_sel; ++i)
     if (layers[i] < 1 || layers[i] > md.n_layers || (i > 0 && layers[i] <= layers[i - 1])) return HSD_E_INVALID_ARG;
@@ -937,34 +1049,34 @@ int hsd_layer_logits(hsd_ctx *c, const int32_t *token_ids, int n_tokens, const i
   int n_splits = std::max(1, std::min((int)kMaxSplits, kAttnBlocksTarget / std::max(1, n_attn * md.nkv)));
   int keys_per_split = (int)align_up((size_t)(R + n_splits - 1) / n_splits, kAttnKeyTile);
   n_splits = (R + keys_per_split - 1) / keys_per_split;
-  float *x = c->dev<float>(L.x);
-  void *h = c->dev<void>(L.h), *q = c->dev<void>(L.q), *att = c->dev<void>(L.att), *act = c->dev<void>(L.act);
-  float *qkv = c->dev<float>(L.qkv);
+  float *x = c->dev<float>(ML.x);
+  void *h = c->dev<void>(ML.h), *q = c->dev<void>(ML.q), *att = c->dev<void>(ML.att), *act = c->dev<void>(ML.act);
+  float *qkv = c->dev<float>(ML.qkv);
   const int *pt = c->dev<int>(L.page_table);
   const size_t es = elem_size(md.dtype);
-  HSD_TRY(launch_embed(md, c->embed, c->dev<int>(L.tokens), rb, x, s));
+  HSD_TRY(launch_embed(md, M.embed, c->dev<int>(L.tokens), rb, x, s));
   int next = 0;
   for (int l = 0; l < md.n_layers && next < n_layers_sel; ++l) {
-    const void *const *w = &c->lw[(size_t)l * 9];
-    void *kp = c->ws + L.k_pool + L.pool_layer_stride * l, *vp = c->ws + L.v_pool + L.pool_layer_stride * l;
+    const void *const *w = &M.lw[(size_t)l * 9];
+    void *kp = c->ws + ML.k_pool + ML.pool_layer_stride * l, *vp = c->ws + ML.v_pool + ML.pool_layer_stride * l;
     HSD_TRY(launch_rmsnorm(md, x, w[0], nullptr, R, h, s));
     GemmSegs qkv_segs = {{w[1], w[2], w[3]}, {md.nq * md.hd, md.nkv * md.hd, md.nkv * md.hd}, 3};
-    HSD_TRY(gemm(c, 0, h, R, md.d, qkv_segs, l * 7 + 0, GEMM_STORE_F32, qkv, nullptr, nullptr));
-    HSD_TRY(launch_rope_kv(md, qkv, rb, c->dev<float>(L.cos_tab), c->dev<float>(L.sin_tab), pt, kp, vp, q, s));
-    HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(L.partials), keys_per_split, n_splits, att, s));
+    HSD_TRY(gemm(c, M, 0, h, R, md.d, qkv_segs, l * 7 + 0, GEMM_STORE_F32, qkv, nullptr, nullptr));
+    HSD_TRY(launch_rope_kv(md, qkv, rb, c->dev<float>(ML.cos_tab), c->dev<float>(ML.sin_tab), pt, kp, vp, q, s));
+    HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(ML.partials), keys_per_split, n_splits, att, s));
     GemmSegs o_segs = {{w[4], nullptr, nullptr}, {md.d, 0, 0}, 1};
-    HSD_TRY(gemm(c, 1, att, R, md.nq * md.hd, o_segs, l * 7 + 3, GEMM_ADD_F32, x, nullptr, nullptr));
+    HSD_TRY(gemm(c, M, 1, att, R, md.nq * md.hd, o_segs, l * 7 + 3, GEMM_ADD_F32, x, nullptr, nullptr));
     HSD_TRY(launch_rmsnorm(md, x, w[5], nullptr, R, h, s));
     GemmSegs gu_segs = {{w[6], w[7], nullptr}, {md.ff, md.ff, 0}, 2};
-    HSD_TRY(gemm(c, 0, h, R, md.d, gu_segs, l * 7 + 4, GEMM_SWIGLU_T, nullptr, act, nullptr));
+    HSD_TRY(gemm(c, M, 0, h, R, md.d, gu_segs, l * 7 + 4, GEMM_SWIGLU_T, nullptr, act, nullptr));
     GemmSegs d_segs = {{w[8], nullptr, nullptr}, {md.d, 0, 0}, 1};
-    HSD_TRY(gemm(c, 2, act, R, md.ff, d_segs, l * 7 + 6, GEMM_ADD_F32, x, nullptr, nullptr));
+    HSD_TRY(gemm(c, M, 2, act, R, md.ff, d_segs, l * 7 + 6, GEMM_ADD_F32, x, nullptr, nullptr));
     if (layers[next] == l + 1) {                         // exit after layer l + 1: shared final norm + head on every row
       // (the normalised rows go to the h buffer, free between two layers and large enough for every row; the
       // buffer of the generation path's final norm holds the few logit rows of a verification only)
-      HSD_TRY(launch_rmsnorm(md, x, c->final_norm, rb.lrow_src, R, h, s));
-      GemmSegs lm_segs = {{c->lm_head, nullptr, nullptr}, {md.V, 0, 0}, 1};
-      HSD_TRY(gemm(c, 0, h, R, md.d, lm_segs, md.n_layers * 7 + kHeadMaps - 1, GEMM_STORE_T_SCATTER, nullptr,
+      HSD_TRY(launch_rmsnorm(md, x, M.final_norm, rb.lrow_src, R, h, s));
+      GemmSegs lm_segs = {{M.lm_head, nullptr, nullptr}, {md.V, 0, 0}, 1};
+      HSD_TRY(gemm(c, M, 0, h, R, md.d, lm_segs, md.n_layers * 7 + kHeadMaps - 1, GEMM_STORE_T_SCATTER, nullptr,
                    (char *)out_logits + (size_t)next * R * md.V * es, rb.lrow_dst));
       ++next;
     }
@@ -974,21 +1086,23 @@ int hsd_layer_logits(hsd_ctx *c, const int32_t *token_ids, int n_tokens, const i
 
 int hsd_set_exit_heads(hsd_ctx *c, const void *const *final_norms, const void *const *lm_heads) {
   if (!c) return HSD_E_INVALID_ARG;
-  const ModelDims &md = c->md;
   int st = sync_stream(c);                      // no pass of this context may be in flight
   if (st) return st;
   for (int i = 0; i < c->n_levels; ++i) {
-    c->level_norm[i] = (final_norms && final_norms[i]) ? final_norms[i] : c->final_norm;
-    c->level_head[i] = (lm_heads && lm_heads[i]) ? lm_heads[i] : c->lm_head;
+    Model &M = c->model_of(i);
+    c->level_norm[i] = (final_norms && final_norms[i]) ? final_norms[i] : M.final_norm;
+    c->level_head[i] = (lm_heads && lm_heads[i]) ? lm_heads[i] : M.lm_head;
     if (((uintptr_t)c->level_head[i] & 15) != 0) return HSD_E_INVALID_ARG;
   }
-  if (!c->use_tc) return HSD_OK;
-  for (int i = 0; i < c->n_levels && !st; ++i)
-    st = tc_make_map(&c->wmaps[(size_t)md.n_layers * 7 + i], c->level_head[i], md.V, md.d, kTcBoxRows);
-  if (!st && cudaMemcpy(c->ws + c->lay.wmaps_dev + (size_t)md.n_layers * 7 * sizeof(CUtensorMap),
-                        &c->wmaps[(size_t)md.n_layers * 7], (size_t)c->n_levels * sizeof(CUtensorMap),
-                        cudaMemcpyHostToDevice) != cudaSuccess)
-    st = HSD_E_CUDA;
+  for (int i = 0; i < c->n_levels && !st; ++i) {
+    Model &M = c->model_of(i);
+    if (!M.use_tc) continue;
+    const size_t slot = (size_t)M.md.n_layers * 7 + i;
+    st = tc_make_map(&M.wmaps[slot], c->level_head[i], M.md.V, M.md.d, kTcBoxRows);
+    if (!st && cudaMemcpy(c->ws + M.lay.wmaps_dev + slot * sizeof(CUtensorMap), &M.wmaps[slot], sizeof(CUtensorMap),
+                          cudaMemcpyHostToDevice) != cudaSuccess)
+      st = HSD_E_CUDA;
+  }
   return st;
 }
 

@@ -227,17 +227,36 @@ __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, 
 //   pend:      the residual-add projection that ran just before; its split pieces are added to the
 //              row in fixed piece order (x <- x + p_0 + p_1 + ...) and x is written back.
 // Requires d % 4 == 0 and d <= 4096.
+//   pieces_target != 0: the CTA was idle in that projection and has passed no grid barrier since; it waits until
+//              the counter of CTAs that have stored their pieces reaches pieces_target.
 template <int NPAD>
-__device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const int *row_list, bool src_embed,
+__device__ __forceinline__ bool norm_phase(const FwdArgs &a, int n_rows, const int *row_list, bool src_embed,
                                            const Gemm *pend, const float *pend_pieces, const __nv_bfloat16 *gain, __nv_bfloat16 *dst,
-                                           float *red, int wt) {
+                                           float *red, int wt, unsigned pieces_target, volatile int *abort_flag) {
   constexpr int MAXV = 4;                                  // float4 slots per thread
   constexpr int PB = 4;                                    // pieces loaded at a time per slot
   const int d = a.d, nvec = d >> 2;
   SplitGeom geo;
   geo.U = 1; geo.Gp = 1; geo.pieces_max = 1;
   if (pend) geo = split_geom(*pend, gridDim.x);
-  for (int i = blockIdx.x; i < n_rows; i += gridDim.x) {
+  // rows go to the LAST CTAs of the grid when the norm may start early: those have no tile of the projection
+  const int first = a.early_norm ? (int)(gridDim.x - 1 - blockIdx.x) : (int)blockIdx.x;
+  if (pieces_target != 0u && first < n_rows) {
+    if (wt == 0) {
+      const unsigned *cnt = a.grid_counter + 16;
+      unsigned long long t0 = 0;
+      for (uint32_t it = 0; (int)(ld_acquire_u32(cnt) - pieces_target) < 0; ++it) {
+        if ((it & 31u) == 31u) {
+          const unsigned long long now = globaltimer_ns();
+          if (t0 == 0) t0 = now;
+          if (*abort_flag || now - t0 > kWaitLimitNs) { *abort_flag = 1; break; }
+        }
+      }
+    }
+    worker_sync();
+    if (*abort_flag) return false;
+  }
+  for (int i = first; i < n_rows; i += gridDim.x) {
     const int row = row_list ? row_list[i] : i;
     float *xrow = a.x + (size_t)row * d;
     float4 v[MAXV];
@@ -315,6 +334,7 @@ __device__ __forceinline__ void norm_phase(const FwdArgs &a, int n_rows, const i
       }
     }
   }
+  return true;
 }
 
 // ------------------------------------------------------------------------------ attention phases
@@ -858,6 +878,12 @@ __device__ __forceinline__ void gemm_epilogue(const FwdArgs &a, WorkerCtx &w, in
         }
       }
     }
+    // residual projection whose norm starts early: tell the norm's CTAs that this CTA's pieces are in place (the
+    // stores of the 128 epilogue threads are ordered before the release by the group barrier, as in the grid barrier)
+    if (a.early_norm && g.mode == MODE_ADD && w.c < geo.Gp) {
+      epi_sync();
+      if (w.wt == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.grid_counter + 16) : "memory");
+    }
   }
 
 // Down projection p of a pass with at most four rows: the worker warps build its activation tiles straight into
@@ -1285,6 +1311,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     // Steps 1 and 7 are empty (no barrier) when the finish is folded into the phase after it.
     const int n_steps = 1 + 10 * a.n_run + (a.L > 0 ? 2 : 0);
     enum { K_EPI, K_FIN, K_ATTN_A, K_ATTN_B, K_NORM, K_NONE };
+    // CTAs with pieces of the two residual projections; pieces stored so far (what the early norm waits for)
+    const unsigned add_ctas_o = (unsigned)min(G, split_geom(make_gemm(a, 1), G).Gp), add_ctas_d = (unsigned)min(G, split_geom(make_gemm(a, 3), G).Gp);
+    unsigned pieces_target = 0u;
 #pragma unroll 1
     for (int t = 0; t < n_steps && alive; ++t) {
       int kind, gp = 0, ready = -1, l = 0;
@@ -1305,14 +1334,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
             if (a.n_splits == 1) { kind = K_NONE; barrier = false; }
             else { kind = K_ATTN_B; ready = p + 1; }
             break;
-          case 4: kind = K_EPI; gp = p + 1; break;
+          case 4: kind = K_EPI; gp = p + 1; barrier = !a.early_norm; break;
           case 5: kind = K_NORM; gp = p + 1; ready = p + 2; break;
           case 6: kind = K_EPI; gp = p + 2; if (a.fuse_gu) ready = p + 3; break;
           case 7:                                            // folded into the down projection in passes with few rows
             if (a.fuse_gu) { kind = K_NONE; barrier = false; }
             else { kind = K_FIN; gp = p + 2; ready = p + 3; }
             break;
-          case 8: kind = K_EPI; gp = p + 3; barrier = (l + 1 < a.n_run || a.L > 0); break;
+          case 8: kind = K_EPI; gp = p + 3; barrier = (l + 1 < a.n_run || a.L > 0) && !a.early_norm; break;
           default:
             kind = (l + 1 < a.n_run || a.L > 0) ? K_NORM : K_NONE; gp = p + 3; ready = p + 4;
             barrier = (kind == K_NORM);
@@ -1339,13 +1368,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
           const Gemm pend = make_gemm(a, first ? 0 : gp);
           const __nv_bfloat16 *gain = first ? a.layers[0].attn_norm
                                             : (last ? a.final_norm : (mid ? layers_sh[l].mlp_norm : layers_sh[l + 1].attn_norm));
-          norm_phase<NPAD>(a, last ? a.L : a.R, last ? a.lrow_src : nullptr, first, first ? nullptr : &pend, pieces_of(a, gp), gain,
-                           last ? a.hf : a.h, red, wt);
+          if (!first && a.early_norm) pieces_target += mid ? add_ctas_o : add_ctas_d;
+          alive = norm_phase<NPAD>(a, last ? a.L : a.R, last ? a.lrow_src : nullptr, first, first ? nullptr : &pend, pieces_of(a, gp), gain,
+                                   last ? a.hf : a.h, red, wt, (!first && a.early_norm) ? pieces_target : 0u, abort_flag);
           break;
         }
         default: break;
       }
-      if (barrier) alive = grid_barrier(a, epoch, abort_flag, wt, ready >= 0 ? ready_bar(ready & 1) : 0u);
+      if (barrier && alive) alive = grid_barrier(a, epoch, abort_flag, wt, ready >= 0 ? ready_bar(ready & 1) : 0u);
     }
   }
   if (a.prof && blockIdx.x == 0 && threadIdx.x == 128) for (int i = 0; i < 16; ++i) a.prof[940 + i] = (unsigned long long)dbg_cy[i];
@@ -1407,6 +1437,12 @@ int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaS
       a.gu_pieces_max = (KB + per - 1) / per + 1;
     }
     if (a.gu_pieces_max > 4) a.fuse_gu = 0;
+  }
+  {  // CTAs without a tile of the residual projections (the device's split_geom): enough of them for every row?
+    const int n_tiles = (a.d + kTcBlockM - 1) / kTcBlockM;
+    int idle = 0;
+    if (n_tiles * 2 <= sm_count) idle = sm_count - n_tiles * std::min(4, sm_count / n_tiles);   // >= the device's count of idle CTAs
+    a.early_norm = (a.early_norm && a.R <= idle && a.L <= idle) ? 1 : 0;
   }
   switch (a.hd) {
     case 128: return launch_hd<128>(a, npad, sm_count, s);

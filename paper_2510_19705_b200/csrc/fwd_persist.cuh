@@ -28,6 +28,9 @@ struct FwdArgs {
   int fuse_qkv;                    // 1: every sequence is one attention item; the item's CTAs finish its q / k / v themselves
   int fuse_gu;                     // 1: at most 4 rows; the down projection's CTAs build their activation tiles from the gate / up pieces
   int gu_pieces_max;               // pieces per gate / up tile at most (its split geometry; filled in by the launcher)
+  int early_norm;                  // 1: the RMSNorm after a residual projection runs on CTAs that have no part in that projection;
+                                   //    they start as soon as its pieces are complete (a counter), one grid barrier less per norm
+                                   //    (filled in by the launcher)
   float *pieces2;                  // split pieces of the down projection while `pieces` still holds gate / up (fuse_gu)
   const int *tokens, *page_table, *row_seq, *row_pos, *lrow_src;
   const int4 *attn_items;          // (first packed row, rows, sequence, position of first row)
@@ -39,7 +42,8 @@ struct FwdArgs {
   int *attn_counters;              // zero on entry, zero on exit
   float *pieces;
   int *tile_counters;              // zero on entry, zero on exit
-  unsigned *grid_counter;          // zero on entry
+  unsigned *grid_counter;          // zero on entry; [16] (64 bytes on) counts the CTAs that have stored their pieces of the
+                                   // residual projections so far (early_norm), zero on entry as well
   int *status;                     // set non-zero when a bounded wait gave up
   unsigned long long *prof;        // optional [gridDim][kFwdProfEvents]: barrier arrive / depart times (ns)
   CUtensorMap amap[4];             // activations h, att, act, hf; box rows = row padding of this launch

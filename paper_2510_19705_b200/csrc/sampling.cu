@@ -2,6 +2,9 @@
 // fused softmax-statistics / acceptance / residual-resample step (Algorithm 2; rule of Section 2).
 #include "sampling.cuh"
 #include "sampling_api.cuh"
+#include "tc_ptx.cuh"
+#include <algorithm>
+#include <atomic>
 
 namespace hsd {
 
@@ -246,8 +249,323 @@ decide_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, in
   }
 }
 
+// ------------------------------------------------------------------------------ fused verification
+// Algorithm 2's decision in ONE launch for bf16 rows: statistics of all p and q rows, the accept tests and the
+// final draw.  Persistent grid, one CTA per SM: a producer thread streams the CTA's rows into a shared-memory
+// ring with bulk copies (so HBM latency hides under the other rows' arithmetic, which is what bounds this
+// kernel: ~16 issue slots per logit for the unfused fp32 exp and the 64-bit sums); the 1024 threads take a row
+// into registers, thread 0 refills the slot with the row three items ahead, and the row is reduced to (max,
+// integer total, weight of the drafted token).
+// Rows are dealt round-robin in sequence-major order, so a sequence's rows finish at about the same time on
+// different SMs; the CTA that delivers a sequence's last row (a counter per sequence) takes that sequence's
+// decision while the rows it needs are still in L2.  No CTA ever waits for another.
+constexpr int kFusedConsumers = 1024;
+constexpr int kFusedThreads = kFusedConsumers;
+constexpr int kFusedSlots = 3;
+constexpr int kFusedVecPerThread = 4;                      // 16-byte vectors of a row per consumer thread
+constexpr int kFusedMaxV = kFusedConsumers * kFusedVecPerThread * 8;
+constexpr uint32_t kFusedPiece = 4096;                     // bytes per bulk copy; 32 of them cover the largest row
+using FusedGroup = WholeBlock;
+
+struct FusedArgs {
+  const __nv_bfloat16 *p, *q;
+  int32_t *tokens;
+  int V, t_max, batch;
+  const VerifySeq *desc;
+  int regular_t;
+  u32 regular_serial, regular_level;
+  RowStat *stats;
+  unsigned *counters;            // zero on entry: [batch] rows delivered per sequence | queue length | tickets drawn |
+                                 // [batch] queue of sequences ready for their decision (b + 1)
+  u64 seed;
+  int32_t *out_tokens, *out_n;
+  int write_in_place;
+  u32 coin24;
+  int *status;                   // optional: set to 1 if a bounded wait gave up
+};
+
+__device__ __forceinline__ VerifySeq fused_seq(const FusedArgs &a, int b) {
+  VerifySeq d;
+  if (a.desc) return a.desc[b];
+  d.t = a.regular_t; d.p_row0 = (long long)b * (a.regular_t + 1); d.q_row0 = (long long)b * a.regular_t;
+  d.tok_off = (long long)b * a.regular_t; d.serial = a.regular_serial; d.seq = b; d.level = a.regular_level;
+  return d;
+}
+
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Inverse CDF over weight(i) of the thread's own 32 tokens, as block_inverse_cdf_chunk, except that the walk
+// through the owning thread's chunk is done by warp 0 together: lane i recomputes the weight of the chunk's
+// token i from global memory (weight_at(k)), a warp scan finds the first token whose inclusive sum passes the
+// threshold.  Integer weights, so the recomputed values are the same.
+template <class WeightFn, class WeightAt>
+__device__ __forceinline__ int fused_inverse_cdf(int V, int k0, u32 U, WeightFn weight, WeightAt weight_at, u64 *sh64 /*[34]*/,
+                                                 int *sh_owner) {
+  u64 local = 0;
+#pragma unroll
+  for (int i = 0; i < kChunkTokens; ++i)
+    if (k0 + i < V) local += weight(i);
+  u64 total;
+  const u64 excl = block_exclusive_scan<FusedGroup>(local, sh64, &total);
+  if (total == 0) return -1;                               // uniform
+  const u64 tau = cdf_threshold(U, total);
+  if (tau >= excl && tau < excl + local) {                 // exactly one thread
+    *sh_owner = threadIdx.x;
+    sh64[33] = excl;
+  }
+  FusedGroup::sync();
+  if (threadIdx.x < 32) {
+    const int lane = threadIdx.x, k = *sh_owner * kChunkTokens + lane;
+    u64 c = k < V ? weight_at(k) : 0ull;
+    for (int o = 1; o < 32; o <<= 1) {
+      const u64 n = __shfl_up_sync(0xFFFFFFFFu, c, o);
+      if (lane >= o) c += n;
+    }
+    const unsigned hit = __ballot_sync(0xFFFFFFFFu, c + sh64[33] > tau && k < V);
+    if (lane == 0) *sh_owner = *sh_owner * kChunkTokens + (__ffs(hit) - 1);
+  }
+  FusedGroup::sync();
+  const int r = *sh_owner;
+  FusedGroup::sync();
+  return r;
+}
+
+// The decision of sequence b (the whole CTA): accept tests on the row statistics, then the final draw from the
+// residual of the first rejected position, or from the last target row.
+__device__ __forceinline__ void fused_decide(const FusedArgs &a, int b, const VerifySeq &d, u64 *sh64, int *sh_int /*[2]*/) {
+  const int tid = threadIdx.x, V = a.V, t_max = a.t_max;
+  const RowStat *st = a.stats + (size_t)b * (2 * t_max + 1);
+  if (tid == 0) sh_int[1] = d.t;
+  FusedGroup::sync();
+  if (tid < d.t) {
+    const int j = tid;
+    const float4 rp = __ldcg(reinterpret_cast<const float4 *>(st + j)), rq = __ldcg(reinterpret_cast<const float4 *>(st + t_max + 1 + j));
+    const RowStat sp = *reinterpret_cast<const RowStat *>(&rp), sq = *reinterpret_cast<const RowStat *>(&rq);
+    const u64 Pp = fixed_prob(sp.Ex, prob_scale(sp.S)), Pq = fixed_prob(sq.Ex, prob_scale(sq.S));
+    const u32 U = uniform24(a.seed, j, d.serial, d.level, PURPOSE_ACCEPT, d.seq);
+    bool ok = (((u64)U * Pq) >> 24) < Pp;                  // u < p(x) / q(x)
+    if (a.coin24 != kNoCoin) ok = U < a.coin24;            // ablation: IID acceptance with a fixed probability
+    if (!ok) atomicMin(&sh_int[1], j);
+  }
+  FusedGroup::sync();
+  const int n = sh_int[1];
+  FusedGroup::sync();                                      // sh_int[1] is reused by the draw
+  const u32 U = uniform24(a.seed, 0, d.serial, d.level, PURPOSE_FINAL, d.seq);
+  const __nv_bfloat16 *prow = a.p + (size_t)(d.p_row0 + n) * V;
+  const float4 rpn = __ldcg(reinterpret_cast<const float4 *>(st + n));
+  const RowStat spn = *reinterpret_cast<const RowStat *>(&rpn);
+  const float mp = spn.m;
+  const int k0 = tid * kChunkTokens;
+  const Chunk32 cp = chunk_load(prow, V, k0);
+  int m_tok = -1;
+  if (n < d.t) {
+    const __nv_bfloat16 *qrow = a.q + (size_t)(d.q_row0 + n) * V;
+    const Chunk32 cq = chunk_load(qrow, V, k0);
+    const float4 rqn = __ldcg(reinterpret_cast<const float4 *>(st + t_max + 1 + n));
+    const RowStat sqn = *reinterpret_cast<const RowStat *>(&rqn);
+    const ProbScale psp = prob_scale(spn.S), psq = prob_scale(sqn.S);
+    const float mq = sqn.m;
+    auto residual = [&](float lp, float lq) {                // both rows' weights in one packed evaluation
+      u32 ep, eq;
+      exp_weight2m(lp, lq, mp, mq, ep, eq);
+      const u64 Pp = fixed_prob(ep, psp), Pq = fixed_prob(eq, psq);
+      return Pp > Pq ? Pp - Pq : 0ull;
+    };
+    m_tok = fused_inverse_cdf(V, k0, U, [&](int i) { return residual(chunk_get(cp, i), chunk_get(cq, i)); },
+                              [&](int k) { return residual(__bfloat162float(prow[k]), __bfloat162float(qrow[k])); }, sh64, &sh_int[1]);
+  }
+  if (m_tok < 0)   // bonus token, or an all-zero residual: draw from the verifier's own row
+    m_tok = fused_inverse_cdf(V, k0, U, [&](int i) { return (u64)exp_weight(chunk_get(cp, i), mp); },
+                              [&](int k) { return (u64)exp_weight(__bfloat162float(prow[k]), mp); }, sh64, &sh_int[1]);
+  if (tid == 0) {
+    a.out_n[b] = n;
+    if (a.write_in_place) a.tokens[d.tok_off + n] = m_tok;
+  }
+  if (a.out_tokens) {
+    for (int j = tid; j <= t_max; j += kFusedConsumers) {
+      int v = -1;
+      if (j < n) v = a.tokens[d.tok_off + j];
+      else if (j == n) v = m_tok;
+      a.out_tokens[(size_t)b * (t_max + 1) + j] = v;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kFusedThreads, 1) verify_fused_kernel(const __grid_constant__ FusedArgs a) {
+  extern __shared__ uint8_t fused_smem_raw[];
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fused_smem_raw) + 127) & ~(uintptr_t)127);
+  const uint32_t row_bytes = (uint32_t)a.V * 2u, slot_bytes = (row_bytes + 127u) & ~127u;
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)kFusedSlots * slot_bytes);   // full[S]
+  __shared__ float shf[32];
+  __shared__ u64 sh64[34];
+  __shared__ int sh_flag[2];                 // [0] this CTA decides the row's sequence, [1] first rejected position
+  __shared__ int sh_abort;
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int rows_per_seq = 2 * a.t_max + 1, n_items = a.batch * rows_per_seq;
+  if (tid == 0) {
+    for (int s = 0; s < kFusedSlots; ++s) ptx::mbar_init(bar0 + 8u * s, 1);
+    sh_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int *abort_flag = &sh_abort;
+  // item i = (sequence b, row r): r <= t_max: target row r (valid if r <= t_b); else draft row r - t_max - 1 (valid if < t_b)
+  auto row_of = [&](int i, VerifySeq &d, int &b, int &r) -> const __nv_bfloat16 * {
+    b = i / rows_per_seq; r = i - b * rows_per_seq;
+    d = fused_seq(a, b);
+    if (r <= a.t_max) return r <= d.t ? a.p + (size_t)(d.p_row0 + r) * a.V : nullptr;
+    const int j = r - a.t_max - 1;
+    return j < d.t ? a.q + (size_t)(d.q_row0 + j) * a.V : nullptr;
+  };
+  // warp 0 keeps the ring full: `ahead` = next item of this CTA that has not been asked for yet.  A row is fetched
+  // as 4 KiB bulk copies, one per lane (one 64 KB copy runs at a fraction of an SM's bandwidth).
+  int ahead = blockIdx.x;
+  auto fetch_next = [&](int slot) {                        // all lanes of warp 0
+    while (ahead < n_items) {
+      VerifySeq d; int b, r;
+      const __nv_bfloat16 *row = row_of(ahead, d, b, r);
+      ahead += gridDim.x;
+      if (!row) continue;
+      if (lane == 0) ptx::mbar_expect_tx(bar0 + 8u * slot, row_bytes);
+      __syncwarp();
+      const uint32_t off = (uint32_t)lane * kFusedPiece;
+      if (off < row_bytes)
+        bulk_load_row(ptx::smem_u32(smem + (size_t)slot * slot_bytes) + off, reinterpret_cast<const uint8_t *>(row) + off,
+                      min(kFusedPiece, row_bytes - off), bar0 + 8u * slot);
+      return;
+    }
+  };
+  if (tid < 32)
+    for (int s = 0; s < kFusedSlots; ++s) fetch_next(s);
+  const int nvec = a.V >> 3;
+  int s = 0;
+  uint32_t par = 0;
+  for (int i = blockIdx.x; i < n_items; i += gridDim.x) {
+    VerifySeq d; int b, r;
+    const __nv_bfloat16 *row = row_of(i, d, b, r);
+    if (!row) continue;                                   // uniform over the CTA
+    // the drafted token's logit (thread 0 only), asked for before the wait
+    int tok = -1;
+    if (r < d.t) tok = a.tokens[d.tok_off + r];
+    else if (r > a.t_max) tok = a.tokens[d.tok_off + (r - a.t_max - 1)];
+    float l_tok = 0.f;
+    const bool has_tok = tok >= 0 && tok < a.V;
+    if (tid == 0 && has_tok) l_tok = __bfloat162float(row[tok]);
+    if (lane == 0) ptx::mbar_wait(bar0 + 8u * s, par, abort_flag);      // a give-up raises the CTA's abort flag
+    __syncwarp();
+    const uint4 *src = reinterpret_cast<const uint4 *>(smem + (size_t)s * slot_bytes);
+    uint4 regs[kFusedVecPerThread];
+#pragma unroll
+    for (int j = 0; j < kFusedVecPerThread; ++j) {
+      const int iv = tid + kFusedConsumers * j;
+      regs[j] = iv < nvec ? src[iv] : make_uint4(0u, 0u, 0u, 0u);
+    }
+    FusedGroup::sync();                                   // every thread holds its part of the row: the slot is free
+    if (*abort_flag) break;                               // uniform: raised before the barrier
+    if (tid < 32) fetch_next(s);
+    if (++s == kFusedSlots) { s = 0; par ^= 1u; }
+    float m = -INFINITY;
+#pragma unroll
+    for (int j = 0; j < kFusedVecPerThread; ++j) {
+      if (tid + kFusedConsumers * j < nvec) {
+        float f[8];
+        StatVec<__nv_bfloat16>::unpack(regs[j], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) m = fmaxf(m, f[e]);
+      }
+    }
+    m = block_max<FusedGroup>(m, shf);
+    u64 local = 0;
+#pragma unroll
+    for (int j = 0; j < kFusedVecPerThread; ++j) {
+      if (tid + kFusedConsumers * j < nvec) {
+        float f[8];
+        StatVec<__nv_bfloat16>::unpack(regs[j], f);
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+          u32 e0, e1;
+#ifndef FUSED_NO_EXP
+          exp_weight2(f[e], f[e + 1], m, e0, e1);
+          local += (u64)e0 + (u64)e1;
+#endif
+        }
+      }
+    }
+#ifdef FUSED_NO_EXP
+    local = (u64)__float_as_uint(m) + regs[0].x;
+#endif
+    const u64 total = block_sum<FusedGroup>(local, sh64);
+    if (tid == 0) {
+      RowStat st;
+      st.m = m; st.S = total; st.Ex = has_tok ? exp_weight(l_tok, m) : 0u;
+      a.stats[(size_t)b * rows_per_seq + r] = st;
+      __threadfence();
+      const unsigned before = atomicAdd(&a.counters[b], 1u);
+      if (before == (unsigned)(2 * d.t)) {                   // 2 t + 1 rows per sequence: this was the last one
+        // the sequence is ready for its decision: append it to the queue (entry = b + 1; 0 = not yet written)
+        const unsigned at = atomicAdd(&a.counters[a.batch], 1u);
+        __threadfence();
+        atomicExch(&a.counters[a.batch + 2 + at], (unsigned)b + 1u);
+      }
+    }
+  }
+  // Decisions.  Taking one where its last row arrives would chain: the CTA that decides delivers its next rows
+  // late, so it is the last arriver of those sequences too.  Instead every CTA, once its rows are done, draws
+  // tickets until all `batch` decisions are handed out; a ticket whose entry is not written yet waits for it
+  // (bounded): the rows it waits for are never this CTA's own.
+  for (;;) {
+    FusedGroup::sync();
+    if (tid == 0) {
+      int b = -1;
+      if (!*abort_flag) {
+        const unsigned t = atomicAdd(&a.counters[a.batch + 1], 1u);
+        if (t < (unsigned)a.batch) {
+          const unsigned *entry = a.counters + a.batch + 2 + t;
+          unsigned v = 0;
+          unsigned long long t0 = 0;
+          for (uint32_t it = 0;; ++it) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(entry) : "memory");
+            if (v != 0u) break;
+            if ((it & 31u) == 31u) {
+              const unsigned long long now = ptx::globaltimer_ns();
+              if (t0 == 0) t0 = now;
+              if (now - t0 > ptx::kWaitLimitNs) { *abort_flag = 1; break; }
+            }
+          }
+          if (v != 0u) b = (int)v - 1;
+        }
+      }
+      sh_flag[0] = b;
+    }
+    FusedGroup::sync();
+    const int b = sh_flag[0];
+    if (b < 0) break;
+    const VerifySeq d = fused_seq(a, b);
+    fused_decide(a, b, d, sh64, sh_flag);
+  }
+  if (tid == 0 && sh_abort) {
+    // copies already asked for must land before the CTA's shared memory goes away (bounded)
+    for (int k = 0; k < kFusedSlots; ++k) {
+      const unsigned long long t0 = ptx::globaltimer_ns();
+      while (!ptx::mbar_try_wait(bar0 + 8u * s, par))
+        if (ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs / 8) break;
+      if (++s == kFusedSlots) { s = 0; par ^= 1u; }
+    }
+  }
+  __syncthreads();
+  if (tid == 0 && sh_abort && a.status) atomicExch(a.status, 1);
+}
+
 // ------------------------------------------------------------------------------ host launchers
-size_t verify_scratch_bytes(int batch, int t_max) { return (size_t)batch * (2 * t_max + 1) * sizeof(RowStat); }
+// Scratch of one verification call: [counter per sequence (fused kernel)] [RowStat per logits row].
+static size_t verify_counter_bytes(int batch) { return ((size_t)(2 * batch + 2) * 4 + 255) / 256 * 256; }
+size_t verify_scratch_bytes(int batch, int t_max) {
+  return verify_counter_bytes(batch) + (size_t)batch * (2 * t_max + 1) * sizeof(RowStat);
+}
 
 template <typename T>
 static int launch_draft_sample_t(const void *logits, int V, const SampleRow *desc, int n_rows, int regular_rows,
@@ -267,9 +585,8 @@ int launch_draft_sample(const void *logits, int dtype, int V, const SampleRow *d
 
 template <typename T>
 static int launch_verify_t(const void *p, const void *q, int32_t *tokens, int V, int batch, int t_max,
-                           const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch,
+                           const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, RowStat *stats,
                            u64 seed, int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s, u32 coin24) {
-  RowStat *stats = (RowStat *)scratch;
   dim3 grid(2 * t_max + 1, batch);
   constexpr int VN = StatVec<T>::N;
   const bool vec_ok = V % VN == 0 && V / VN <= kStatVecPerThread * kStatThreads && ((uintptr_t)p & 15) == 0 &&
@@ -286,34 +603,72 @@ static int launch_verify_t(const void *p, const void *q, int32_t *tokens, int V,
   return hsd_launch_status();
 }
 
+static int fused_sm_count() {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 148;
+    sms = n;
+  }
+  return sms;
+}
+
 int launch_verify(const void *p, const void *q, int32_t *tokens, int dtype, int V, int batch, int t_max,
-                  const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch, u64 seed,
-                  int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s, u32 coin24) {
+                  const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch,
+                  u64 seed, int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s,
+                  u32 coin24) {
   if (batch == 0) return HSD_OK;
+  unsigned *counters = (unsigned *)scratch;
+  RowStat *stats = (RowStat *)((char *)scratch + verify_counter_bytes(batch));
+  // bf16 rows that a bulk copy can fetch (16-byte multiples) and 1024 threads can hold: one fused launch
+  const size_t slot = ((size_t)V * 2 + 127) / 128 * 128, smem = kFusedSlots * slot + 2 * kFusedSlots * 8 + 128;
+  const bool fused = dtype == HSD_BF16 && V % 8 == 0 && V <= kFusedMaxV && smem <= 220 * 1024 && ((uintptr_t)p & 15) == 0 &&
+                     (q == nullptr || ((uintptr_t)q & 15) == 0) && t_max < kFusedConsumers;
+  if (fused) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      HSD_CUDA_OK(cudaFuncSetAttribute(verify_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+      attr_set = true;
+    }
+    HSD_CUDA_OK(cudaMemsetAsync(counters, 0, verify_counter_bytes(batch), s));
+    FusedArgs a;
+    a.p = (const __nv_bfloat16 *)p; a.q = (const __nv_bfloat16 *)q; a.tokens = tokens; a.V = V; a.t_max = t_max; a.batch = batch;
+    a.desc = desc; a.regular_t = regular_t; a.regular_serial = regular_serial; a.regular_level = regular_level;
+    a.stats = stats; a.counters = counters; a.seed = seed; a.out_tokens = out_tokens; a.out_n = out_n;
+    a.write_in_place = write_in_place; a.coin24 = coin24; a.status = nullptr;
+    const int n_items = batch * (2 * t_max + 1);
+    verify_fused_kernel<<<std::min(fused_sm_count(), n_items), kFusedThreads, smem, s>>>(a);
+    hsd_count_launches(1);
+    return hsd_launch_status();
+  }
   return dtype == HSD_BF16 ? launch_verify_t<__nv_bfloat16>(p, q, tokens, V, batch, t_max, desc, regular_t, regular_serial,
-                                                            regular_level, scratch, seed, out_tokens, out_n, write_in_place, s, coin24)
+                                                            regular_level, stats, seed, out_tokens, out_n, write_in_place, s, coin24)
                            : launch_verify_t<float>(p, q, tokens, V, batch, t_max, desc, regular_t, regular_serial,
-                                                    regular_level, scratch, seed, out_tokens, out_n, write_in_place, s, coin24);
+                                                    regular_level, stats, seed, out_tokens, out_n, write_in_place, s, coin24);
 }
 
 // ------------------------------------------------------------------------------ static scratch
 // Scratch for hsd_verify_level_static: lives in the library image, so every GPU that loads the
 // library holds these bytes until the process exits.  One RowStat per logits row of a call.
-constexpr int kStaticStatRows = 4096;                       // 64 KiB
-static __device__ __align__(256) unsigned char g_static_verify_scratch[kStaticStatRows * sizeof(RowStat)];
+constexpr int kStaticStatRows = 4096;                       // 64 KiB of row statistics + 32.25 KiB of counters and queue
+constexpr size_t kStaticScratchBytes = kStaticStatRows * sizeof(RowStat) + ((2 * kStaticStatRows + 2) * 4 + 255) / 256 * 256;
+static __device__ __align__(256) unsigned char g_static_verify_scratch[kStaticScratchBytes];
 
 // In host code the array's name is only a stand-in for the symbol, not a device address: the
-// address has to be asked for, once per device, with that device current.
-static void *g_static_scratch_ptr[64] = {nullptr};
+// address has to be asked for, once per device, with that device current.  The answer is kept per
+// device in an atomic (two host threads may make a device's first call at once: both look the
+// symbol up and store the same value).  It does not survive cudaDeviceReset(): a process that
+// resets a device must not use this entry point on it afterwards.
+static std::atomic<void *> g_static_scratch_ptr[64];
 static int static_scratch_address(void **out) {
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HSD_E_CUDA;
-  if (!g_static_scratch_ptr[dev]) {
-    void *p = nullptr;
+  void *p = g_static_scratch_ptr[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress(&p, g_static_verify_scratch) != cudaSuccess || !p) return HSD_E_CUDA;
-    g_static_scratch_ptr[dev] = p;
+    g_static_scratch_ptr[dev].store(p, std::memory_order_release);
   }
-  *out = g_static_scratch_ptr[dev];
+  *out = p;
   return HSD_OK;
 }
 
@@ -382,8 +737,8 @@ int hsd_verify_level_static(int level, const void *target_logits, const void *dr
   void *scratch = nullptr;
   int st = hsd::static_scratch_address(&scratch);          // first call on this device looks the symbol up
   if (st) return st;
-  // every RowStat the decision reads is written by the statistics kernel of the same call first,
-  // so nothing left over from an earlier call needs clearing
+  // every RowStat the decision reads is written by the same call first; the per-sequence counters have to start
+  // at zero and are cleared on the stream inside launch_verify (a memset node, no allocation)
   return hsd::launch_verify(target_logits, draft_logits, const_cast<int32_t *>(draft_tokens), dtype, vocab, batch, t,
                             nullptr, t, (u32)call_serial, (u32)level, scratch, seed, out_tokens, out_n_accepted, 0,
                             (cudaStream_t)stream);

@@ -55,8 +55,11 @@ __device__ __forceinline__ u32 exp_weight(float l, float m) {
 // Two weights at once with the packed fp32 multiply / add of sm_100 (each half is an IEEE
 // round-to-nearest operation, and t + (-j) equals t - j exactly, so the results are bit-identical
 // to exp_weight); halves the instruction count of the vocabulary-wide pass.
-__device__ __forceinline__ void exp_weight2(float l0, float l1, float m, u32 &e0, u32 &e1) {
-  float2 x = __fadd2_rn(make_float2(l0, l1), make_float2(-m, -m));
+__device__ __forceinline__ void exp_weight2m(float l0, float l1, float m0, float m1, u32 &e0, u32 &e1);
+__device__ __forceinline__ void exp_weight2(float l0, float l1, float m, u32 &e0, u32 &e1) { exp_weight2m(l0, l1, m, m, e0, e1); }
+// ... with a row maximum of its own for each half (two rows side by side)
+__device__ __forceinline__ void exp_weight2m(float l0, float l1, float m0, float m1, u32 &e0, u32 &e1) {
+  float2 x = __fadd2_rn(make_float2(l0, l1), make_float2(-m0, -m1));
   x.x = fmaxf(x.x, -32.0f);
   x.y = fmaxf(x.y, -32.0f);
   const float log2e = __uint_as_float(0x3FB8AA3Bu);
@@ -96,29 +99,54 @@ __device__ __forceinline__ u64 cdf_threshold(u32 U, u64 total) {
   return (u64)U * (total >> 24) + (((u64)U * (total & 0xFFFFFFull)) >> 24);
 }
 
-// ---- block-wide reductions (blockDim.x a multiple of 32, at most 1024)
+// ---- block-wide reductions over a group of threads: the whole block (blockDim.x a multiple of 32, at most
+// 1024), or the first N threads of a block that has other warps besides (named barrier ID).
+struct WholeBlock {
+  __device__ static __forceinline__ void sync() { __syncthreads(); }
+  __device__ static __forceinline__ int threads() { return blockDim.x; }
+};
+template <int ID, int N> struct FirstThreads {
+  __device__ static __forceinline__ void sync() { asm volatile("bar.sync %0, %1;" ::"n"(ID), "n"(N) : "memory"); }
+  __device__ static __forceinline__ int threads() { return N; }
+};
+
+template <class G = WholeBlock>
 __device__ __forceinline__ float block_max(float v, float *sh /*[32]*/) {
   for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-  int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
-  __syncthreads();
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = G::threads() >> 5;
+  G::sync();
   if (l == 0) sh[w] = v;
-  __syncthreads();
+  G::sync();
   float r = (l < nw) ? sh[l] : -INFINITY;
   for (int o = 16; o > 0; o >>= 1) r = fmaxf(r, __shfl_xor_sync(0xFFFFFFFFu, r, o));
   return r;
 }
 
+// Sum of one u64 per thread; every thread gets the total.
+template <class G = WholeBlock>
+__device__ __forceinline__ u64 block_sum(u64 v, u64 *sh /*[33]*/) {
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = G::threads() >> 5;
+  G::sync();
+  if (l == 0) sh[w] = v;
+  G::sync();
+  u64 r = (l < nw) ? sh[l] : 0ull;
+  for (int o = 16; o > 0; o >>= 1) r += __shfl_xor_sync(0xFFFFFFFFu, r, o);
+  return r;
+}
+
 // Exclusive prefix sum of one u64 per thread in thread order; *total receives the block sum.
+template <class G = WholeBlock>
 __device__ __forceinline__ u64 block_exclusive_scan(u64 v, u64 *sh /*[33]*/, u64 *total) {
-  int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = blockDim.x >> 5;
+  int w = threadIdx.x >> 5, l = threadIdx.x & 31, nw = G::threads() >> 5;
   u64 inc = v;
   for (int o = 1; o < 32; o <<= 1) {
     u64 n = __shfl_up_sync(0xFFFFFFFFu, inc, o);
     if (l >= o) inc += n;
   }
-  __syncthreads();
+  G::sync();
   if (l == 31) sh[w] = inc;
-  __syncthreads();
+  G::sync();
   if (w == 0) {
     u64 t = (l < nw) ? sh[l] : 0ull, ti = t;
     for (int o = 1; o < 32; o <<= 1) {
@@ -128,7 +156,7 @@ __device__ __forceinline__ u64 block_exclusive_scan(u64 v, u64 *sh /*[33]*/, u64
     if (l < nw) sh[l] = ti - t;          // exclusive warp offsets
     if (l == 31) sh[32] = ti;            // block total
   }
-  __syncthreads();
+  G::sync();
   *total = sh[32];
   return sh[w] + inc - v;
 }
@@ -200,18 +228,18 @@ __device__ __forceinline__ float chunk_max(const Chunk32 &c, int V, int k0) {
 }
 // Inverse CDF over weights weight(i) of the thread's own 32 tokens (i = local index, compile-time in the
 // unrolled loops).  Same result as block_inverse_cdf with the same weights.
-template <class WeightFn>
+template <class G = WholeBlock, class WeightFn>
 __device__ __forceinline__ int block_inverse_cdf_chunk(int V, int k0, u32 U, WeightFn weight, u64 *sh64 /*[34]*/, u64 *total_out) {
   u64 local = 0;
 #pragma unroll
   for (int i = 0; i < kChunkTokens; ++i)
     if (k0 + i < V) local += weight(i);
   u64 total;
-  u64 excl = block_exclusive_scan(local, sh64, &total);
+  u64 excl = block_exclusive_scan<G>(local, sh64, &total);
   if (total_out) *total_out = total;
   int *result = reinterpret_cast<int *>(&sh64[33]);
   if (threadIdx.x == 0) *result = -1;
-  __syncthreads();
+  G::sync();
   if (total != 0) {
     u64 tau = cdf_threshold(U, total);
     if (tau >= excl && tau < excl + local) {
@@ -226,9 +254,9 @@ __device__ __forceinline__ int block_inverse_cdf_chunk(int V, int k0, u32 U, Wei
       }
     }
   }
-  __syncthreads();
+  G::sync();
   int r = *result;
-  __syncthreads();
+  G::sync();
   return r;
 }
 

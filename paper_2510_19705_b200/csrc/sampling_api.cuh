@@ -37,8 +37,11 @@ int launch_draft_sample(const void *logits, int dtype, int V, const SampleRow *d
 // coin24 != kNoCoin: the ablation of Appendix "Examining the assumptions": every accept test becomes a biased
 // coin, accepted iff the test's own 24-bit uniform is below coin24 (= acceptance probability x 2^24).
 constexpr u32 kNoCoin = 0xFFFFFFFFu;
+// scratch: verify_scratch_bytes(batch, t_max) bytes, 16-byte aligned.  It starts with the counters and the
+// decision queue of the fused kernel, which are cleared on the stream before the kernel.
 int launch_verify(const void *p, const void *q, int32_t *tokens, int dtype, int V, int batch, int t_max,
-                  const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch, u64 seed,
-                  int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s, u32 coin24 = kNoCoin);
+                  const VerifySeq *desc, int regular_t, u32 regular_serial, u32 regular_level, void *scratch,
+                  u64 seed, int32_t *out_tokens, int32_t *out_n, int write_in_place, cudaStream_t s,
+                  u32 coin24 = kNoCoin);
 
 }  // namespace hsd

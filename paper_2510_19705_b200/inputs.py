@@ -44,6 +44,27 @@ WORKLOADS = {
 }
 
 
+# Hierarchies of separate models (one decoder per level, shared vocabulary): list of model configs, weight seeds.
+STACKS = {
+    # fp32, three decoders of different depth / width / head layout (vocabulary 512)
+    "tiny_stack": dict(models=[model_cfg(1, 64, 2, 2, 192, 512, "fp32"), model_cfg(2, 96, 4, 2, 256, 512, "fp32", head_dim=32),
+                               model_cfg(3, 128, 4, 4, 512, 512, "fp32")],
+                       weight_seeds=(21, 22, 23), T=(3, 2), prompt=16, n_new=48, page=16, prompt_seed=2),
+    # bf16 on the tensor-core path: two drafters of their own shape below the mini3 target
+    "mini_stack": dict(models=[model_cfg(1, 256, 4, 1, 512, 2048, "bf16", head_dim=64), model_cfg(2, 512, 8, 2, 704, 2048, "bf16", head_dim=64),
+                               model_cfg(6, 256, 8, 2, 704, 2048, "bf16", head_dim=32)],
+                       weight_seeds=(31, 32, 7), T=(3, 2), prompt=24, n_new=40, page=16, prompt_seed=7),
+}
+
+
+def truncated_model(cfg, weights, n_layers):
+    """The first n_layers layers of a decoder as a model of its own (same tensors, no copies): with the shared final
+    norm and head this is early-exit level e = n_layers written as a separate model."""
+    c = dict(cfg, n_layers=n_layers)
+    w = dict(weights, layers=list(weights["layers"][:n_layers]))
+    return c, w
+
+
 def _gen(seed, device):
     g = torch.Generator(device=device)
     g.manual_seed(int(seed))

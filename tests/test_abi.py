@@ -31,7 +31,7 @@ def test_strerror_and_argument_validation_need_no_gpu():
     assert lib.hsd_draft_sample(None, 1, 1, 8, 0, 0, 0, None, None) == -1
     assert lib.hsd_verify_level(0, None, None, None, 1, 1, 8, 0, 0, 0, None, 0, None, None, None) == -1
     assert lib.hsd_verify_workspace_bytes(0, 3) == 0
-    assert lib.hsd_verify_workspace_bytes(4, 3) == 4 * 7 * 16
+    assert lib.hsd_verify_workspace_bytes(4, 3) == 256 + 4 * 7 * 16      # counters (one per sequence, padded) + row statistics
 
 
 def test_context_setters_reject_a_null_context_without_a_gpu():

@@ -140,11 +140,12 @@ def test_page_size_does_not_change_the_stream(lib):
 
 
 @pytest.mark.parametrize("name", ["mini3", "mini4long"])
-def test_folded_finish_phases_give_the_stream_of_the_separate_phases(lib, name, monkeypatch):
+def test_folded_finish_phases_give_the_stream_of_the_separate_phases(lib, name):
     """Decode passes fold the QKV finish (piece sum, rotary embedding, cache write) into the attention phase and,
     with at most four rows, the gate / up finish (piece sum, SwiGLU) into the down projection, whose CTAs build
-    their activation tiles in shared memory.  HSD_NO_FUSE_QKV / HSD_NO_FUSE_GU keep the separate phases.  Same
-    sums in the same order: all four combinations give the same token stream."""
+    their activation tiles in shared memory; the norm after a residual projection starts on idle CTAs without a
+    grid barrier in between.  hsd_set_phase_folding keeps the separate phases / the barrier.  Same sums in the same
+    order: every combination gives the same token stream."""
     wl = inputs.WORKLOADS[name]
     cfg = wl["model"]
     w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
@@ -152,13 +153,10 @@ def test_folded_finish_phases_give_the_stream_of_the_separate_phases(lib, name, 
     prompts = inputs.make_prompts(cfg["vocab"], batch, wl["prompt"], wl["prompt_seed"]).cuda()
     max_seq = wl["prompt"] + wl["n_new"] + sum(wl["T"]) + len(wl["exits"]) + 8
     outs = []
-    for keep in ((), ("HSD_NO_FUSE_QKV",), ("HSD_NO_FUSE_GU",), ("HSD_NO_FUSE_QKV", "HSD_NO_FUSE_GU")):
-        for k in ("HSD_NO_FUSE_QKV", "HSD_NO_FUSE_GU"):
-            if k in keep:
-                monkeypatch.setenv(k, "1")
-            else:
-                monkeypatch.delenv(k, raising=False)
+    for fold_qkv, fold_gu, early in ((True, True, True), (False, True, True), (True, False, False), (False, False, False),
+                                     (True, True, False)):
         eng = lib.Hsd(cfg, w, wl["exits"], wl["T"], max_batch=batch, max_seq=max_seq, page_size=wl["page"])
+        eng.set_phase_folding(fold_qkv, fold_gu, early)
         outs.append(eng.generate(prompts, wl["n_new"], 1)[0].cpu())
         eng.close()
     for o in outs[1:]:
@@ -277,3 +275,66 @@ def test_iid_coin_acceptance_streams_match_oracle(lib):
     toks, stats, _ = eng.generate(p_gpu, wl["n_new"], 0)
     want, run = _oracle_run(om, T, prompts[0].tolist(), wl["n_new"], 0)
     assert np.array_equal(toks[0].cpu().numpy(), want)
+
+
+# ----------------------------------------------------------------------------- separate models (one decoder per level)
+def _to_cuda(w):
+    return {k: (v.cuda() if k != "layers" else [{n: t.cuda() for n, t in l.items()} for l in v]) for k, v in w.items()}
+
+
+def _setup_stack(name, lib, max_batch=1):
+    from oracle.transformer import ModelStack
+    st = inputs.STACKS[name]
+    cfgs = st["models"]
+    w_cpu = [inputs.make_weights(c, s) for c, s in zip(cfgs, st["weight_seeds"])]
+    T = list(st["T"])
+    max_seq = st["prompt"] + st["n_new"] + sum(T) + len(cfgs) + 8
+    eng = lib.Hsd(cfgs, [_to_cuda(w) for w in w_cpu], None, T, max_batch=max_batch, max_seq=max_seq, page_size=st["page"])
+    om = ModelStack([Transformer(c, inputs.weights_to_numpy(w), (c["n_layers"],)) for c, w in zip(cfgs, w_cpu)])
+    prompts = inputs.make_prompts(cfgs[0]["vocab"], max_batch, st["prompt"], st["prompt_seed"])
+    return st, eng, om, prompts, T
+
+
+def test_separate_models_fp32_streams_match_oracle_bit_exact(lib):
+    """Section 3.1's general hierarchy (hsd_create_models): three decoders of different depth, width and head
+    layout over one vocabulary, each with a KV cache of its own.  Streams and per-level counters equal the
+    oracle's run of Algorithm 1 over the same three models; a batch gives each sequence its single-run stream."""
+    st, eng, om, prompts, T = _setup_stack("tiny_stack", lib, max_batch=3)
+    for seed in range(3):
+        toks, stats, _ = eng.generate(prompts[:1].cuda(), st["n_new"], seed)
+        want, run = _oracle_run(om, T, prompts[0].tolist(), st["n_new"], seed)
+        assert np.array_equal(toks[0].cpu().numpy(), want), seed
+        _check_stats(stats, run)
+    toks, _, _ = eng.generate(prompts.cuda(), st["n_new"], 1)
+    for b in range(3):
+        want, _ = _oracle_run(om, T, prompts[b].tolist(), st["n_new"], 1, seq=b)
+        assert np.array_equal(toks[b].cpu().numpy(), want), b
+
+
+def test_separate_models_equal_early_exits_when_they_are_truncated_copies(lib):
+    """The first e_i layers of one decoder handed over as separate models (own caches, own prompt passes) compute
+    the same functions M_i as the early-exit hierarchy: identical streams and counters (fp32, and bf16 on the
+    tensor-core path)."""
+    for name in ("tiny3", "mini3"):
+        wl = inputs.WORKLOADS[name]
+        cfg, exits, T = wl["model"], wl["exits"], list(wl["T"])
+        w = _to_cuda(inputs.make_weights(cfg, wl["weight_seed"]))
+        prompts = inputs.make_prompts(cfg["vocab"], 1, wl["prompt"], wl["prompt_seed"]).cuda()
+        max_seq = wl["prompt"] + wl["n_new"] + sum(T) + len(exits) + 8
+        a = lib.Hsd(cfg, w, exits, T, max_batch=1, max_seq=max_seq, page_size=wl["page"])
+        parts = [inputs.truncated_model(cfg, w, e) for e in exits]
+        b = lib.Hsd([p[0] for p in parts], [p[1] for p in parts], None, T, max_batch=1, max_seq=max_seq, page_size=wl["page"])
+        ta, sa, _ = a.generate(prompts, wl["n_new"], 3)
+        tb, sb, _ = b.generate(prompts, wl["n_new"], 3)
+        assert torch.equal(ta, tb), name
+        for x, y in zip(sa, sb):
+            assert all(x[k] == y[k] for k in STAT_KEYS), name
+        a.close()
+        b.close()
+
+
+def test_separate_models_bf16_decisions_and_logits(lib, tmp_path):
+    """Separate bf16 decoders on the tensor-core path (the persistent forward per model): every decision follows
+    the oracle on the logged logits, the logits match the oracle's forward of the level's own model within 2e-2."""
+    st, eng, om, prompts, T = _setup_stack("mini_stack", lib)
+    _bf16_trace_check(lib, st, eng, om, prompts, tmp_path)

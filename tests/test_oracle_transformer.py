@@ -156,3 +156,29 @@ def test_bf16_forward_is_sensitive_to_fp32_level_noise():
         T.bf16_round = orig
     rel = float(np.sqrt(((got - ref) ** 2).mean()) / ref.std())
     assert 2e-4 < rel < 5e-2, rel          # orders of magnitude above the 2e-6 that went in, still small
+
+
+def test_stack_of_truncated_copies_is_the_early_exit_model():
+    """Section 3.1's list of models, pinned to the early-exit family: the first e_i layers of one decoder written
+    as separate models (own key / value memo each) give the rows, and Algorithm 1 the token stream and counters,
+    of the early-exit model, exactly."""
+    from oracle.hsd import HSD, SpecDecisions
+    from oracle.transformer import ModelStack
+    w, m = _setup(CFG32)
+    w_np = inputs.weights_to_numpy(w)
+    exits = (1, 2, 3)
+    parts = []
+    for e in exits:
+        c, wt = inputs.truncated_model(CFG32, w_np, e)
+        parts.append(Transformer(c, wt, (e,)))
+    stack = ModelStack(parts)
+    toks = inputs.make_prompts(CFG32["vocab"], 1, 9, seed=4)[0].tolist()
+    for level in range(3):
+        a = m.rows(level, toks, [3, 1, 4])
+        b = stack.rows(level, toks, [3, 1, 4])
+        assert all(np.array_equal(x, y) for x, y in zip(a, b))
+    m.reset()
+    stack.reset()
+    r1, r2 = HSD(m, (2, 2), SpecDecisions(5)), HSD(stack, (2, 2), SpecDecisions(5))
+    assert r1.generate(toks, 24) == r2.generate(toks, 24)
+    assert [s.as_tuple() for s in r1.stats] == [s.as_tuple() for s in r2.stats]

@@ -40,3 +40,25 @@ def test_static_scratch_variant_rejects_what_does_not_fit(lib):
         lib.hsd_verify_level_static(1, p, q, x, 0, 0, out, n)
     lib.hsd_verify_level_static(1, p[:455].contiguous(), q[:455].contiguous(), x[:455].contiguous(), 0, 0, out, n)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("dtype,V", [("bf16", 64), ("fp32", 16)])
+def test_static_scratch_variant_at_exactly_its_limit_and_without_allocating(lib, dtype, V):
+    # batch * (2 t + 1) == 4096: the last row of statistics and the last counter of the built-in array are used
+    B, t = 4096, 0
+    p, _ = inputs.make_accept_logits(B, 1, V, seed=5, device="cuda", dtype=dtype)
+    p = p[:, :1].contiguous()
+    out = torch.full((B, 1), -7, dtype=torch.int32, device="cuda")
+    n = torch.full((B,), -7, dtype=torch.int32, device="cuda")
+    want_out, want_n = lib.hsd_verify_level(1, p, None, None, 3, 0)
+    lib.hsd_verify_level_static(1, p, None, None, 3, 0, out, n)          # first use: kernels loaded, address looked up
+    torch.cuda.synchronize()
+    assert torch.equal(out, want_out) and torch.equal(n, want_n)
+    # the device's free memory is the same before and after a call: nothing was allocated (or freed)
+    free_before, _ = torch.cuda.mem_get_info()
+    lib.hsd_verify_level_static(1, p, None, None, 3, 1, out, n)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    want_out, want_n = lib.hsd_verify_level(1, p, None, None, 3, 1)
+    assert torch.equal(out, want_out) and torch.equal(n, want_n)
