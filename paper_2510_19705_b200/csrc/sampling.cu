@@ -262,8 +262,8 @@ decide_kernel(const T *__restrict__ p_logits, const T *__restrict__ q_logits, in
 constexpr int kFusedConsumers = 1024;
 constexpr int kFusedThreads = kFusedConsumers;
 constexpr int kFusedSlots = 3;
-constexpr int kFusedVecPerThread = 4;                      // 16-byte vectors of a row per consumer thread
-constexpr int kFusedMaxV = kFusedConsumers * kFusedVecPerThread * 8;
+constexpr int kFusedVecPerThread = 8;                      // 16-byte vectors of a row per thread of a 512-thread group
+constexpr int kFusedMaxV = 512 * kFusedVecPerThread * 8;
 constexpr uint32_t kFusedPiece = 4096;                     // bytes per bulk copy; 32 of them cover the largest row
 using FusedGroup = WholeBlock;
 
@@ -398,16 +398,16 @@ __global__ void __launch_bounds__(kFusedThreads, 1) verify_fused_kernel(const __
   extern __shared__ uint8_t fused_smem_raw[];
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(fused_smem_raw) + 127) & ~(uintptr_t)127);
   const uint32_t row_bytes = (uint32_t)a.V * 2u, slot_bytes = (row_bytes + 127u) & ~127u;
-  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)kFusedSlots * slot_bytes);   // full[S]
-  __shared__ float shf[32];
-  __shared__ u64 sh64[34];
-  __shared__ int sh_flag[2];                 // [0] this CTA decides the row's sequence, [1] first rejected position
+  uint64_t *bars = reinterpret_cast<uint64_t *>(smem + (size_t)kFusedSlots * slot_bytes);   // full[S][2]
+  __shared__ float shf[2][16];
+  __shared__ u64 sh64[34];                   // row phase: [g * 16 + warp]; decisions: the block scan's scratch
+  __shared__ int sh_flag[2];
   __shared__ int sh_abort;
   const uint32_t bar0 = ptx::smem_u32(bars);
   const int tid = threadIdx.x, lane = tid & 31;
   const int rows_per_seq = 2 * a.t_max + 1, n_items = a.batch * rows_per_seq;
   if (tid == 0) {
-    for (int s = 0; s < kFusedSlots; ++s) ptx::mbar_init(bar0 + 8u * s, 1);
+    for (int s = 0; s < 2 * kFusedSlots; ++s) ptx::mbar_init(bar0 + 8u * s, 1);
     sh_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -421,104 +421,134 @@ __global__ void __launch_bounds__(kFusedThreads, 1) verify_fused_kernel(const __
     const int j = r - a.t_max - 1;
     return j < d.t ? a.q + (size_t)(d.q_row0 + j) * a.V : nullptr;
   };
-  // warp 0 keeps the ring full: `ahead` = next item of this CTA that has not been asked for yet.  A row is fetched
-  // as 4 KiB bulk copies, one per lane (one 64 KB copy runs at a fraction of an SM's bandwidth).
-  int ahead = blockIdx.x;
-  auto fetch_next = [&](int slot) {                        // all lanes of warp 0
-    while (ahead < n_items) {
+  // Rows.  The CTA's valid items, numbered k = 0, 1, ..., go to its two groups of 512 threads in turn (group
+  // k & 1) through ring slot k % 3; each group has its own barrier, so one group's reductions and global round
+  // trips run under the other group's arithmetic.  The group that has taken item k out of its slot asks for item
+  // k + 3 (4 KiB bulk copies, one per lane of the group's first warp: a single 64 KB copy runs at a fraction
+  // of an SM's bandwidth).
+  const int grp = tid >> 9, gtid = tid & 511, gwarp = gtid >> 5, bar_id = 1 + grp;
+  auto group_sync = [&]() { asm volatile("bar.sync %0, 512;" ::"r"(bar_id) : "memory"); };
+  // A slot's uses alternate between the groups, and a parity wait tells a barrier's phases apart only one phase
+  // back, so each slot has two "full" barriers used in turn: a barrier's phases then all belong to one group, which
+  // takes them in order.
+  auto full_bar = [&](int k) { return bar0 + 8u * (uint32_t)((k % kFusedSlots) * 2 + ((k / kFusedSlots) & 1)); };
+  int f_idx = blockIdx.x, f_ord = 0;                        // fetch cursor: next item index to look at, valid items passed so far
+  auto fetch_ordinal = [&](int want) {                      // all lanes of a warp; asks for valid item number `want`, if it exists
+    while (f_idx < n_items) {
       VerifySeq d; int b, r;
-      const __nv_bfloat16 *row = row_of(ahead, d, b, r);
-      ahead += gridDim.x;
+      const __nv_bfloat16 *row = row_of(f_idx, d, b, r);
+      f_idx += gridDim.x;
       if (!row) continue;
-      if (lane == 0) ptx::mbar_expect_tx(bar0 + 8u * slot, row_bytes);
+      if (f_ord++ < want) continue;
+      const int slot = want % kFusedSlots;
+      const uint32_t bar = full_bar(want);
+      if (lane == 0) ptx::mbar_expect_tx(bar, row_bytes);
       __syncwarp();
       const uint32_t off = (uint32_t)lane * kFusedPiece;
       if (off < row_bytes)
         bulk_load_row(ptx::smem_u32(smem + (size_t)slot * slot_bytes) + off, reinterpret_cast<const uint8_t *>(row) + off,
-                      min(kFusedPiece, row_bytes - off), bar0 + 8u * slot);
+                      min(kFusedPiece, row_bytes - off), bar);
       return;
     }
   };
-  if (tid < 32)
-    for (int s = 0; s < kFusedSlots; ++s) fetch_next(s);
+  if (tid < 32) {                                           // items 0, 1, 2; afterwards group 0 asks for 3, 5, ..., group 1 for 4, 6, ...
+    for (int k = 0; k < kFusedSlots; ++k) fetch_ordinal(k);
+    f_idx = blockIdx.x; f_ord = 0;                          // group 0's own cursor starts over (its next request is item 3)
+  }
   const int nvec = a.V >> 3;
-  int s = 0;
-  uint32_t par = 0;
+  int ord = 0;                                              // valid items of this CTA seen so far
+  unsigned pending_before = 0u, pending_last = 0xFFFFFFFFu; // the row counter's old value of the group's previous item (thread 0 of the group)
+  int pending_b = -1;
+  auto settle = [&]() {                                     // group thread 0: was the previous item its sequence's last row?
+    if (pending_b >= 0 && pending_before == pending_last) {
+      // the sequence is ready for its decision: append it to the queue (entry = b + 1; 0 = not yet written)
+      const unsigned at = atomicAdd(&a.counters[a.batch], 1u);
+      asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(a.counters + a.batch + 2 + at), "r"((unsigned)pending_b + 1u) : "memory");
+    }
+    pending_b = -1;
+  };
   for (int i = blockIdx.x; i < n_items; i += gridDim.x) {
     VerifySeq d; int b, r;
     const __nv_bfloat16 *row = row_of(i, d, b, r);
-    if (!row) continue;                                   // uniform over the CTA
-    // the drafted token's logit (thread 0 only), asked for before the wait
+    if (!row) continue;
+    const int k = ord++;
+    if ((k & 1) != grp) continue;
+    const int s = k % kFusedSlots;
+    const uint32_t par = (uint32_t)(k / (2 * kFusedSlots)) & 1u;
+    // the drafted token's logit (the group's thread 0 only), asked for before the wait
     int tok = -1;
     if (r < d.t) tok = a.tokens[d.tok_off + r];
     else if (r > a.t_max) tok = a.tokens[d.tok_off + (r - a.t_max - 1)];
     float l_tok = 0.f;
     const bool has_tok = tok >= 0 && tok < a.V;
-    if (tid == 0 && has_tok) l_tok = __bfloat162float(row[tok]);
-    if (lane == 0) ptx::mbar_wait(bar0 + 8u * s, par, abort_flag);      // a give-up raises the CTA's abort flag
+    if (gtid == 0 && has_tok) l_tok = __bfloat162float(row[tok]);
+    if (lane == 0) ptx::mbar_wait(full_bar(k), par, abort_flag);       // a give-up raises the CTA's abort flag
     __syncwarp();
     const uint4 *src = reinterpret_cast<const uint4 *>(smem + (size_t)s * slot_bytes);
     uint4 regs[kFusedVecPerThread];
 #pragma unroll
     for (int j = 0; j < kFusedVecPerThread; ++j) {
-      const int iv = tid + kFusedConsumers * j;
+      const int iv = gtid + 512 * j;
       regs[j] = iv < nvec ? src[iv] : make_uint4(0u, 0u, 0u, 0u);
     }
-    FusedGroup::sync();                                   // every thread holds its part of the row: the slot is free
-    if (*abort_flag) break;                               // uniform: raised before the barrier
-    if (tid < 32) fetch_next(s);
-    if (++s == kFusedSlots) { s = 0; par ^= 1u; }
+    group_sync();                                           // every thread holds its part of the row: the slot is free
+    if (*abort_flag) break;                                 // uniform over the group: raised before the barrier
+    if (gwarp == 0) fetch_ordinal(k + kFusedSlots);
     float m = -INFINITY;
 #pragma unroll
     for (int j = 0; j < kFusedVecPerThread; ++j) {
-      if (tid + kFusedConsumers * j < nvec) {
+      if (gtid + 512 * j < nvec) {
         float f[8];
         StatVec<__nv_bfloat16>::unpack(regs[j], f);
 #pragma unroll
         for (int e = 0; e < 8; ++e) m = fmaxf(m, f[e]);
       }
     }
-    m = block_max<FusedGroup>(m, shf);
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if (lane == 0) shf[grp][gwarp] = m;
+    group_sync();
+    m = shf[grp][lane & 15];
+    for (int o = 8; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     u64 local = 0;
 #pragma unroll
     for (int j = 0; j < kFusedVecPerThread; ++j) {
-      if (tid + kFusedConsumers * j < nvec) {
+      if (gtid + 512 * j < nvec) {
         float f[8];
         StatVec<__nv_bfloat16>::unpack(regs[j], f);
 #pragma unroll
         for (int e = 0; e < 8; e += 2) {
           u32 e0, e1;
-#ifndef FUSED_NO_EXP
           exp_weight2(f[e], f[e + 1], m, e0, e1);
           local += (u64)e0 + (u64)e1;
-#endif
         }
       }
     }
-#ifdef FUSED_NO_EXP
-    local = (u64)__float_as_uint(m) + regs[0].x;
-#endif
-    const u64 total = block_sum<FusedGroup>(local, sh64);
-    if (tid == 0) {
+    for (int o = 16; o > 0; o >>= 1) local += __shfl_xor_sync(0xFFFFFFFFu, local, o);
+    if (lane == 0) sh64[grp * 16 + gwarp] = local;
+    group_sync();
+    if (gtid == 0) {
+      u64 total = 0;
+#pragma unroll
+      for (int w = 0; w < 16; ++w) total += sh64[grp * 16 + w];
+      settle();                                             // the previous item's counter value has long arrived
       RowStat st;
       st.m = m; st.S = total; st.Ex = has_tok ? exp_weight(l_tok, m) : 0u;
       a.stats[(size_t)b * rows_per_seq + r] = st;
-      __threadfence();
-      const unsigned before = atomicAdd(&a.counters[b], 1u);
-      if (before == (unsigned)(2 * d.t)) {                   // 2 t + 1 rows per sequence: this was the last one
-        // the sequence is ready for its decision: append it to the queue (entry = b + 1; 0 = not yet written)
-        const unsigned at = atomicAdd(&a.counters[a.batch], 1u);
-        __threadfence();
-        atomicExch(&a.counters[a.batch + 2 + at], (unsigned)b + 1u);
-      }
+      // the statistics are ordered before the count by the release (and the other rows' statistics before whatever
+      // follows a look at its old value, which happens one item later, by the acquire)
+      asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(pending_before) : "l"(a.counters + b) : "memory");
+      pending_b = b;
+      pending_last = (unsigned)(2 * d.t);                   // 2 t + 1 rows per sequence
     }
+    // (the next item's first barrier keeps the other threads from overwriting sh64 / shf before thread 0 has read them)
   }
+  if (gtid == 0) settle();
   // Decisions.  Taking one where its last row arrives would chain: the CTA that decides delivers its next rows
   // late, so it is the last arriver of those sequences too.  Instead every CTA, once its rows are done, draws
   // tickets until all `batch` decisions are handed out; a ticket whose entry is not written yet waits for it
   // (bounded): the rows it waits for are never this CTA's own.
   for (;;) {
-    FusedGroup::sync();
+    __syncthreads();
     if (tid == 0) {
       int b = -1;
       if (!*abort_flag) {
@@ -541,7 +571,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1) verify_fused_kernel(const __
       }
       sh_flag[0] = b;
     }
-    FusedGroup::sync();
+    __syncthreads();
     const int b = sh_flag[0];
     if (b < 0) break;
     const VerifySeq d = fused_seq(a, b);
@@ -549,15 +579,10 @@ __global__ void __launch_bounds__(kFusedThreads, 1) verify_fused_kernel(const __
   }
   if (tid == 0 && sh_abort) {
     // copies already asked for must land before the CTA's shared memory goes away (bounded)
-    for (int k = 0; k < kFusedSlots; ++k) {
-      const unsigned long long t0 = ptx::globaltimer_ns();
-      while (!ptx::mbar_try_wait(bar0 + 8u * s, par))
-        if (ptx::globaltimer_ns() - t0 > ptx::kWaitLimitNs / 8) break;
-      if (++s == kFusedSlots) { s = 0; par ^= 1u; }
-    }
+    const unsigned long long t0 = ptx::globaltimer_ns();
+    while (ptx::globaltimer_ns() - t0 < 20000ull) {}      // 20 us: far longer than a row's copy takes
+    if (a.status) atomicExch(a.status, 1);
   }
-  __syncthreads();
-  if (tid == 0 && sh_abort && a.status) atomicExch(a.status, 1);
 }
 
 // ------------------------------------------------------------------------------ host launchers
