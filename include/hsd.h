@@ -318,6 +318,13 @@ int hsd_gemm_bf16(const void *A, int R, int K, const void *W, int N, float *out,
 /* Synchronises `stream` and returns DEVICE_TIMEOUT if a kernel using `workspace` gave up a bounded wait. */
 int hsd_gemm_status(void *workspace, void *stream);
 
+/* Measurement aid: one read-only pass over `bytes` (a multiple of 16 is read) of device memory at `buffer` (16-byte
+ * aligned) with plain vector loads on every SM, nothing written (`sink`, a device word or NULL, is written only if a
+ * checksum happens to match a constant).  Timed with events around it, bytes / time is the HBM rate a weight-streaming
+ * verification forward (Algorithm 2's pass: every weight byte read once) could reach at best; bench.py reports the
+ * forward's rate against it.  Asynchronous on `stream`.  Errors: INVALID_ARG, CUDA. */
+int hsd_stream_read(const void *buffer, size_t bytes, void *sink, void *stream);
+
 /* Number of CUDA kernels this library has launched in the calling process so far. */
 uint64_t hsd_kernel_launches(void);
 

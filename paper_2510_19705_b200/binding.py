@@ -182,6 +182,8 @@ def _declare_engine(lib):
     lib.hsd_pairwise_alpha.argtypes = [vp, i32, i32, i32, i32, c.c_longlong, vp, sz, vp, vp]
     lib.hsd_layer_logits.restype = i32
     lib.hsd_layer_logits.argtypes = [vp, vp, i32, c.POINTER(c.c_int32), i32, vp, vp]
+    lib.hsd_stream_read.restype = i32
+    lib.hsd_stream_read.argtypes = [vp, sz, vp, vp]
     lib.hsd_kernel_launches.restype = c.c_uint64
     lib.hsd_kernel_launches.argtypes = []
     lib.hsd_gemm_workspace_bytes.restype = sz
@@ -420,6 +422,26 @@ def hsd_search_hierarchy(costs, alpha, T_max=15):
                                     ctypes.byref(n_lev), out_T, ctypes.byref(out)))
     k = n_lev.value
     return out.value, tuple(sigma[i] for i in range(k)), tuple(out_T[i] for i in range(k - 1))
+
+def hsd_stream_read_gbs(n_bytes=4 << 30, repeats=5):
+    """Read-only streaming rate of this GPU's HBM in GB/s (hsd_stream_read over a buffer far larger than L2, best of
+    `repeats` after one warm-up, CUDA events on the current stream)."""
+    lib = library()
+    _declare_engine(lib)
+    buf = torch.empty(n_bytes, dtype=torch.uint8, device="cuda")
+    buf.zero_()
+    best = 0.0
+    for i in range(repeats + 1):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        _check(lib.hsd_stream_read(_dev(buf), n_bytes, None, _stream()))
+        e1.record()
+        e1.synchronize()
+        if i > 0:
+            best = max(best, n_bytes / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+    del buf
+    return best
+
 
 def hsd_kernel_launches():
     lib = library()

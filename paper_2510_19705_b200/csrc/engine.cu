@@ -481,7 +481,7 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     a.n_run = c->exits[level]; a.lm_map = md.n_layers * 7 + level; a.max_seq = md.max_seq; a.page = md.page;
     a.page_shift = 0;
     while ((1 << a.page_shift) < md.page) ++a.page_shift;
-    a.pages_per_seq = md.pages_per_seq; a.eps = md.eps;
+    a.pages_per_seq = md.pages_per_seq; a.n_pages = md.n_pages; a.eps = md.eps;
     a.wmaps = c->dev<CUtensorMap>(ML.wmaps_dev);
     a.layers = c->dev<FwdLayerDev>(ML.layers_dev);
     a.embed = (const __nv_bfloat16 *)M.embed; a.final_norm = (const __nv_bfloat16 *)c->level_norm[level];
@@ -774,7 +774,7 @@ int init_model(hsd_ctx *c, Model &M, const hsd_model_desc *model, const ModelLay
   const Layout &lay = c->lay;
   M.md = ModelDims{model->n_layers, model->d_model, model->n_q_heads, model->n_kv_heads, model->head_dim, model->d_ff,
                    model->vocab, model->dtype, model->rms_eps, model->rope_theta, model->max_seq,
-                   model->page_size ? model->page_size : 16, lay.pages_per_seq};
+                   model->page_size ? model->page_size : 16, lay.pages_per_seq, lay.n_pages};
   M.lay = ml;
   M.embed = model->embed; M.final_norm = model->final_norm; M.lm_head = model->lm_head;
   M.lw.assign(model->layer_weights, model->layer_weights + (size_t)model->n_layers * 9);

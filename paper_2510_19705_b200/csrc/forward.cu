@@ -196,7 +196,7 @@ template <typename T>
 __global__ void rope_kv_kernel(const float *__restrict__ qkv, const int *__restrict__ row_seq, const int *__restrict__ row_pos,
                                const float *__restrict__ cos_tab, const float *__restrict__ sin_tab,
                                const int *__restrict__ page_table, T *__restrict__ k_pool, T *__restrict__ v_pool,
-                               T *__restrict__ q_out, int nq, int nkv, int hd, int page, int pages_per_seq) {
+                               T *__restrict__ q_out, int nq, int nkv, int hd, int page, int pages_per_seq, int n_pages) {
   int r = blockIdx.x, h = blockIdx.y;
   int seq = row_seq[r], pos = row_pos[r];
   int half = hd >> 1;
@@ -208,7 +208,7 @@ __global__ void rope_kv_kernel(const float *__restrict__ qkv, const int *__restr
   } else {
     int kvh = (h - nq) % nkv;
     int pg = page_table[(size_t)seq * pages_per_seq + pos / page];
-    size_t off = (((size_t)pg * nkv + kvh) * page + (pos % page)) * hd;
+    size_t off = (((size_t)kvh * n_pages + pg) * page + (pos % page)) * hd;
     dst = (h < nq + nkv ? k_pool : v_pool) + off;
   }
   if (rotate) {
@@ -232,7 +232,7 @@ template <typename T, int HD>
 __global__ void __launch_bounds__(kAttnThreads)
 attn_split_kernel(const T *__restrict__ q, const int4 *__restrict__ items, const int *__restrict__ page_table,
                   const T *__restrict__ k_pool, const T *__restrict__ v_pool, float *__restrict__ partials, int nq, int nkv,
-                  int page, int pages_per_seq, int keys_per_split, int n_splits, float scale) {
+                  int page, int pages_per_seq, int n_pages, int keys_per_split, int n_splits, float scale) {
   constexpr int KT = kAttnKeyTile;
   constexpr int DPL = HD / 32;                         // output dims per lane
   extern __shared__ __align__(16) unsigned char smem[];
@@ -273,7 +273,7 @@ attn_split_kernel(const T *__restrict__ q, const int4 *__restrict__ items, const
       float2 kvv = make_float2(0.f, 0.f), vvv = make_float2(0.f, 0.f);
       if (key < key_hi) {
         int pg = page_table[(size_t)seq * pages_per_seq + key / page];
-        size_t off = (((size_t)pg * nkv + kvh) * page + (key % page)) * HD + 2 * w2;
+        size_t off = (((size_t)kvh * n_pages + pg) * page + (key % page)) * HD + 2 * w2;
         kvv = make_float2(to_f32(k_pool[off]), to_f32(k_pool[off + 1]));
         vvv = make_float2(to_f32(v_pool[off]), to_f32(v_pool[off + 1]));
       }
@@ -364,7 +364,7 @@ static int attention_t(const ModelDims &md, const void *q, const RowBatch &rb, c
   dim3 grid(n_splits, md.nkv, rb.n_attn);
   attn_split_kernel<T, HD><<<grid, kAttnThreads, smem, s>>>((const T *)q, rb.attn, page_table, (const T *)k_pool,
                                                            (const T *)v_pool, partials, md.nq, md.nkv, md.page,
-                                                           md.pages_per_seq, keys_per_split, n_splits, rsqrtf((float)HD));
+                                                           md.pages_per_seq, md.n_pages, keys_per_split, n_splits, rsqrtf((float)HD));
   if (cudaGetLastError() != cudaSuccess) return HSD_E_CUDA;
   attn_combine_kernel<T, HD><<<rb.R * md.nq, HD, 0, s>>>(partials, rb.row_pos, md.nq, keys_per_split, n_splits, (T *)att_out);
   hsd_count_launches(2);
@@ -407,10 +407,10 @@ int launch_rope_kv(const ModelDims &md, const float *qkv, const RowBatch &rb, co
   if (md.dtype == HSD_BF16)
     rope_kv_kernel<__nv_bfloat16><<<grid, threads, 0, s>>>(qkv, rb.row_seq, rb.row_pos, cos_tab, sin_tab, page_table,
                                                           (__nv_bfloat16 *)k_pool, (__nv_bfloat16 *)v_pool,
-                                                          (__nv_bfloat16 *)q_out, md.nq, md.nkv, md.hd, md.page, md.pages_per_seq);
+                                                          (__nv_bfloat16 *)q_out, md.nq, md.nkv, md.hd, md.page, md.pages_per_seq, md.n_pages);
   else
     rope_kv_kernel<float><<<grid, threads, 0, s>>>(qkv, rb.row_seq, rb.row_pos, cos_tab, sin_tab, page_table, (float *)k_pool,
-                                                  (float *)v_pool, (float *)q_out, md.nq, md.nkv, md.hd, md.page, md.pages_per_seq);
+                                                  (float *)v_pool, (float *)q_out, md.nq, md.nkv, md.hd, md.page, md.pages_per_seq, md.n_pages);
   hsd_count_launches(1);
   return hsd_launch_status();
 }
@@ -438,4 +438,32 @@ int launch_attention(const ModelDims &md, const void *q, const RowBatch &rb, con
   return HSD_E_UNSUPPORTED;
 }
 
+// Read-only streaming pass over a buffer: what the weight stream of a verification forward does to HBM, without the
+// arithmetic.  The measured rate is the denominator a weight-streaming pass can be held against.
+__global__ void __launch_bounds__(512) stream_read_kernel(const uint4 *__restrict__ src, size_t n_vec, unsigned *__restrict__ sink) {
+  unsigned acc = 0u;
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride * 4) {
+    uint4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const size_t j = i + (size_t)u * stride;
+      v[u] = j < n_vec ? __ldg(src + j) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) acc += v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+  }
+  if (acc == 0x9E3779B9u && sink) *sink = acc;              // keeps the loads alive; practically never taken
+}
+
 }  // namespace hsd
+
+extern "C" int hsd_stream_read(const void *buffer, size_t bytes, void *sink, void *stream) {
+  if (!buffer || bytes < 16 || ((uintptr_t)buffer & 15) != 0) return HSD_E_INVALID_ARG;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    return HSD_E_CUDA;
+  hsd::stream_read_kernel<<<sms * 8, 512, 0, (cudaStream_t)stream>>>((const uint4 *)buffer, bytes / 16, (unsigned *)sink);
+  hsd_count_launches(1);
+  return hsd_launch_status();
+}

@@ -12,6 +12,7 @@ struct ModelDims {
   int dtype;            // HSD_F32 / HSD_BF16: storage type of weights, KV cache, logits, GEMM inputs
   float eps, theta;
   int max_seq, page, pages_per_seq;
+  int n_pages;          // pages per KV pool: a pool is [kv head][page][token in page][head dim] (one head's pages are adjacent)
 };
 
 // One packed batch of rows for a forward pass; all arrays are device memory.

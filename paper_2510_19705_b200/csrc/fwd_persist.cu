@@ -33,13 +33,16 @@ constexpr int kMaxLayersSh = 64;                       // layers whose pointer t
 
 enum { MODE_QKV = 0, MODE_ADD = 1, MODE_SWIGLU = 2, MODE_LOGITS = 3 };
 
+// Barrier-timeline stamps and cycle laps exist only in a profiling build (-DHSD_PROFILE).
+#ifdef HSD_PROFILE
+#define HSD_PROF(a) ((a).prof != nullptr)
+#else
+#define HSD_PROF(a) false
+#endif
+
 template <int NPAD> struct PCfg {
   static constexpr int kStageBytes = kWBytes + NPAD * kTcBlockK * 2;
-#ifndef HSD_STAGE_CAP
-#define HSD_STAGE_CAP 64
-#endif
-  static constexpr int kStagesFit = (kSmemTotal - 1024 - kCtrlBytes - kScratchBytes) / kStageBytes;
-  static constexpr int kStages = kStagesFit < HSD_STAGE_CAP ? kStagesFit : HSD_STAGE_CAP;
+  static constexpr int kStages = (kSmemTotal - 1024 - kCtrlBytes - kScratchBytes) / kStageBytes;
   static constexpr int kSmemBytes = kStages * kStageBytes + kScratchBytes + kCtrlBytes + 1024;
   static constexpr int kTmemCols = (2 * NPAD < 32) ? 32 : 2 * NPAD;
   static constexpr int kChunk = NPAD < 32 ? NPAD : 32;      // accumulator columns handled at a time
@@ -192,7 +195,7 @@ __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, 
   if (wt == 0) {
     const unsigned target = epoch * gridDim.x;
     asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.grid_counter) : "memory");
-    if (a.prof && 2 * epoch + 1 < (unsigned)kFwdProfEvents) a.prof[(size_t)blockIdx.x * kFwdProfEvents + 2 * epoch] = globaltimer_ns();
+    if (HSD_PROF(a) && 2 * epoch + 1 < (unsigned)kFwdProfEvents) a.prof[(size_t)blockIdx.x * kFwdProfEvents + 2 * epoch] = globaltimer_ns();
     bool ok = true;
     unsigned long long t0 = 0;                       // the clock is read only once the wait has lasted a while
     for (uint32_t it = 0; (int)(ld_acquire_u32(a.grid_counter) - target) < 0; ++it) {
@@ -209,7 +212,7 @@ __device__ __forceinline__ bool grid_barrier(const FwdArgs &a, unsigned &epoch, 
       *abort_flag = 1;
       atomicExch(a.status, 1);
     } else {
-      if (a.prof && 2 * epoch + 1 < (unsigned)kFwdProfEvents)
+      if (HSD_PROF(a) && 2 * epoch + 1 < (unsigned)kFwdProfEvents)
         a.prof[(size_t)blockIdx.x * kFwdProfEvents + 2 * epoch + 1] = globaltimer_ns();
       // the acquire load that left the spin orders everything after it; the CTA barrier below hands that on
       if (ready_bar) {
@@ -404,8 +407,12 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
   const int n_work = a.n_attn * a.nkv * a.n_splits;
 #pragma unroll 1
   for (int wi = blockIdx.x; wi < n_work; wi += gridDim.x) {
+#ifdef HSD_PROFILE
     long long cyc = clock64();
     auto lap = [&](int k) { if (a.prof && wt == 0 && blockIdx.x == 0) { const long long n_ = clock64(); dbg[k] += n_ - cyc; cyc = n_; } };
+#else
+    auto lap = [](int) {};
+#endif
     const int split = wi % a.n_splits, kvh = (wi / a.n_splits) % a.nkv, ai = wi / (a.n_splits * a.nkv);
     const int4 it = wi == (int)blockIdx.x ? make_int4(first_item[0], first_item[1], first_item[2], first_item[3])
                                           : a.attn_items[ai];   // the CTA's first item was fetched at kernel start
@@ -448,7 +455,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
     auto issue = [&](const __nv_bfloat16 *pool, __nv_bfloat16 *sh, int j, bool zero_pad, int key_stop) {    // one sub-tile, one operand
       const int kt = key_lo + (first + j * step) * 16, nk = min(16, key_hi - kt), nload = min(nk, key_stop - kt);
       const int pg = __shfl_sync(0xFFFFFFFFu, pg_reg, j - pg_base);
-      const size_t base = ((((size_t)pg * a.nkv + kvh) << a.page_shift) + (kt & (a.page - 1))) * HD;
+      const size_t base = ((((size_t)kvh * a.n_pages + pg) << a.page_shift) + (kt & (a.page - 1))) * HD;
 #pragma unroll
       for (int i = 0; i < 16 * CPR / 32; ++i) {
         const int idx = i * 32 + lane, kk = idx / CPR, ch = idx % CPR;
@@ -539,7 +546,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
         } else {
           const int pos = pos0 + rr;
           __nv_bfloat16 *pool = kind == 1 ? lay.k_pool : lay.v_pool;
-          const size_t off = (((size_t)row_pg_sh[row0 + rr] * a.nkv + kvh) * a.page + (pos & (a.page - 1))) * HD + c8 * 8;
+          const size_t off = (((size_t)kvh * a.n_pages + row_pg_sh[row0 + rr]) * a.page + (pos & (a.page - 1))) * HD + c8 * 8;
           *reinterpret_cast<uint4 *>(pool + off) = vl;
           *reinterpret_cast<uint4 *>(pool + off + HALF) = vh;
           const int st = (pos - key_lo) >> 4, kk = (pos - key_lo) & 15;
@@ -570,8 +577,10 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
     for (int j = 0; j < n_mine; ++j) {
       const int kt = key_lo + (first + j * step) * 16;
       if (j + 1 < n_mine && j + 1 - pg_base >= 32) load_pages(j + 1);
+      lap(14);
       asm volatile("cp.async.wait_group 1;" ::: "memory");       // K of this sub-tile landed; V may be in flight
       __syncwarp();
+      lap(10);
       // ---- S = Q K^T for 16 query vectors x 16 keys
       float sacc[2][4];
 #pragma unroll
@@ -594,6 +603,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
         }
       }
       __syncwarp();                                              // every lane is done with the K buffer
+      lap(11);
       if (j + 1 < n_mine) issue(kpool, shK, j + 1, false, kAllKeys);
       else asm volatile("cp.async.commit_group;" ::: "memory");  // keep the group count uniform
       // ---- online softmax on the accumulator rows (g and g + 8); P re-packed as the A operand of P V
@@ -635,8 +645,10 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
           pl[n * 2 + h] = *reinterpret_cast<const unsigned *>(&lo);
         }
       }
+      lap(12);
       asm volatile("cp.async.wait_group 1;" ::: "memory");       // V of this sub-tile landed; the next K may be in flight
       __syncwarp();
+      lap(13);
       // ---- O = O * corr + P V (the rescale is skipped while no row of the warp has a new maximum)
       if (__any_sync(0xFFFFFFFFu, corr_h[0] != 1.f || corr_h[1] != 1.f)) {
 #pragma unroll
@@ -815,7 +827,7 @@ __device__ __forceinline__ void final_store(const FwdArgs &a, const Gemm &g, con
           if (ti.seg == 0) {
             a.q[(size_t)r * g.seg_n[0] + n] = __float2bfloat16_rn(out);
           } else {
-            const size_t off = (((size_t)rpg[r] * a.nkv + head) * a.page + (rpos[r] & (a.page - 1))) * hd + dd;
+            const size_t off = (((size_t)head * a.n_pages + rpg[r]) * a.page + (rpos[r] & (a.page - 1))) * hd + dd;
             (ti.seg == 1 ? lay.k_pool : lay.v_pool)[off] = __float2bfloat16_rn(out);
           }
         }
@@ -1144,10 +1156,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   // tcgen05.commit costs the tensor pipe as much as three MMAs of this shape), and
   // tcgen05.fence::after_thread_sync (~0.1 us while MMAs are in flight) is issued only where another
   // thread's tcgen05 operations must come first (accumulator reuse), not after the wait on TMA data.
-#ifndef HSD_WGS
-#define HSD_WGS 1
-#endif
-  constexpr int WGS = (STAGES % HSD_WGS == 0) ? HSD_WGS : 1;       // landing slots handed back together
+  constexpr int WGS = 1;                                          // landing slots handed back together
   if (warp == 0) {
     // ------------------------------------------------------------ weight-tile producer (runs ahead)
     if (lane == 0) {
@@ -1270,7 +1279,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     w.wt = wt; w.lane = lane; w.q = q; w.G = G; w.c = c; w.seg_idx = 0;
 
     // ---- phase program
-    if (a.prof && wt == 0) a.prof[(size_t)blockIdx.x * kFwdProfEvents] = globaltimer_ns();
+    if (HSD_PROF(a) && wt == 0) a.prof[(size_t)blockIdx.x * kFwdProfEvents] = globaltimer_ns();
     for (int l = wt; l < a.n_run; l += 256) layers_sh[l] = a.layers[l];
     if (a.R <= kRopeCacheRows)
       for (int i = wt; i < a.R * (HD / 2); i += 256) {
@@ -1378,7 +1387,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       if (barrier && alive) alive = grid_barrier(a, epoch, abort_flag, wt, ready >= 0 ? ready_bar(ready & 1) : 0u);
     }
   }
-  if (a.prof && blockIdx.x == 0 && threadIdx.x == 128) for (int i = 0; i < 16; ++i) a.prof[940 + i] = (unsigned long long)dbg_cy[i];
+  if (HSD_PROF(a) && blockIdx.x == 0 && threadIdx.x == 128) for (int i = 0; i < 16; ++i) a.prof[940 + i] = (unsigned long long)dbg_cy[i];
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();

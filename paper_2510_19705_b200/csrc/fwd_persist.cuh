@@ -15,7 +15,7 @@ struct FwdLayerDev {
 
 struct FwdArgs {
   // geometry
-  int d, nq, nkv, hd, ff, V, n_run, lm_map, max_seq, page, page_shift, pages_per_seq;   // page = 1 << page_shift
+  int d, nq, nkv, hd, ff, V, n_run, lm_map, max_seq, page, page_shift, pages_per_seq, n_pages;   // page = 1 << page_shift; KV pools are [kv head][n_pages][page][hd]
   float eps;
   // immutable inputs
   const CUtensorMap *wmaps;        // global memory: 7 per layer (wq wk wv wo wg wu wd), then the output head

@@ -40,7 +40,7 @@ WORKLOADS = {
     # 16-token pages, head size 128, and prompts long enough that every attention key split spans
     # several key tiles and many pages.
     "mini4long": dict(model=model_cfg(6, 256, 4, 1, 704, 2048, "bf16", head_dim=128), exits=(1, 2, 4, 6),
-                      T=(2, 2, 3), batch=2, prompt=1900, n_new=24, page=16, weight_seed=9, prompt_seed=9),
+                      T=(2, 2, 3), batch=2, prompt=2100, n_new=24, page=16, weight_seed=9, prompt_seed=9),
 }
 
 

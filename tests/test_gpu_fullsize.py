@@ -231,7 +231,7 @@ def test_bf16_batch_decisions_and_logits(lib, tmp_path, B):
 
 def test_long_context_four_levels_paged_batch(lib, tmp_path):
     """The long-context configuration's structure at a size the oracle can follow: 4 levels with draft lengths
-    (2, 2, 3), two sequences, 16-token pages, 1900-token prompts (every attention key split spans more than one
+    (2, 2, 3), two sequences, 16-token pages, 2100-token prompts (the long-context attention path: every key split spans more than one
     key tile and several pages).  Every decision follows the oracle on the logged logits; each sequence's first
     verification at the top level and at level 1 matches the oracle's forward."""
     wl = inputs.WORKLOADS["mini4long"]
