@@ -306,7 +306,7 @@ int hsd_pairwise_alpha(const void *logits, int dtype, int n_models, int n_rows, 
  * One weight-streaming matrix product of the verifier forward in isolation (the contraction
  * behind every projection of Algorithm 2's multi-row forward pass): out[r, n] = sum_k A[r, k] W[n, k],
  * bf16 inputs, fp32 accumulation on the tensor cores, fp32 output.
- *   A    device bf16 [R, K] row-major, 1 <= R <= 128, K a multiple of 64
+ *   A    device bf16 [R, K] row-major, 1 <= R <= 256, K a multiple of 64
  *   W    device bf16 [N, K] row-major
  *   out  device fp32 [R, N]
  *   workspace  device, 256-byte aligned, >= hsd_gemm_workspace_bytes(R, N, K); ignored on entry

@@ -21,7 +21,7 @@ constexpr int kRingSlots = 48;
 constexpr int kTimerPairs = 64;
 constexpr int kAttnBlocksTarget = 512;
 constexpr int kMaxSplits = 64;
-constexpr int kPrefillRows = 128;
+constexpr int kPrefillRows = 128;              // rows of one prompt chunk: the largest pass the one-launch forward takes
 constexpr uint32_t kTraceMagic = 0x48534454u;
 
 constexpr size_t kTcCtrlBytes = 16384 + 256;    // status word (first 256 bytes) + per-tile counters
@@ -149,7 +149,7 @@ Layout make_layout(const hsd_model_desc *models, int n_models, int n_levels, con
     M.tc_pieces_bytes = 0;
     if (m->dtype == HSD_BF16) {
       const int sms = device_sm_count();
-      const int npads[4] = {16, 32, 64, 128};
+      const int npads[5] = {16, 32, 64, 128, 256};
       const int shapes[5][4] = {{nq * hd, nkv * hd, nkv * hd, d}, {d, 0, 0, nq * hd}, {m->d_ff, m->d_ff, 0, d},
                                 {d, 0, 0, m->d_ff}, {m->vocab, 0, 0, d}};
       const int modes[5] = {GEMM_STORE_F32, GEMM_ADD_F32, GEMM_SWIGLU_T, GEMM_ADD_F32, GEMM_STORE_T_SCATTER};
@@ -191,7 +191,7 @@ struct Model {
   std::vector<const void *> lw;
   bool use_tc = false, use_persist = false;   // tensor-core GEMMs / the one-launch persistent forward (bf16 models)
   std::vector<CUtensorMap> wmaps;             // [n_layers * 7 + kHeadMaps]: wq wk wv wo wg wu wd per layer, then the levels' heads, the shared head
-  CUtensorMap amaps[4][4];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128}
+  CUtensorMap amaps[4][5];                    // activation buffers {h, att, act, hf} x row padding {16, 32, 64, 128, 256}
   CUtensorMap amaps_rows[4][16];              // the same buffers with a box of exactly 1..16 rows (persistent forward, few rows)
 };
 
@@ -330,11 +330,11 @@ int gemm(hsd_ctx *c, Model &M, int abuf, const void *A, int R, int K, const Gemm
   a.status = (int *)(c->ws + c->status_off);
   a.counters = (int *)(c->ws + M.lay.tc_scratch + 256);
   a.pieces = (float *)(c->ws + M.lay.tc_scratch + kTcCtrlBytes);
-  for (int r0 = 0; r0 < R; r0 += 128) {
-    a.R = std::min(128, R - r0);
+  for (int r0 = 0; r0 < R; r0 += 256) {
+    a.R = std::min(256, R - r0);
     a.row0 = r0;
     int np = tc_npad(a.R);
-    a.a = M.amaps[abuf][np == 16 ? 0 : np == 32 ? 1 : np == 64 ? 2 : 3];
+    a.a = M.amaps[abuf][np == 16 ? 0 : np == 32 ? 1 : np == 64 ? 2 : np == 128 ? 3 : 4];
     int st = launch_gemm_tc(a, c->sm_count, c->stream);
     if (st) return st;
   }
@@ -457,6 +457,9 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     }
     n_splits = best_s;
   }
+  // passes with more rows than the one-launch forward takes (prompt chunks): every attention item keeps one key split
+  const bool big_pass = M.use_persist && !(R <= 128 && n_logit <= 128);
+  if (big_pass) n_splits = 1;
   int keys_per_split = (int)align_up((size_t)(max_kv + n_splits - 1) / n_splits, M.use_persist ? 16 : kAttnKeyTile);
   n_splits = (max_kv + keys_per_split - 1) / keys_per_split;
   if ((size_t)R * n_splits > (size_t)ML.partial_rows) return HSD_E_INVALID_ARG;
@@ -561,7 +564,18 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     GemmSegs qkv_segs = {{w[1], w[2], w[3]}, {md.nq * md.hd, md.nkv * md.hd, md.nkv * md.hd}, 3};
     HSD_TRY(gemm(c, M, 0, h, R, md.d, qkv_segs, l * 7 + 0, GEMM_STORE_F32, qkv, nullptr, nullptr));
     HSD_TRY(launch_rope_kv(md, qkv, rb, c->dev<float>(ML.cos_tab), c->dev<float>(ML.sin_tab), pt, kp, vp, q, s));
-    HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(ML.partials), keys_per_split, n_splits, att, s));
+    if (big_pass) {                                       // tensor-core attention of the persistent forward, as a launch of its own
+      FwdArgs fa = {};
+      fa.d = md.d; fa.nq = md.nq; fa.nkv = md.nkv; fa.hd = md.hd; fa.ff = md.ff; fa.V = md.V; fa.max_seq = md.max_seq; fa.page = md.page;
+      while ((1 << fa.page_shift) < md.page) ++fa.page_shift;
+      fa.pages_per_seq = md.pages_per_seq; fa.n_pages = md.n_pages;
+      fa.R = R; fa.n_attn = n_attn; fa.attn_rows = arows; fa.n_splits = 1; fa.keys_per_split = keys_per_split;
+      fa.page_table = pt; fa.attn_items = rb.attn; fa.row_seq = rb.row_seq; fa.row_pos = rb.row_pos;
+      fa.q = (__nv_bfloat16 *)q; fa.att = (__nv_bfloat16 *)att; fa.attn_partials = c->dev<float>(ML.partials);
+      HSD_TRY(launch_attention_tiles(fa, (__nv_bfloat16 *)kp, (__nv_bfloat16 *)vp, c->sm_count, s));
+    } else {
+      HSD_TRY(launch_attention(md, q, rb, pt, kp, vp, c->dev<float>(ML.partials), keys_per_split, n_splits, att, s));
+    }
     GemmSegs o_segs = {{w[4], nullptr, nullptr}, {md.d, 0, 0}, 1};
     HSD_TRY(gemm(c, M, 1, att, R, md.nq * md.hd, o_segs, l * 7 + 3, GEMM_ADD_F32, x, nullptr, nullptr));
     HSD_TRY(launch_rmsnorm(md, x, w[5], nullptr, R, h, s));
@@ -808,9 +822,9 @@ int init_model(hsd_ctx *c, Model &M, const hsd_model_desc *model, const ModelLay
   const size_t abuf_off[4] = {ml.h, ml.att, ml.act, ml.hf};
   const long long acols[4] = {md.d, (long long)md.nq * md.hd, md.ff, md.d};
   const long long arows[4] = {lay.max_rows, lay.max_rows, lay.max_rows, lay.max_logit_rows};
-  const int npads[4] = {16, 32, 64, 128};
+  const int npads[5] = {16, 32, 64, 128, 256};
   for (int b = 0; b < 4 && !st; ++b)
-    for (int p = 0; p < 4 && !st; ++p) st = tc_make_map(&M.amaps[b][p], c->ws + abuf_off[b], arows[b], acols[b], npads[p]);
+    for (int p = 0; p < 5 && !st; ++p) st = tc_make_map(&M.amaps[b][p], c->ws + abuf_off[b], arows[b], acols[b], npads[p]);
   for (int b = 0; b < 4 && !st; ++b)
     for (int r = 1; r <= 16 && !st; ++r) st = tc_make_map(&M.amaps_rows[b][r - 1], c->ws + abuf_off[b], arows[b], acols[b], r);
   if (!st && cudaMemset(c->ws + ml.tc_scratch, 0, kTcCtrlBytes) != cudaSuccess) st = HSD_E_CUDA;
@@ -1128,7 +1142,7 @@ int hsd_set_trace(hsd_ctx *c, const char *path, int logit_calls) {
 }
 
 size_t hsd_gemm_workspace_bytes(int R, int N, int K) {
-  if (R < 1 || R > 128 || N < 1 || K < kTcBlockK || K % kTcBlockK) return 0;
+  if (R < 1 || R > 256 || N < 1 || K < kTcBlockK || K % kTcBlockK) return 0;
   int seg[3] = {N, 0, 0};
   return kTcCtrlBytes + tc_plan(seg, 1, GEMM_STORE_F32, K, tc_npad(R), device_sm_count()).scratch_bytes;
 }

@@ -1396,6 +1396,45 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, 1);
 }
 
+// The attention tiles phase as a launch of its own (prompt passes with more rows than the persistent forward takes):
+// one key split per item, so every work item writes its rows of the attention output itself.  256 threads = the
+// phase's eight worker warps; q / k / v of the pass are in place (separate finish kernels).
+template <int HD>
+__global__ void __launch_bounds__(256, 2) attn_tiles_kernel(const __grid_constant__ FwdArgs a, __nv_bfloat16 *k_pool, __nv_bfloat16 *v_pool) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t *scratch = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  __shared__ PageCache pcache;
+  __shared__ int first_item_sh[4];
+  __shared__ int qkv_geom_sh[8];
+  __shared__ long long dbg_cy[16];
+  if (threadIdx.x == 0) {
+    pcache.tag_item = -1;
+    pcache.tag_tile = -1;
+    const int n_work = a.n_attn * a.nkv * a.n_splits;
+    int4 fi = make_int4(0, 0, 0, 0);
+    if ((int)blockIdx.x < n_work) fi = a.attn_items[blockIdx.x / (a.n_splits * a.nkv)];
+    first_item_sh[0] = fi.x; first_item_sh[1] = fi.y; first_item_sh[2] = fi.z; first_item_sh[3] = fi.w;
+  }
+  __syncthreads();
+  FwdLayerDev lay;
+  lay.attn_norm = nullptr; lay.mlp_norm = nullptr; lay.k_pool = k_pool; lay.v_pool = v_pool;
+  attn_tiles_phase<128, HD>(a, lay, scratch, &pcache, (int)threadIdx.x, dbg_cy, first_item_sh, qkv_geom_sh, nullptr, nullptr, nullptr);
+}
+
+template <int HD>
+int launch_attn_tiles_t(const FwdArgs &a, __nv_bfloat16 *k_pool, __nv_bfloat16 *v_pool, int sm_count, cudaStream_t s) {
+  static bool attr_set = false;
+  const int smem = kScratchBytes + 1024;
+  if (!attr_set) {
+    HSD_CUDA_OK(cudaFuncSetAttribute(attn_tiles_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_set = true;
+  }
+  const int n_work = a.n_attn * a.nkv * a.n_splits;
+  attn_tiles_kernel<HD><<<std::min(n_work, 2 * sm_count), 256, smem, s>>>(a, k_pool, v_pool);
+  hsd_count_launches(1);
+  return hsd_launch_status();
+}
+
 template <int NPAD, int HD>
 int launch_t(const FwdArgs &args, int sm_count, cudaStream_t s) {
   using Cfg = PCfg<NPAD>;
@@ -1423,6 +1462,16 @@ int launch_hd(const FwdArgs &args, int npad, int sm_count, cudaStream_t s) {
 }
 
 }  // namespace
+
+int launch_attention_tiles(const FwdArgs &args, __nv_bfloat16 *k_pool, __nv_bfloat16 *v_pool, int sm_count, cudaStream_t s) {
+  if (args.fuse_qkv || args.n_splits != 1 || args.n_attn < 1) return HSD_E_INVALID_ARG;
+  switch (args.hd) {
+    case 128: return launch_attn_tiles_t<128>(args, k_pool, v_pool, sm_count, s);
+    case 64: return launch_attn_tiles_t<64>(args, k_pool, v_pool, sm_count, s);
+    case 32: return launch_attn_tiles_t<32>(args, k_pool, v_pool, sm_count, s);
+    default: return HSD_E_UNSUPPORTED;
+  }
+}
 
 bool fwd_persist_supported(int hd, int group) {
   return (hd == 32 || hd == 64 || hd == 128) && group >= 1 && group <= 8 && fwd_attn_rows(group, hd) * group <= 32;

@@ -58,5 +58,8 @@ inline int fwd_attn_rows(int group, int hd) {
 }
 bool fwd_persist_supported(int hd, int group);
 int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaStream_t s);
+// The attention tiles phase alone, one key split per item (args: geometry, R, n_attn, attn_rows, n_splits = 1,
+// keys_per_split, page table, attn_items, q, att; fuse_qkv = 0): the item's rows of `att` are written.
+int launch_attention_tiles(const FwdArgs &args, __nv_bfloat16 *k_pool, __nv_bfloat16 *v_pool, int sm_count, cudaStream_t s);
 
 }  // namespace hsd

@@ -21,7 +21,8 @@ constexpr int kSmemBudget = 232448 - 1024;                    // 227 KiB minus a
 
 template <int NPAD> struct TcCfg {
   static constexpr int kStageBytes = kStageWBytes + NPAD * kTcBlockK * 2;
-  static constexpr int kStagingBytes = kTcBlockM * (NPAD + 1) * 4;
+  static constexpr int kChunk = NPAD < 32 ? NPAD : 32;        // accumulator columns (token rows) the epilogue handles at a time
+  static constexpr int kStagingBytes = kTcBlockM * (kChunk + 1) * 4;
   static constexpr int kCtrlBytes = 1024;
   static constexpr int kStages = (kSmemBudget - kCtrlBytes - kStagingBytes) / kStageBytes;
   static constexpr int kSmemBytes = kStages * kStageBytes + kStagingBytes + kCtrlBytes + 1024;
@@ -178,25 +179,80 @@ gemm_tc_kernel(const __grid_constant__ TcGemmArgs args, int n_tiles, int KB, int
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (!wait_ok[seg_idx & 1]) { ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      float v[NPAD];
-#pragma unroll
-      for (int j = 0; j < NPAD / 16; ++j)
-        tmem_ld16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * NPAD + j * 16), v + j * 16);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(acce_bar(ab));
+      constexpr int CH = Cfg::kChunk;
       const TileInfo ti = tile_info(args, tile);
       const bool whole = (kb0 == 0 && kb1 == KB);
-      bool finish = whole;
+      const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * NPAD);
+      int n_pieces = 1, piece = 0;
       if (!whole) {
-        // split tile: publish this piece; the last arriver sums all pieces in piece order
         const int first_owner = unit_owner(U, G, (long long)tile * KB);
         const int last_owner = unit_owner(U, G, (long long)tile * KB + KB - 1);
-        const int n_pieces = last_owner - first_owner + 1, piece = c - first_owner;
-        float *mine = args.pieces + ((size_t)tile * pieces_max + piece) * NPAD * kTcBlockM;
+        n_pieces = last_owner - first_owner + 1;
+        piece = c - first_owner;
+      }
+      // values of the tile's row m for token rows c0 .. c0 + CH - 1 -> the projection's output
+      auto finish_chunk = [&](int c0, float *v) {
+        if (MODE == GEMM_SWIGLU_T) {
 #pragma unroll
-        for (int r = 0; r < NPAD; ++r) mine[r * kTcBlockM + m] = v[r];
+          for (int r = 0; r < CH; ++r) staging[m * (CH + 1) + r] = v[r];
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          for (int i = et; i < kTcBoxRows * CH; i += 128) {
+            const int cc = i % kTcBoxRows, r = c0 + i / kTcBoxRows;
+            const int col = ti.row0 + cc;
+            if (r < args.R && col < args.seg_n[0]) {
+              const float g = staging[cc * (CH + 1) + (r - c0)], up = staging[(cc + kTcBoxRows) * (CH + 1) + (r - c0)];
+              args.out_bf16[(size_t)(args.row0 + r) * args.ldo + col] = __float2bfloat16_rn(ptx::silu_mul(g, up));
+            }
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        } else {
+          const int n = ti.row0 + m;
+          if (n < args.seg_n[ti.seg]) {
+            const int col = ti.col0 + n;
+            if (MODE == GEMM_ADD_F32) {
+              // residual add: all of the chunk's old values are fetched before the first store (a read-modify-write
+              // per row would be one dependent round trip per row)
+              float old[CH];
+#pragma unroll
+              for (int i = 0; i < CH; ++i)
+                old[i] = c0 + i < args.R ? __ldcg(args.out_f32 + (size_t)(args.row0 + c0 + i) * args.ldo + col) : 0.f;
+#pragma unroll
+              for (int i = 0; i < CH; ++i)
+                if (c0 + i < args.R) args.out_f32[(size_t)(args.row0 + c0 + i) * args.ldo + col] = old[i] + v[i];
+            } else {
+#pragma unroll
+              for (int i = 0; i < CH; ++i) {
+                const int r = c0 + i;
+                if (r < args.R) {
+                  if (MODE == GEMM_STORE_F32) args.out_f32[(size_t)(args.row0 + r) * args.ldo + col] = v[i];
+                  else args.out_bf16[(size_t)args.dst[args.row0 + r] * args.ldo + col] = __float2bfloat16_rn(v[i]);
+                }
+              }
+            }
+          }
+        }
+      };
+      float *mine = args.pieces + ((size_t)tile * pieces_max + piece) * NPAD * kTcBlockM;
+#pragma unroll 1
+      for (int c0 = 0; c0 < NPAD; c0 += CH) {
+        float v[CH];
+#pragma unroll
+        for (int j = 0; j < CH / 16; ++j) tmem_ld16(tbase + (uint32_t)(c0 + j * 16), v + j * 16);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (c0 + CH >= NPAD) {                     // accumulator fully read: hand it back to the MMA warp
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acce_bar(ab));
+        }
+        if (c0 >= args.R) continue;                // padding rows: nothing to write
+        if (whole) finish_chunk(c0, v);
+        else {
+#pragma unroll
+          for (int i = 0; i < CH; ++i) mine[(c0 + i) * kTcBlockM + m] = v[i];
+        }
+      }
+      if (!whole) {
+        // split tile: this piece is published; the last arriver sums all pieces in piece order
         __threadfence();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (et == 0) {
@@ -207,44 +263,20 @@ gemm_tc_kernel(const __grid_constant__ TcGemmArgs args, int n_tiles, int KB, int
           __threadfence();
         }
         asm volatile("bar.sync 1, 128;" ::: "memory");
-        finish = (*last_flag != 0);
-        if (finish) {
-#pragma unroll
-          for (int r = 0; r < NPAD; ++r) v[r] = 0.f;
-          for (int p = 0; p < n_pieces; ++p) {
-            const float *src = args.pieces + ((size_t)tile * pieces_max + p) * NPAD * kTcBlockM;
-#pragma unroll
-            for (int r = 0; r < NPAD; ++r) v[r] += __ldcg(src + r * kTcBlockM + m);
-          }
-        }
+        const bool finish = (*last_flag != 0);
         asm volatile("bar.sync 1, 128;" ::: "memory");   // last_flag may be rewritten by the next tile
-      }
-      if (finish) {
-        if (MODE == GEMM_SWIGLU_T) {
+        if (finish) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < NPAD && c0 < args.R; c0 += CH) {
+            float v[CH];
 #pragma unroll
-          for (int r = 0; r < NPAD; ++r) staging[m * (NPAD + 1) + r] = v[r];
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          for (int i = et; i < kTcBoxRows * args.R; i += 128) {
-            int cc = i % kTcBoxRows, r = i / kTcBoxRows;
-            int col = ti.row0 + cc;
-            if (col < args.seg_n[0]) {
-              float g = staging[cc * (NPAD + 1) + r], up = staging[(cc + kTcBoxRows) * (NPAD + 1) + r];
-              args.out_bf16[(size_t)(args.row0 + r) * args.ldo + col] = __float2bfloat16_rn(ptx::silu_mul(g, up));
-            }
-          }
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-        } else {
-          const int n = ti.row0 + m;
-          if (n < args.seg_n[ti.seg]) {
-            const int col = ti.col0 + n;
+            for (int i = 0; i < CH; ++i) v[i] = 0.f;
+            for (int p = 0; p < n_pieces; ++p) {
+              const float *src = args.pieces + ((size_t)tile * pieces_max + p) * NPAD * kTcBlockM;
 #pragma unroll
-            for (int r = 0; r < NPAD; ++r) {
-              if (r < args.R) {
-                if (MODE == GEMM_STORE_F32) args.out_f32[(size_t)(args.row0 + r) * args.ldo + col] = v[r];
-                else if (MODE == GEMM_ADD_F32) args.out_f32[(size_t)(args.row0 + r) * args.ldo + col] += v[r];
-                else args.out_bf16[(size_t)args.dst[args.row0 + r] * args.ldo + col] = __float2bfloat16_rn(v[r]);
-              }
+              for (int i = 0; i < CH; ++i) v[i] += __ldcg(src + (c0 + i) * kTcBlockM + m);
             }
+            finish_chunk(c0, v);
           }
         }
       }
@@ -316,7 +348,7 @@ int tc_make_map(CUtensorMap *map, const void *base, long long rows, long long co
   return r == CUDA_SUCCESS ? HSD_OK : HSD_E_CUDA;
 }
 
-int tc_npad(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : 128; }
+int tc_npad(int rows) { return rows <= 16 ? 16 : rows <= 32 ? 32 : rows <= 64 ? 64 : rows <= 128 ? 128 : 256; }
 
 TcGemmPlan tc_plan(const int *seg_n, int n_segs, int mode, int K, int npad, int sm_count) {
   TcGemmPlan p;
@@ -334,14 +366,15 @@ TcGemmPlan tc_plan(const int *seg_n, int n_segs, int mode, int K, int npad, int 
 }
 
 int launch_gemm_tc(const TcGemmArgs &args, int sm_count, cudaStream_t s) {
-  if (args.R < 1 || args.R > 128 || args.K % kTcBlockK != 0) return HSD_E_UNSUPPORTED;
+  if (args.R < 1 || args.R > 256 || args.K % kTcBlockK != 0) return HSD_E_UNSUPPORTED;
   const int npad = tc_npad(args.R);
   TcGemmPlan plan = tc_plan(args.seg_n, args.n_segs, args.mode, args.K, npad, sm_count);
   switch (npad) {
     case 16: return launch_mode<16>(args, plan, s);
     case 32: return launch_mode<32>(args, plan, s);
     case 64: return launch_mode<64>(args, plan, s);
-    default: return launch_mode<128>(args, plan, s);
+    case 128: return launch_mode<128>(args, plan, s);
+    default: return launch_mode<256>(args, plan, s);
   }
 }
 

@@ -199,11 +199,12 @@ def test_model_shapes_decisions_and_sampled_logits(lib, tmp_path, name, n_new, o
     assert len(seen) == oracle_calls
 
 
-@pytest.mark.parametrize("B", [2, 8])
+@pytest.mark.parametrize("B", [2, 8, 48])
 def test_bf16_batch_decisions_and_logits(lib, tmp_path, B):
-    # several sequences in one bf16 batch (8: passes of 17-32 rows, the 32-row padding of the GEMMs): every
-    # decision follows the oracle on the logged logits, and each sequence's first verification logits match the
-    # oracle's forward of that sequence
+    # several sequences in one bf16 batch (8: passes of 17-32 rows, the 32-row padding of the GEMMs; 48: passes of
+    # more than 128 rows, which run one kernel per operation: 256-row tensor-core GEMMs and the attention tiles phase
+    # as a launch of its own): every decision follows the oracle on the logged logits, and each sequence's first
+    # verification logits match the oracle's forward of that sequence
     wl = inputs.WORKLOADS["mini3"]
     cfg = wl["model"]
     w_cpu = inputs.make_weights(cfg, wl["weight_seed"])

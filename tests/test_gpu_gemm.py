@@ -5,9 +5,10 @@ import torch
 
 pytestmark = pytest.mark.gpu
 
-SHAPES = [  # (R, N, K): one tile / ragged N / several row paddings / deep split-K / full projection sizes
+SHAPES = [  # (R, N, K): one tile / ragged N / several row paddings / deep split-K / full projection sizes / prompt chunks
     (1, 128, 64), (3, 200, 128), (5, 300, 256), (16, 1024, 512), (17, 520, 320), (40, 257, 192), (100, 1000, 512),
     (128, 384, 1024), (8, 4096, 14336), (6, 6144, 4096), (2, 32000, 4096),
+    (129, 384, 512), (200, 1000, 1024), (256, 6144, 4096), (255, 4096, 14336),      # prompt-chunk row counts (256-row padding)
 ]
 
 
