@@ -11,9 +11,10 @@ template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(flo
 // ------------------------------------------------------------------------------ embedding gather
 template <typename T>
 __global__ void embed_kernel(const T *__restrict__ embed, const int *__restrict__ tokens, const int *__restrict__ row_seq,
-                             const int *__restrict__ row_pos, int d, int max_seq, float *__restrict__ x) {
+                             const int *__restrict__ row_pos, int d, int max_seq, int V, float *__restrict__ x) {
   int r = blockIdx.x;
-  int tok = tokens[(size_t)row_seq[r] * max_seq + row_pos[r]];
+  // an id outside the vocabulary (only possible after non-finite logits) must not become an address
+  int tok = min(max(tokens[(size_t)row_seq[r] * max_seq + row_pos[r]], 0), V - 1);
   const T *src = embed + (size_t)tok * d;
   for (int k = threadIdx.x; k < d; k += blockDim.x) x[(size_t)r * d + k] = to_f32(src[k]);
 }
@@ -375,9 +376,9 @@ static int attention_t(const ModelDims &md, const void *q, const RowBatch &rb, c
 int launch_embed(const ModelDims &md, const void *embed, const int *tokens, const RowBatch &rb, float *x, cudaStream_t s) {
   if (rb.R == 0) return HSD_OK;
   if (md.dtype == HSD_BF16)
-    embed_kernel<__nv_bfloat16><<<rb.R, 256, 0, s>>>((const __nv_bfloat16 *)embed, tokens, rb.row_seq, rb.row_pos, md.d, md.max_seq, x);
+    embed_kernel<__nv_bfloat16><<<rb.R, 256, 0, s>>>((const __nv_bfloat16 *)embed, tokens, rb.row_seq, rb.row_pos, md.d, md.max_seq, md.V, x);
   else
-    embed_kernel<float><<<rb.R, 256, 0, s>>>((const float *)embed, tokens, rb.row_seq, rb.row_pos, md.d, md.max_seq, x);
+    embed_kernel<float><<<rb.R, 256, 0, s>>>((const float *)embed, tokens, rb.row_seq, rb.row_pos, md.d, md.max_seq, md.V, x);
   hsd_count_launches(1);
   return hsd_launch_status();
 }

@@ -264,7 +264,9 @@ __device__ __forceinline__ bool norm_phase(const FwdArgs &a, int n_rows, const i
     float *xrow = a.x + (size_t)row * d;
     float4 v[MAXV];
     if (src_embed) {
-      const __nv_bfloat16 *erow = a.embed + (size_t)a.tokens[(size_t)a.row_seq[row] * a.max_seq + a.row_pos[row]] * d;
+      // an id outside the vocabulary (only possible after non-finite logits) must not become an address
+      const int tok = min(max(a.tokens[(size_t)a.row_seq[row] * a.max_seq + a.row_pos[row]], 0), a.V - 1);
+      const __nv_bfloat16 *erow = a.embed + (size_t)tok * d;
       uint2 raw[MAXV];
 #pragma unroll
       for (int j = 0; j < MAXV; ++j) {
