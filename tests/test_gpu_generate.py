@@ -117,6 +117,27 @@ def test_degenerate_hierarchies(lib):
     _check_stats(stats, run)
 
 
+def test_shortest_inputs_engine_reuse_and_rejected_calls(lib):
+    # a one-token prompt, a request that ends inside the first round (only its first token is returned), the same
+    # engine used again with fewer sequences and another seed; every stream equals the oracle's
+    wl, cfg, eng, om, prompts, T = _setup("tiny3", lib, max_batch=3)
+    for batch, P, n_new, seed in ((3, 1, 1, 4), (1, 1, 7, 5), (2, 3, 30, 6), (3, wl["prompt"], wl["n_new"], 7)):
+        pr = prompts[:batch, :P].contiguous()
+        toks, stats, _ = eng.generate(pr.cuda(), n_new, seed)
+        assert tuple(toks.shape) == (batch, n_new)
+        for b in range(batch):
+            want, _ = _oracle_run(om, T, pr[b].tolist(), n_new, seed, seq=b)
+            assert np.array_equal(toks[b].cpu().numpy(), want), (batch, P, n_new, b)
+    # calls that cannot run are refused with an error code before anything is launched
+    for batch, P, n_new in ((4, 4, 4), (1, wl["prompt"], 10 ** 6), (1, 0, 4), (1, 4, 0)):
+        pr = torch.zeros((batch, max(P, 1)), dtype=torch.int32).cuda()
+        with pytest.raises(lib.HsdError, match="invalid argument"):
+            eng.generate(pr[:, :P] if P else pr[:, :0], n_new, 1)
+    toks, _, _ = eng.generate(prompts[:1].cuda(), 5, 7)          # the engine is still usable afterwards
+    want, _ = _oracle_run(om, T, prompts[0].tolist(), 5, 7)
+    assert np.array_equal(toks[0].cpu().numpy(), want)
+
+
 def test_batch_sequences_equal_their_single_runs(lib):
     # sequences are independent: sequence b of a batch = the same prompt run alone with the same seed
     wl, cfg, eng, om, prompts, T = _setup("tiny3", lib, max_batch=3)
