@@ -155,6 +155,8 @@ def _declare_engine(lib):
     lib.hsd_create_models.argtypes = [c.POINTER(_ModelDesc), i32, c.POINTER(c.c_int32), vp, sz, c.POINTER(vp)]
     lib.hsd_set_phase_folding.restype = i32
     lib.hsd_set_phase_folding.argtypes = [vp, i32, i32, i32]
+    lib.hsd_set_tensor_attention.restype = i32
+    lib.hsd_set_tensor_attention.argtypes = [vp, i32]
     lib.hsd_generate.restype = i32
     lib.hsd_generate.argtypes = [vp, vp, i32, i32, i32, u64, vp, vp, c.POINTER(LevelStats), c.POINTER(c.c_double)]
     lib.hsd_set_trace.restype = i32
@@ -262,6 +264,11 @@ class Hsd:
         """hsd_set_phase_folding: keep (False) or fold (True) the two finish phases of decode passes; keep (False) or
         drop (True) the grid barrier between a residual projection and its norm."""
         _check(self._lib.hsd_set_phase_folding(self._ctx, int(bool(fold_qkv)), int(bool(fold_gate_up)), int(bool(early_norm))))
+
+    def set_tensor_attention(self, enabled=True):
+        """hsd_set_tensor_attention: long key ranges on the tensor-memory attention path (True) or on the warp-level
+        path like the short ones (False); "prefer": on, and key splits never shorter than that path takes."""
+        _check(self._lib.hsd_set_tensor_attention(self._ctx, 2 if enabled == "prefer" else int(bool(enabled))))
 
     def set_exit_heads(self, heads):
         """heads: list over levels of None (shared head) or dict(lm_head[, final_norm]) of CUDA tensors in the

@@ -21,6 +21,8 @@ constexpr int kRingSlots = 48;
 constexpr int kTimerPairs = 64;
 constexpr int kAttnBlocksTarget = 512;
 constexpr int kMaxSplits = 64;
+constexpr int kTcAttnMinKeys = 1024;           // = the kernel's thresholds for the tensor-memory attention path:
+constexpr int kTcAttnMinVectors = 13;          //   keys of a work item, query vectors of an attention item
 constexpr int kPrefillRows = 128;              // rows of one prompt chunk: the largest pass the one-launch forward takes
 constexpr uint32_t kTraceMagic = 0x48534454u;
 
@@ -230,6 +232,8 @@ struct hsd_ctx {
   bool no_fuse_qkv = false;                   // keep the QKV finish phase in every pass (hsd_set_phase_folding)
   bool no_fuse_gu = false;                    // keep the gate / up finish phase in every pass
   bool no_early_norm = false;                 // keep the grid barrier between a residual projection and its norm
+  bool no_tc_attn = false;                    // long key ranges on the mma.sync path as well (hsd_set_tensor_attention)
+  bool prefer_tc_attn = false;                // never cut the keys into splits shorter than that path takes (a test hook)
   int sm_count;
   std::vector<const void *> level_head, level_norm;   // output head and final norm gain of each level (the model's own unless set)
   std::vector<uint32_t> coin24;               // per level: kNoCoin, or the IID acceptance probability x 2^24 (ablation)
@@ -419,6 +423,7 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   const int blocks_target = M.use_persist ? c->sm_count : kAttnBlocksTarget;
   const int max_splits = M.use_persist ? 20 : kMaxSplits;      // the persistent merge phase takes <= 20 splits
   int n_splits = std::max(1, std::min(max_splits, blocks_target / std::max(1, n_attn * md.nkv)));
+  const bool tc_capable = M.use_persist && md.hd == 128 && !c->no_tc_attn && R <= 128 && n_logit <= 128;
   if (M.use_persist && max_kv >= 2048) {
     // Long contexts: the key loop dominates and the items differ in cost, so the split count is chosen by a
     // small model of the tiles phase: a work unit (item, KV head, split) costs a fixed part plus its keys x
@@ -435,8 +440,10 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
       double everywhere = 0;
       long long off = 0;
       for (int i = 0; i < n_attn; ++i) {
-        const int kv = attn[i].w + attn[i].y, mt = (attn[i].y * qgroup + 15) / 16;
-        const double unit = 5.0 + mt * ((std::min(kps, kv) + 127) / 128) * 1.9;
+        const int kv = attn[i].w + attn[i].y, mt = (attn[i].y * qgroup + 15) / 16, keys = std::min(kps, kv);
+        // key ranges of kTcAttnMinKeys and more run on tensor memory: 64-key tiles, whatever the number of query vectors
+        const bool tc_item = tc_capable && keys >= kTcAttnMinKeys && attn[i].y * qgroup >= kTcAttnMinVectors;
+        const double unit = tc_item ? 6.0 + ((keys + 63) / 64) * 0.8 : 5.0 + mt * ((keys + 127) / 128) * 1.9;
         // all s_try x nkv slots of the item are dealt out; splits past its last key return at once
         const long long used = (long long)std::min(s_try, (kv + kps - 1) / kps) * md.nkv, slots = (long long)s_try * md.nkv;
         everywhere += unit * (double)(used / G);
@@ -456,6 +463,7 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
       if (t < best) { best = t; best_s = s_try; }
     }
     n_splits = best_s;
+    if (tc_capable && c->prefer_tc_attn) n_splits = std::max(1, std::min(n_splits, max_kv / kTcAttnMinKeys));
   }
   // passes with more rows than the one-launch forward takes (prompt chunks): every attention item keeps one key split
   const bool big_pass = M.use_persist && !(R <= 128 && n_logit <= 128);
@@ -511,6 +519,11 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     a.fuse_gu = (R <= 4 && !c->no_fuse_gu) ? 1 : 0;
     // the norms after the residual projections start on otherwise idle CTAs as soon as the pieces are there
     a.early_norm = c->no_early_norm ? 0 : 1;
+    // long key ranges: attention work items on tcgen05 / tensor memory (they take their q / k / v from the finish phase)
+    int max_vectors = 0;
+    for (int i = 0; i < n_attn; ++i) max_vectors = std::max(max_vectors, attn[i].y * qgroup);
+    a.tc_attn = (tc_capable && keys_per_split >= kTcAttnMinKeys && max_vectors >= kTcAttnMinVectors) ? 1 : 0;
+    if (a.tc_attn) a.fuse_qkv = 0;
     a.pieces2 = (float *)(c->ws + ML.tc_pieces2);
     for (int b = 0; b < 4; ++b) a.amap[b] = box_rows <= 16 ? M.amaps_rows[b][box_rows - 1] : M.amaps[b][pi];
     a.prof = nullptr;
@@ -956,6 +969,13 @@ int hsd_set_phase_folding(hsd_ctx *c, int fold_qkv, int fold_gate_up, int early_
   c->no_fuse_qkv = fold_qkv == 0;
   c->no_fuse_gu = fold_gate_up == 0;
   c->no_early_norm = early_norm == 0;
+  return HSD_OK;
+}
+
+int hsd_set_tensor_attention(hsd_ctx *c, int enabled) {
+  if (!c) return HSD_E_INVALID_ARG;
+  c->no_tc_attn = enabled == 0;
+  c->prefer_tc_attn = enabled == 2;
   return HSD_OK;
 }
 

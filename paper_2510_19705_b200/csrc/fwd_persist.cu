@@ -372,6 +372,329 @@ __device__ __forceinline__ void ldmatrix_x4_trans(unsigned *r, const void *row_p
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_u32(row_ptr)));
 }
 
+// ------------------------------------------------------------------------------ long key ranges on tcgen05
+// One work item (attention item, KV head, key split) with a long key range, head size 128, at most 32 query
+// vectors.  Keys go through in tiles of 64, dealt to two independent streams (tile j to stream j & 1), each with
+// its own running reference maximum, row sums and output accumulator; per tile
+//   S[128 x 64]   = Q[128 (<= 32 real rows) x 128] K_tile[64 x 128]^T       tcgen05.mma, both operands K-major
+//   P             = exp2((S - m_ref) scale log2 e)  as bf16, row per thread  (m_ref moves only when a row maximum
+//                                                                             passes it by a factor 256: then O is rescaled)
+//   O[128 x 128] += P[128 x 64] V_tile[64 keys x 128]                        V as the MN-major B operand, as it lies in the cache
+// S and O live in tensor memory (S double-buffered per stream: 2 x 2 x 64 columns, O 2 x 128: all 512 columns,
+// the GEMM accumulators are idle during this phase).  Rows 32..127 of the A operands are whatever shared memory
+// follows the real rows: their results are never read.  The eight worker warps: per stream (warps 0-3 / 4-7) warp
+// 0 = softmax (the only one whose TMEM lane quarter holds real rows), warp 1 = K tiles (three buffers: a K buffer
+// is free as soon as S is complete), warp 2 = V tiles (two buffers), warp 3 = MMA issue (one lane).  Shared memory:
+// the weight ring and the attention scratch together (the weight producer does not run ahead over this phase).
+constexpr int kTcaTile = 64, kTcaKBufs = 3, kTcaVBufs = 2;
+constexpr int kTcaTileBytes = 2 * kTcaTile * 128;                 // two 64-column blocks of [64 keys][128 B]
+constexpr int kTcaOffK = 8192, kTcaOffV = kTcaOffK + 2 * kTcaKBufs * kTcaTileBytes, kTcaOffP = kTcaOffV + 2 * kTcaVBufs * kTcaTileBytes;
+constexpr int kTcaOffBar = kTcaOffP + 4 * 4096 + 12288, kTcaBytes = kTcaOffBar + 256;
+constexpr int kTcaMinKeys = 1024;                                 // shorter key ranges stay on the mma.sync path
+constexpr int kTcaMinVectors = 13;                                // ... and items with fewer query vectors (its cost grows with them, this path's does not)
+static_assert(kTcaBytes <= 4 * (kWBytes + 128 * kTcBlockK * 2) + kScratchBytes - 2 * 12 * 64 * 4, "tcgen05 attention buffers exceed the ring + scratch");
+
+__device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lbo_bytes) {   // MN-major, 128-byte swizzle
+  uint64_t d = (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)(lbo_bytes >> 4) << 16;                          // between the 64-element blocks along N
+  d |= (uint64_t)(1024 >> 4) << 32;                               // between the 8-row groups along K
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const float *o) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+               ::"r"(taddr), "r"(__float_as_uint(o[0])), "r"(__float_as_uint(o[1])), "r"(__float_as_uint(o[2])),
+               "r"(__float_as_uint(o[3])), "r"(__float_as_uint(o[4])), "r"(__float_as_uint(o[5])), "r"(__float_as_uint(o[6])),
+               "r"(__float_as_uint(o[7])), "r"(__float_as_uint(o[8])), "r"(__float_as_uint(o[9])), "r"(__float_as_uint(o[10])),
+               "r"(__float_as_uint(o[11])), "r"(__float_as_uint(o[12])), "r"(__float_as_uint(o[13])), "r"(__float_as_uint(o[14])),
+               "r"(__float_as_uint(o[15])) : "memory");
+}
+
+struct TcaItem { int row0, nrows, seq, pos0, kvh, split, key_lo, key_hi, nqv, group; };
+
+__device__ __noinline__ void attn_item_tc(const FwdArgs &a, const __nv_bfloat16 *kpool, const __nv_bfloat16 *vpool, uint8_t *smem,
+                                          uint32_t tmem, const TcaItem it, int wt, volatile int *abort_flag) {
+  constexpr int HD = 128, TK = kTcaTile, NKB = kTcaKBufs, NVB = kTcaVBufs;
+  const uint32_t s0 = smem_u32(smem), b0 = s0 + kTcaOffBar;
+  // per stream s: k_free[3] (= S complete) k_full[3] v_full[2] v_free[2] p_ready[2]
+  auto k_full = [&](int s, int b) { return b0 + 8u * (s * 12 + b); };
+  auto k_free = [&](int s, int b) { return b0 + 8u * (s * 12 + 3 + b); };
+  auto v_full = [&](int s, int b) { return b0 + 8u * (s * 12 + 6 + b); };
+  auto v_free = [&](int s, int b) { return b0 + 8u * (s * 12 + 8 + b); };
+  auto p_ready = [&](int s, int b) { return b0 + 8u * (s * 12 + 10 + b); };
+  const int warp = wt >> 5, lane = wt & 31, s = warp >> 2, role = warp & 3;
+  if (wt == 0) {
+    for (int ss = 0; ss < 2; ++ss) {
+      for (int b = 0; b < NKB; ++b) { mbar_init(k_full(ss, b), 32); mbar_init(k_free(ss, b), 1); }
+      for (int b = 0; b < NVB; ++b) { mbar_init(v_full(ss, b), 32); mbar_init(v_free(ss, b), 1); mbar_init(p_ready(ss, b), 1); }
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  // Q: K-major, 128-byte swizzle, k-block kb (64 columns) at kb * 4096, rows 0..31 (rows past the item's vectors zero)
+  for (int i = wt; i < 32 * 16; i += 256) {
+    const int qi = i >> 4, c = i & 15, kb = c >> 3, cc = c & 7;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (qi < it.nqv) {
+      const int r = qi / it.group, gq = qi - r * it.group;
+      v = __ldcg(reinterpret_cast<const uint4 *>(a.q + ((size_t)(it.row0 + r) * a.nq + it.kvh * it.group + gq) * HD + c * 8));
+    }
+    *reinterpret_cast<uint4 *>(smem + kb * 4096 + (qi >> 3) * 1024 + (qi & 7) * 128 + ((cc ^ (qi & 7)) << 4)) = v;
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  tc_fence_before();
+  worker_sync();
+  tc_fence_after();
+  const int n_tiles = (it.key_hi - it.key_lo + TK - 1) / TK;
+  const int n_mine = (n_tiles - s + 1) / 2;                      // tiles s, s + 2, ...
+  const float sc = rsqrtf((float)HD) * 1.4426950408889634f;      // raw scores -> log2 units
+  float m_ref = -INFINITY, l = 0.f;                              // the softmax warps' state (raw score units)
+  bool ok = true;
+  const uint32_t tS = tmem + (uint32_t)(s * 128), tO = tmem + 256u + (uint32_t)(s * 128);
+  if (role == 1 || role == 2) {
+    // ---------------- loader warp of one operand: LAG tiles in flight behind the one being issued
+    const bool isk = role == 1;
+    const int NB = isk ? NKB : NVB, LAG = isk ? 2 : 1;
+    const __nv_bfloat16 *pool = isk ? kpool : vpool;
+    const uint32_t base = isk ? kTcaOffK + s * NKB * kTcaTileBytes : kTcaOffV + s * NVB * kTcaTileBytes;
+    const int *pt = a.page_table + (size_t)it.seq * a.pages_per_seq;
+    for (int t = 0; t < n_mine + LAG; ++t) {
+      if (t >= LAG) {                                            // tile t - LAG has landed: hand it over before anything can block
+        if (isk) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        const int tt = t - LAG;
+        mbar_arrive(isk ? k_full(s, tt % NKB) : v_full(s, tt % NVB));
+      }
+      if (t < n_mine) {
+        const int b = t % NB;
+        if (t >= NB) {
+          const int use = t / NB - 1;                            // completion number of the buffer's previous use
+          if (lane == 0) mbar_wait(isk ? k_free(s, b) : v_free(s, b), (uint32_t)(use & 1), abort_flag);
+          __syncwarp();
+        }
+        if (*abort_flag) break;
+        const int key0 = it.key_lo + (2 * t + s) * TK;
+        // the tile's four 16-key groups lie in one page each (pages hold >= 16 tokens, key ranges start on multiples of 16)
+        int pg = 0;
+        if (lane < 4 && key0 + lane * 16 < it.key_hi) pg = pt[(key0 + lane * 16) >> a.page_shift];
+        const uint32_t tb = base + b * kTcaTileBytes;
+        const int c = lane & 15, blk = c >> 3, cc = c & 7, h = lane >> 4;
+        if (key0 + TK <= it.key_hi) {
+          // a whole tile: per 16-key group one source base (its page) and eight copies per lane, rows 2 i + h; the
+          // swizzled destination differs from row to row by compile-time constants only
+          const uint32_t dst0 = s0 + tb + blk * (TK * 128) + h * 128;
+          const int cch = cc ^ h;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int pgr = __shfl_sync(0xFFFFFFFFu, pg, g);
+            const __nv_bfloat16 *src = pool + ((((size_t)it.kvh * a.n_pages + pgr) << a.page_shift) + ((key0 + 16 * g) & (a.page - 1)) + h) * HD + c * 8;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r7 = (2 * i) & 7;                         // (row & 7) without h; row = 16 g + 2 i + h
+              const uint32_t dst = dst0 + (uint32_t)((2 * g + (i >> 2)) * 1024 + r7 * 128) + (uint32_t)((cch ^ r7) << 4);
+              asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src + (size_t)(2 * i) * HD) : "memory");
+            }
+          }
+        } else {
+#pragma unroll 4
+          for (int i = 0; i < TK / 2; ++i) {
+            const int r = 2 * i + h, key = key0 + r;
+            const int pgr = __shfl_sync(0xFFFFFFFFu, pg, r >> 4);
+            const uint32_t off = tb + blk * (TK * 128) + (r >> 3) * 1024 + (r & 7) * 128 + ((cc ^ (r & 7)) << 4);
+            if (key < it.key_hi)
+              cp_async16(smem + off, pool + ((((size_t)it.kvh * a.n_pages + pgr) << a.page_shift) + (key & (a.page - 1))) * HD + c * 8);
+            else
+              *reinterpret_cast<uint4 *>(smem + off) = make_uint4(0u, 0u, 0u, 0u);    // P is 0 there, V must be finite
+          }
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else if (role == 3) {
+    // ---------------- MMA issue for stream s (one lane)
+    if (lane == 0) {
+      const uint32_t id1 = umma_idesc_bf16(TK), id2 = umma_idesc_bf16(HD) | (1u << 16);     // bit 16: B is MN-major
+      auto issue_s = [&](int t) {                                 // S[t & 1] = Q K_t^T
+        const int b = t % NKB;
+        ok = mbar_wait(k_full(s, b), (uint32_t)((t / NKB) & 1), abort_flag);
+        if (!ok) return;
+#pragma unroll
+        for (int ks = 0; ks < HD / 16; ++ks) {
+          const uint64_t da = umma_desc(s0 + (ks >> 2) * 4096 + (ks & 3) * 32);
+          const uint64_t db = umma_desc(s0 + kTcaOffK + (s * NKB + b) * kTcaTileBytes + (ks >> 2) * (TK * 128) + (ks & 3) * 32);
+          umma_bf16(tS + (uint32_t)((t & 1) * 64), da, db, id1, ks > 0 ? 1u : 0u);
+        }
+        umma_commit(k_free(s, b));                                // S(t) complete = the K buffer is free
+      };
+      if (n_mine > 0) issue_s(0);
+      if (n_mine > 1 && ok) issue_s(1);
+      for (int t = 0; t < n_mine && ok; ++t) {
+        // P(t) is written (so S(t) has been read as well) and V(t) has landed
+        ok = mbar_wait(p_ready(s, t & 1), (uint32_t)((t >> 1) & 1), abort_flag);
+        if (!ok) break;
+        const int vb = t % NVB;
+        ok = mbar_wait(v_full(s, vb), (uint32_t)((t / NVB) & 1), abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t p_off = kTcaOffP + (s * 2 + (t & 1)) * 4096;
+#pragma unroll
+        for (int ks = 0; ks < TK / 16; ++ks) {
+          const uint64_t da = umma_desc(s0 + p_off + ks * 32);
+          const uint64_t db = umma_desc_mn(s0 + kTcaOffV + (s * NVB + vb) * kTcaTileBytes + ks * 2048, TK * 128);
+          umma_bf16(tO, da, db, id2, (t > 0 || ks > 0) ? 1u : 0u);
+        }
+        umma_commit(v_free(s, vb));
+        if (t + 2 < n_mine) issue_s(t + 2);                       // its S buffer (t & 1) was read before P(t) was written
+      }
+    }
+  } else {
+    // ---------------- stream s: softmax (thread = query vector `lane`)
+    auto sync_ok = [&]() { ok = __shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0) != 0; };
+    const int qpos = it.pos0 + lane / it.group;                   // causal limit of this thread's query vector
+    const bool real = lane < it.nqv;
+    for (int t = 0; t < n_mine && ok; ++t) {
+      if (lane == 0) ok = mbar_wait(k_free(s, t % NKB), (uint32_t)((t / NKB) & 1), abort_flag);
+      sync_ok();
+      if (!ok) break;
+      tc_fence_after();
+      float sv[TK];
+#pragma unroll
+      for (int c = 0; c < TK; c += 16) tmem_ld16(tS + (uint32_t)((t & 1) * 64 + c), sv + c);
+      tmem_ld_wait();
+      const int key0 = it.key_lo + (2 * t + s) * TK;
+      if (!real) {
+#pragma unroll
+        for (int c = 0; c < TK; ++c) sv[c] = 0.f;
+      } else if (key0 + TK > it.key_hi || key0 + TK - 1 > qpos) {
+#pragma unroll
+        for (int c = 0; c < TK; ++c)
+          if (key0 + c >= it.key_hi || key0 + c > qpos) sv[c] = -INFINITY;
+      }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < TK; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], sv[c]);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      // the reference maximum moves only when a row's maximum has passed it by more than 8 in log2 units
+      const bool grow = (mx - m_ref) * sc > 8.f;                  // false while both are -inf (no key of the row so far)
+      if (t == 0) m_ref = mx;
+      else if (__any_sync(0xFFFFFFFFu, grow)) {
+        // O of this stream is rescaled: its previous P V must be complete
+        if (lane == 0) ok = mbar_wait(v_free(s, (t - 1) % NVB), (uint32_t)(((t - 1) / NVB) & 1), abort_flag);
+        sync_ok();
+        if (!ok) break;
+        tc_fence_after();
+        const float m_new = grow ? mx : m_ref;
+        const float f = (m_new > -INFINITY && m_ref > -INFINITY) ? ex2_approx((m_ref - m_new) * sc) : (m_new > -INFINITY ? 0.f : 1.f);
+#pragma unroll 1
+        for (int c = 0; c < HD; c += 16) {
+          float o[16];
+          tmem_ld16(tO + (uint32_t)c, o);
+          tmem_ld_wait();
+#pragma unroll
+          for (int e = 0; e < 16; ++e) o[e] *= f;
+          tmem_st16(tO + (uint32_t)c, o);
+        }
+        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        l *= f;
+        m_ref = m_new;
+      }
+      // P buffer t & 1 was read by the P V of tile t - 2
+      if (t >= 2) {
+        if (lane == 0) ok = mbar_wait(v_free(s, (t - 2) % NVB), (uint32_t)(((t - 2) / NVB) & 1), abort_flag);
+        sync_ok();
+        if (!ok) break;
+      }
+      uint8_t *prow = smem + kTcaOffP + (s * 2 + (t & 1)) * 4096 + (lane >> 3) * 1024 + (lane & 7) * 128;
+      const float mneg = m_ref > -INFINITY ? -m_ref * sc : 0.f;   // a row without keys so far: exp2(-inf) = 0 everywhere
+      float l4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+      for (int c8 = 0; c8 < TK / 8; ++c8) {
+        unsigned w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float p0 = ex2_approx(fmaf(sv[c8 * 8 + 2 * e], sc, mneg)), p1 = ex2_approx(fmaf(sv[c8 * 8 + 2 * e + 1], sc, mneg));
+          l4[e] += p0 + p1;
+          const __nv_bfloat162 pb = __floats2bfloat162_rn(p0, p1);
+          w[e] = *reinterpret_cast<const unsigned *>(&pb);
+        }
+        *reinterpret_cast<uint4 *>(prow + ((c8 ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      l += (l4[0] + l4[1]) + (l4[2] + l4[3]);
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(p_ready(s, t & 1));
+    }
+    if (ok && n_mine > 0) {                                       // the stream's last P V
+      const int tl = n_mine - 1;
+      if (lane == 0) ok = mbar_wait(v_free(s, tl % NVB), (uint32_t)((tl / NVB) & 1), abort_flag);
+      sync_ok();
+    }
+    tc_fence_after();
+  }
+  // ---- all MMAs of the item are complete once both softmax warps are here; stream 1 hands (O, m, l) to stream 0
+  //      through shared memory (over the K buffers), stream 0 writes the item's result
+  tc_fence_before();
+  worker_sync();
+  tc_fence_after();
+  if (*abort_flag) return;
+  float *xch = reinterpret_cast<float *>(smem + kTcaOffK);       // [32][HD + 2]
+  if (role == 0 && s == 1) {
+    if (n_mine > 0)
+      for (int c = 0; c < HD; c += 16) {
+        float o[16];
+        tmem_ld16(tO + (uint32_t)c, o);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 16; ++e) xch[lane * (HD + 2) + c + e] = o[e];
+      }
+    xch[lane * (HD + 2) + HD] = n_mine > 0 ? m_ref : -INFINITY;
+    xch[lane * (HD + 2) + HD + 1] = n_mine > 0 ? l : 0.f;
+  }
+  tc_fence_before();
+  worker_sync();
+  if (role == 0 && s == 0) {
+    const float m1 = xch[lane * (HD + 2) + HD], l1 = xch[lane * (HD + 2) + HD + 1];
+    const float mm = fmaxf(m_ref, m1);
+    const float f0 = m_ref > -INFINITY ? ex2_approx((m_ref - mm) * sc) : 0.f, f1 = m1 > -INFINITY ? ex2_approx((m1 - mm) * sc) : 0.f;
+    const float lt = l * f0 + l1 * f1;
+    const bool real = lane < it.nqv;
+    const int r = it.row0 + lane / it.group, hq = it.kvh * it.group + lane % it.group;
+    float *dst = a.attn_partials + (((size_t)r * a.nq + hq) * a.n_splits + it.split) * (HD + 2);
+    __nv_bfloat16 *adst = a.att + ((size_t)r * a.nq + hq) * HD;
+    const float inv = lt > 0.f ? 1.f / lt : 0.f;
+    for (int c = 0; c < HD; c += 16) {
+      float o[16];
+      tmem_ld16(tO + (uint32_t)c, o);
+      tmem_ld_wait();
+      if (real) {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const float o1 = m1 > -INFINITY ? xch[lane * (HD + 2) + c + e] : 0.f;
+          o[e] = (f0 > 0.f ? o[e] * f0 : 0.f) + o1 * f1;
+        }
+        if (a.n_splits == 1) {
+#pragma unroll
+          for (int e = 0; e < 16; e += 2)
+            *reinterpret_cast<__nv_bfloat162 *>(adst + c + e) = __floats2bfloat162_rn(o[e] * inv, o[e + 1] * inv);
+        } else {
+#pragma unroll
+          for (int e = 0; e < 16; e += 2) *reinterpret_cast<float2 *>(dst + c + e) = make_float2(o[e], o[e + 1]);
+        }
+      }
+    }
+    if (real && a.n_splits > 1) { dst[HD] = mm * rsqrtf((float)HD); dst[HD + 1] = lt; }   // m in natural-log units, as the merge phase expects
+    tc_fence_before();
+  }
+}
+
 // Phase A: warp-level online softmax.  A work item is (attention item, KV head, key split); its keys
 // are cut into 16-key sub-tiles (one KV page or part of one: the launcher requires pages of >= 16
 // tokens) that the warps take in turn, each warp with its own running (m, l, O) in registers and its
@@ -382,10 +705,10 @@ __device__ __forceinline__ void ldmatrix_x4_trans(unsigned *r, const void *row_p
 // (rows x group) every warp works on its own sub-tiles; with 17..32 the warps pair up on a sub-tile,
 // one 16-row m-tile each.  At the end the warps' states are merged through shared memory and the
 // split's partial (o, m, l) goes to global memory.
-template <int NPAD, int HD>
+template <int NPAD, int HD, bool TC>
 __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLayerDev &lay, uint8_t *scratch, PageCache *pc, int wt, long long *dbg,
                                                  const int *first_item, const int *qkv_geom, const int *row_pg_sh, const float *rope_cos_sh,
-                                                 const float *rope_sin_sh) {
+                                                 const float *rope_sin_sh, uint8_t *tc_smem, uint32_t tmem, volatile int *abort_flag) {
   constexpr int CPR = HD / 8;                      // 16-byte chunks per row
   // Rows of Q, K, V in shared memory: HD >= 64: unpadded, the 16-byte chunk index XORed with the row's low
   // three bits; HD = 32: padded by 16 bytes.  Either way the fragment loads (eight rows, same chunk) and
@@ -423,6 +746,16 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
     const int key_lo = split * a.keys_per_split, key_hi = min(kv_len, key_lo + a.keys_per_split);
     if (key_lo >= kv_len) continue;                              // uniform over the CTA
     const int nqv = nrows * group, n_mt = (nqv + 15) >> 4;
+    if (TC && HD == 128 && key_hi - key_lo >= kTcaMinKeys && nqv >= kTcaMinVectors) {   // tensor memory path (uniform over the CTA)
+      worker_sync();                                             // the previous item is done with the shared memory
+      if (wt == 0) pc->tag_item = -1;
+      TcaItem ti;
+      ti.row0 = row0; ti.nrows = nrows; ti.seq = seq; ti.pos0 = pos0; ti.kvh = kvh; ti.split = split;
+      ti.key_lo = key_lo; ti.key_hi = key_hi; ti.nqv = nqv; ti.group = group;
+      attn_item_tc(a, kpool, vpool, tc_smem, tmem, ti, wt, abort_flag);
+      if (*abort_flag) return;
+      continue;
+    }
     const int n_sub = (key_hi - key_lo + 15) >> 4;
     const int first = n_mt == 2 ? (warp >> 1) : warp, step = n_mt == 2 ? 4 : 8, mt = n_mt == 2 ? (warp & 1) : 0;
     const int n_mine = first < n_sub ? (n_sub - first + step - 1) / step : 0;       // sub-tiles of this warp
@@ -1093,7 +1426,9 @@ __device__ __forceinline__ void gemm_finish(const FwdArgs &a, WorkerCtx &w, int 
   }
 }
 
-template <int NPAD, int HD>
+// TC: the launch's long attention work items run on tensor memory (a.tc_attn; head size 128 only).  A kernel of its
+// own, so that the other launches keep their code (and its place in the instruction cache) unchanged.
+template <int NPAD, int HD, bool TC>
 __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __grid_constant__ FwdArgs a) {
   using Cfg = PCfg<NPAD>;
   constexpr int STAGES = Cfg::kStages;
@@ -1130,6 +1465,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
   auto accf_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
   auto acce_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
   auto ready_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 4 + b); };
+  const uint32_t attn_done_bar = smem_u32(dbg_cy + 15);         // the last counter slot (laps use 0..14)
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = gridDim.x, c = blockIdx.x;
@@ -1139,13 +1475,15 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
     for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 2); mbar_init(empty_bar(s), 1); }
     for (int b = 0; b < 2; ++b) { mbar_init(accf_bar(b), 1); mbar_init(acce_bar(b), 4); mbar_init(ready_bar(b), 1); }
     *abort_flag = 0;
+    for (int i = 0; i < 15; ++i) dbg_cy[i] = 0;
+    mbar_init(attn_done_bar, 1);
     for (int i = 0; i < 16; ++i) ring_pos_sh[i] = 0xFFFFFFFFu;
-    for (int i = 0; i < 16; ++i) dbg_cy[i] = 0;
     pcache->tag_item = -1;
     pcache->tag_tile = -1;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 2) tmem_alloc(smem_u32(tmem_slot), Cfg::kTmemCols);
+  constexpr uint32_t tmem_cols = TC ? 512u : (uint32_t)Cfg::kTmemCols;      // the attention phase takes all of tensor memory
+  if (warp == 2) tmem_alloc(smem_u32(tmem_slot), tmem_cols);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -1170,6 +1508,9 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
         const Gemm g = make_gemm(a, p);
         SegIter it = seg_begin(g, G, c);
         Seg sg;
+        // the tensor-memory attention phase uses the ring's memory: the O projection's tiles wait until it is over
+        // (one completion per layer, waited for in every layer, so the parity never is ambiguous)
+        if (TC && (p & 3) == 1 && p < 4 * a.n_run && !mbar_wait(attn_done_bar, (uint32_t)((p >> 2) & 1), abort_flag)) { ok = false; break; }
         if (built_down(a, p)) ring_pos_sh[(p >> 2) & 15] = (unsigned)s | (par << 8) | ((unsigned)p << 16);   // where the builders' tiles go
         while (ok && seg_next(g, it, sg)) {
           const Tile ti = tile_of(g, sg.tile);
@@ -1369,7 +1710,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
           break;
         case K_FIN: gemm_finish<NPAD>(a, w, gp); break;
         case K_ATTN_A:
-          attn_tiles_phase<NPAD, HD>(a, layers_sh[l], scratch, pcache, wt, dbg_cy, first_item_sh, qkv_geom_sh, row_pg_sh, rope_cos_sh, rope_sin_sh);
+          attn_tiles_phase<NPAD, HD, TC>(a, layers_sh[l], scratch, pcache, wt, dbg_cy, first_item_sh, qkv_geom_sh, row_pg_sh, rope_cos_sh, rope_sin_sh,
+                                     ring, tmem_base, abort_flag);
+          if (TC) {                                               // the ring's memory is the weight producer's again
+            worker_sync();
+            if (wt == 0) mbar_arrive(attn_done_bar);
+          }
           break;
         case K_ATTN_B: attn_merge_phase<HD>(a, row_pos_sh, wt); break;
         case K_NORM: {
@@ -1389,12 +1735,12 @@ __global__ void __launch_bounds__(kFwdThreads, 1) fwd_persistent_kernel(const __
       if (barrier && alive) alive = grid_barrier(a, epoch, abort_flag, wt, ready >= 0 ? ready_bar(ready & 1) : 0u);
     }
   }
-  if (HSD_PROF(a) && blockIdx.x == 0 && threadIdx.x == 128) for (int i = 0; i < 16; ++i) a.prof[940 + i] = (unsigned long long)dbg_cy[i];
+  if (HSD_PROF(a) && blockIdx.x == 0 && threadIdx.x == 128) for (int i = 0; i < 15; ++i) a.prof[940 + i] = (unsigned long long)dbg_cy[i];
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  if (warp == 2) tmem_dealloc(tmem_base, Cfg::kTmemCols);
+  if (warp == 2) tmem_dealloc(tmem_base, tmem_cols);
   if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, 1);
 }
 
@@ -1420,7 +1766,8 @@ __global__ void __launch_bounds__(256, 2) attn_tiles_kernel(const __grid_constan
   __syncthreads();
   FwdLayerDev lay;
   lay.attn_norm = nullptr; lay.mlp_norm = nullptr; lay.k_pool = k_pool; lay.v_pool = v_pool;
-  attn_tiles_phase<128, HD>(a, lay, scratch, &pcache, (int)threadIdx.x, dbg_cy, first_item_sh, qkv_geom_sh, nullptr, nullptr, nullptr);
+  attn_tiles_phase<128, HD, false>(a, lay, scratch, &pcache, (int)threadIdx.x, dbg_cy, first_item_sh, qkv_geom_sh, nullptr, nullptr, nullptr,
+                            nullptr, 0u, nullptr);
 }
 
 template <int HD>
@@ -1437,28 +1784,28 @@ int launch_attn_tiles_t(const FwdArgs &a, __nv_bfloat16 *k_pool, __nv_bfloat16 *
   return hsd_launch_status();
 }
 
-template <int NPAD, int HD>
+template <int NPAD, int HD, bool TC>
 int launch_t(const FwdArgs &args, int sm_count, cudaStream_t s) {
   using Cfg = PCfg<NPAD>;
   static bool attr_set = false;
   if (!attr_set) {
-    HSD_CUDA_OK(cudaFuncSetAttribute(fwd_persistent_kernel<NPAD, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
+    HSD_CUDA_OK(cudaFuncSetAttribute(fwd_persistent_kernel<NPAD, HD, TC>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::kSmemBytes));
     attr_set = true;
   }
   void *params[1] = {const_cast<FwdArgs *>(&args)};
-  HSD_CUDA_OK(cudaLaunchCooperativeKernel((const void *)fwd_persistent_kernel<NPAD, HD>, dim3(sm_count), dim3(kFwdThreads), params,
+  HSD_CUDA_OK(cudaLaunchCooperativeKernel((const void *)fwd_persistent_kernel<NPAD, HD, TC>, dim3(sm_count), dim3(kFwdThreads), params,
                                           (size_t)Cfg::kSmemBytes, s));
   hsd_count_launches(1);
   return HSD_OK;
 }
 
-template <int HD>
+template <int HD, bool TC>
 int launch_hd(const FwdArgs &args, int npad, int sm_count, cudaStream_t s) {
   switch (npad) {
-    case 16: return launch_t<16, HD>(args, sm_count, s);
-    case 32: return launch_t<32, HD>(args, sm_count, s);
-    case 64: return launch_t<64, HD>(args, sm_count, s);
-    case 128: return launch_t<128, HD>(args, sm_count, s);
+    case 16: return launch_t<16, HD, TC>(args, sm_count, s);
+    case 32: return launch_t<32, HD, TC>(args, sm_count, s);
+    case 64: return launch_t<64, HD, TC>(args, sm_count, s);
+    case 128: return launch_t<128, HD, TC>(args, sm_count, s);
     default: return HSD_E_INVALID_ARG;
   }
 }
@@ -1488,6 +1835,7 @@ int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaS
     long long kb = std::max(args.ff, std::max(args.d, args.nq * args.hd)) / kTcBlockK;
     if (tiles * kb * sm_count >= (1ll << 31)) return HSD_E_UNSUPPORTED;
   }
+  if (args.tc_attn && (args.hd != 128 || args.fuse_qkv)) return HSD_E_INVALID_ARG;
   FwdArgs a = args;
   {  // pieces per gate / up tile (the device's split_geom, for a grid of sm_count CTAs)
     const int n_tiles = (a.ff + kTcBoxRows - 1) / kTcBoxRows, KB = a.d / kTcBlockK;
@@ -1505,9 +1853,9 @@ int launch_forward_persistent(const FwdArgs &args, int npad, int sm_count, cudaS
     a.early_norm = (a.early_norm && a.R <= idle && a.L <= idle) ? 1 : 0;
   }
   switch (a.hd) {
-    case 128: return launch_hd<128>(a, npad, sm_count, s);
-    case 64: return launch_hd<64>(a, npad, sm_count, s);
-    case 32: return launch_hd<32>(a, npad, sm_count, s);
+    case 128: return a.tc_attn ? launch_hd<128, true>(a, npad, sm_count, s) : launch_hd<128, false>(a, npad, sm_count, s);
+    case 64: return launch_hd<64, false>(a, npad, sm_count, s);
+    case 32: return launch_hd<32, false>(a, npad, sm_count, s);
     default: return HSD_E_UNSUPPORTED;
   }
 }

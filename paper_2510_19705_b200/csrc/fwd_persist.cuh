@@ -31,6 +31,7 @@ struct FwdArgs {
   int early_norm;                  // 1: the RMSNorm after a residual projection runs on CTAs that have no part in that projection;
                                    //    they start as soon as its pieces are complete (a counter), one grid barrier less per norm
                                    //    (filled in by the launcher)
+  int tc_attn;                     // 1: work items with long key ranges run on tcgen05 / tensor memory (head size 128; needs fuse_qkv = 0)
   float *pieces2;                  // split pieces of the down projection while `pieces` still holds gate / up (fuse_gu)
   const int *tokens, *page_table, *row_seq, *row_pos, *lrow_src;
   const int4 *attn_items;          // (first packed row, rows, sequence, position of first row)

@@ -230,7 +230,8 @@ def test_bf16_batch_decisions_and_logits(lib, tmp_path, B):
         _assert_bf16_logits_close(rec["logits"], om.last_logits64, ref_p, ("mini3 batch", b))
 
 
-def test_long_context_four_levels_paged_batch(lib, tmp_path):
+@pytest.mark.parametrize("tensor_attention", [True, "prefer"])
+def test_long_context_four_levels_paged_batch(lib, tmp_path, tensor_attention):
     """The long-context configuration's structure at a size the oracle can follow: 4 levels with draft lengths
     (2, 2, 3), two sequences, 16-token pages, 2100-token prompts (the long-context attention path: every key split spans more than one
     key tile and several pages).  Every decision follows the oracle on the logged logits; each sequence's first
@@ -241,6 +242,7 @@ def test_long_context_four_levels_paged_batch(lib, tmp_path):
     w = {k: (v.cuda() if k != "layers" else [{n: t.cuda() for n, t in l.items()} for l in v]) for k, v in w_cpu.items()}
     prompts = inputs.make_prompts(cfg["vocab"], B, wl["prompt"], wl["prompt_seed"])
     eng = lib.Hsd(cfg, w, wl["exits"], T, max_batch=B, max_seq=wl["prompt"] + n_new + 32, page_size=wl["page"])
+    eng.set_tensor_attention(tensor_attention)         # "prefer": the prompt chunks' attention runs on the tensor-memory path
     path = str(tmp_path / "trace.bin")
     eng.set_trace(path, logit_calls=10 ** 6)
     toks, stats, _ = eng.generate(prompts.cuda(), n_new, seed)
@@ -265,15 +267,46 @@ def test_long_context_four_levels_paged_batch(lib, tmp_path):
             _assert_bf16_logits_close(rec["logits"], ref, ref_p, ("mini4long", b, lvl))
 
 
-def _run_traced(lib, cfg, w, exits, T, prompts, n_new, seed, page, tmp_path, tag="trace"):
+def _run_traced(lib, cfg, w, exits, T, prompts, n_new, seed, page, tmp_path, tag="trace", setup=None):
     B, P = prompts.shape
     eng = lib.Hsd(cfg, w, exits, T, max_batch=B, max_seq=P + n_new + sum(T) + 16, page_size=page)
+    if setup:
+        setup(eng)
     path = str(tmp_path / (tag + ".bin"))
     eng.set_trace(path, logit_calls=10 ** 6)
     toks, stats, _ = eng.generate(prompts.cuda(), n_new, seed)
     eng.set_trace(None)
     eng.close()
     return toks.cpu(), stats, lib.read_trace(path)
+
+
+def test_tensor_memory_attention_agrees_with_the_warp_level_path(lib, tmp_path):
+    """Long key ranges with many query vectors (the prompt chunks of the long-context model: 32 vectors per item, up to
+    2100 keys) run on the tensor-memory attention path; switched off they run on the warp-level path.  The first
+    verification of every level, which attends over everything the prompt pass wrote, must agree between the two
+    within bf16 rounding of the logits, and must differ somewhere (else the path under test did not run)."""
+    wl = inputs.WORKLOADS["mini4long"]
+    cfg, T, B = wl["model"], wl["T"], wl["batch"]
+    w = inputs.make_weights(cfg, wl["weight_seed"], device="cuda")
+    prompts = inputs.make_prompts(cfg["vocab"], B, wl["prompt"], wl["prompt_seed"])
+    runs = []
+    for on in ("prefer", False):
+        _, _, recs = _run_traced(lib, cfg, w, wl["exits"], T, prompts, 4, 6, wl["page"], tmp_path, tag="tca%d" % bool(on),
+                                 setup=lambda eng: eng.set_tensor_attention(on))
+        runs.append(recs)
+    differs = False
+    for b in range(B):
+        for lvl in range(len(wl["exits"])):
+            ra = next(r for r in runs[0] if r["seq"] == b and r["level"] == lvl)
+            rb = next(r for r in runs[1] if r["seq"] == b and r["level"] == lvl)
+            if lvl and not np.array_equal(ra["tokens"], rb["tokens"]):
+                continue                                  # another draft went up: other rows, nothing to compare
+            la, lb = np.asarray(ra["logits"], dtype=np.float64), np.asarray(rb["logits"], dtype=np.float64)
+            n = min(len(la), len(lb))
+            d = np.abs(la[:n] - lb[:n])
+            differs = differs or bool(d.max() > 0)
+            assert d.max() <= 6e-2 and np.sqrt((d ** 2).mean()) <= 6e-3, (b, lvl, d.max(), np.sqrt((d ** 2).mean()))
+    assert differs
 
 
 @pytest.mark.parametrize("name,T,P,n_new", [("1b3", (4, 2), 96, 24), ("8b3", (1, 1), 96, 12)])
