@@ -185,11 +185,11 @@ int hsd_set_phase_folding(hsd_ctx *ctx, int fold_qkv, int fold_gate_up, int earl
 
 /* Which kernel path attention work items with long key ranges take (the paper gives no kernel design; its
  * verification pass of Algorithm 2 attends over the whole context).  enabled != 0 (the default): on models with
- * head size 128, an item with 13 or more query vectors whose key range has 1024 keys or more runs on the
+ * head size 128, an item with 8 or more query vectors whose key range has 2048 keys or more runs on the
  * fifth-generation tensor cores with its scores and outputs in tensor memory; enabled = 0: every item runs on the warp-level path.  Both paths compute the
  * same attention (softmax weights rounded to bf16 before the P V product on the tensor-memory path, to bf16 hi + lo
  * on the other), so results agree to rounding, not bit for bit.  enabled = 2 additionally keeps the key splits of
- * long contexts at 1024 keys or more, so that small test models reach that path too.  A test hook and a tuning knob.
+ * long contexts at 2048 keys or more, so that small test models reach that path too.  A test hook and a tuning knob.
  * Errors: INVALID_ARG. */
 int hsd_set_tensor_attention(hsd_ctx *ctx, int enabled);
 

@@ -21,8 +21,8 @@ constexpr int kRingSlots = 48;
 constexpr int kTimerPairs = 64;
 constexpr int kAttnBlocksTarget = 512;
 constexpr int kMaxSplits = 64;
-constexpr int kTcAttnMinKeys = 1024;           // = the kernel's thresholds for the tensor-memory attention path:
-constexpr int kTcAttnMinVectors = 13;          //   keys of a work item, query vectors of an attention item
+constexpr int kTcAttnMinKeys = 2048;           // = the kernel's thresholds for the tensor-memory attention path:
+constexpr int kTcAttnMinVectors = 8;          //   keys of a work item, query vectors of an attention item
 constexpr int kPrefillRows = 128;              // rows of one prompt chunk: the largest pass the one-launch forward takes
 constexpr uint32_t kTraceMagic = 0x48534454u;
 
@@ -423,7 +423,13 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
   const int blocks_target = M.use_persist ? c->sm_count : kAttnBlocksTarget;
   const int max_splits = M.use_persist ? 20 : kMaxSplits;      // the persistent merge phase takes <= 20 splits
   int n_splits = std::max(1, std::min(max_splits, blocks_target / std::max(1, n_attn * md.nkv)));
-  const bool tc_capable = M.use_persist && md.hd == 128 && !c->no_tc_attn && R <= 128 && n_logit <= 128;
+  // the tensor-memory attention path: head size 128, a pass of the one-launch forward in which at least half of the
+  // attention items have enough query vectors for it to pay (the pass then has its QKV finish phase and holds the
+  // O projection's weights back until the attention phase is over)
+  int n_vec_items = 0;
+  for (int i = 0; i < n_attn; ++i)
+    if (attn[i].y * (md.nq / md.nkv) >= kTcAttnMinVectors) ++n_vec_items;
+  const bool tc_capable = M.use_persist && md.hd == 128 && !c->no_tc_attn && R <= 128 && n_logit <= 128 && 2 * n_vec_items >= n_attn;
   if (M.use_persist && max_kv >= 2048) {
     // Long contexts: the key loop dominates and the items differ in cost, so the split count is chosen by a
     // small model of the tiles phase: a work unit (item, KV head, split) costs a fixed part plus its keys x
@@ -520,9 +526,7 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
     // the norms after the residual projections start on otherwise idle CTAs as soon as the pieces are there
     a.early_norm = c->no_early_norm ? 0 : 1;
     // long key ranges: attention work items on tcgen05 / tensor memory (they take their q / k / v from the finish phase)
-    int max_vectors = 0;
-    for (int i = 0; i < n_attn; ++i) max_vectors = std::max(max_vectors, attn[i].y * qgroup);
-    a.tc_attn = (tc_capable && keys_per_split >= kTcAttnMinKeys && max_vectors >= kTcAttnMinVectors) ? 1 : 0;
+    a.tc_attn = (tc_capable && keys_per_split >= kTcAttnMinKeys) ? 1 : 0;
     if (a.tc_attn) a.fuse_qkv = 0;
     a.pieces2 = (float *)(c->ws + ML.tc_pieces2);
     for (int b = 0; b < 4; ++b) a.amap[b] = box_rows <= 16 ? M.amaps_rows[b][box_rows - 1] : M.amaps[b][pi];

@@ -390,8 +390,8 @@ constexpr int kTcaTile = 64, kTcaKBufs = 3, kTcaVBufs = 2;
 constexpr int kTcaTileBytes = 2 * kTcaTile * 128;                 // two 64-column blocks of [64 keys][128 B]
 constexpr int kTcaOffK = 8192, kTcaOffV = kTcaOffK + 2 * kTcaKBufs * kTcaTileBytes, kTcaOffP = kTcaOffV + 2 * kTcaVBufs * kTcaTileBytes;
 constexpr int kTcaOffBar = kTcaOffP + 4 * 4096 + 12288, kTcaBytes = kTcaOffBar + 256;
-constexpr int kTcaMinKeys = 1024;                                 // shorter key ranges stay on the mma.sync path
-constexpr int kTcaMinVectors = 13;                                // ... and items with fewer query vectors (its cost grows with them, this path's does not)
+constexpr int kTcaMinKeys = 2048;                                 // shorter key ranges stay on the mma.sync path
+constexpr int kTcaMinVectors = 8;                                // ... and items with fewer query vectors (its cost grows with them, this path's does not)
 static_assert(kTcaBytes <= 4 * (kWBytes + 128 * kTcBlockK * 2) + kScratchBytes - 2 * 12 * 64 * 4, "tcgen05 attention buffers exceed the ring + scratch");
 
 __device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lbo_bytes) {   // MN-major, 128-byte swizzle
