@@ -448,7 +448,7 @@ int forward(hsd_ctx *c, int level, const std::vector<SeqWork> &work) {
       for (int i = 0; i < n_attn; ++i) {
         const int kv = attn[i].w + attn[i].y, mt = (attn[i].y * qgroup + 15) / 16, keys = std::min(kps, kv);
         // key ranges of kTcAttnMinKeys and more run on tensor memory: 64-key tiles, whatever the number of query vectors
-        const bool tc_item = tc_capable && keys >= kTcAttnMinKeys && attn[i].y * qgroup >= kTcAttnMinVectors;
+        const bool tc_item = tc_capable && keys >= kTcAttnMinKeys;      // in such a pass every long key range takes that path
         const double unit = tc_item ? 6.0 + ((keys + 63) / 64) * 0.8 : 5.0 + mt * ((keys + 127) / 128) * 1.9;
         // all s_try x nkv slots of the item are dealt out; splits past its last key return at once
         const long long used = (long long)std::min(s_try, (kv + kps - 1) / kps) * md.nkv, slots = (long long)s_try * md.nkv;

@@ -391,7 +391,6 @@ constexpr int kTcaTileBytes = 2 * kTcaTile * 128;                 // two 64-colu
 constexpr int kTcaOffK = 8192, kTcaOffV = kTcaOffK + 2 * kTcaKBufs * kTcaTileBytes, kTcaOffP = kTcaOffV + 2 * kTcaVBufs * kTcaTileBytes;
 constexpr int kTcaOffBar = kTcaOffP + 4 * 4096 + 12288, kTcaBytes = kTcaOffBar + 256;
 constexpr int kTcaMinKeys = 2048;                                 // shorter key ranges stay on the mma.sync path
-constexpr int kTcaMinVectors = 8;                                // ... and items with fewer query vectors (its cost grows with them, this path's does not)
 static_assert(kTcaBytes <= 4 * (kWBytes + 128 * kTcBlockK * 2) + kScratchBytes - 2 * 12 * 64 * 4, "tcgen05 attention buffers exceed the ring + scratch");
 
 __device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lbo_bytes) {   // MN-major, 128-byte swizzle
@@ -746,7 +745,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
     const int key_lo = split * a.keys_per_split, key_hi = min(kv_len, key_lo + a.keys_per_split);
     if (key_lo >= kv_len) continue;                              // uniform over the CTA
     const int nqv = nrows * group, n_mt = (nqv + 15) >> 4;
-    if (TC && HD == 128 && key_hi - key_lo >= kTcaMinKeys && nqv >= kTcaMinVectors) {   // tensor memory path (uniform over the CTA)
+    if (TC && HD == 128 && key_hi - key_lo >= kTcaMinKeys) {     // tensor memory path (uniform over the CTA)
       worker_sync();                                             // the previous item is done with the shared memory
       if (wt == 0) pc->tag_item = -1;
       TcaItem ti;
@@ -1077,35 +1076,38 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
   }
 }
 
-// Phase B: merge the split partials of one (row, head) per 128 threads; a single batch of loads.
+// Phase B: merge the split partials of one (row, head) per HD / 2 threads (two output dimensions each); a single
+// batch of loads.
 template <int HD>
 __device__ __forceinline__ void attn_merge_phase(const FwdArgs &a, const int *row_pos_sh, int wt) {
-  const int half = wt >> 7, dd = wt & 127;
+  constexpr int TPI = HD / 2, PER = 256 / TPI;                    // threads per item, items per CTA turn
+  const int g = wt / TPI, dd = (wt % TPI) * 2;
   const int n_items = a.R * a.nq;
-  for (int it = blockIdx.x * 2 + half; it < n_items; it += 2 * gridDim.x) {
-    if (dd >= HD) continue;
+  for (int it = blockIdx.x * PER + g; it < n_items; it += PER * gridDim.x) {
     const int r = it / a.nq;
     const int used = min(a.n_splits, row_pos_sh[r] / a.keys_per_split + 1);   // splits holding keys <= own position
     const float *src = a.attn_partials + (size_t)it * a.n_splits * (HD + 2);
-    float ms[kAttnMaxSplits], ls[kAttnMaxSplits], os[kAttnMaxSplits];
+    float ms[kAttnMaxSplits], ls[kAttnMaxSplits];
+    float2 os[kAttnMaxSplits];
 #pragma unroll
     for (int s = 0; s < kAttnMaxSplits; ++s) {
       const bool on = s < used;
-      ms[s] = on ? __ldcg(src + s * (HD + 2) + HD) : -INFINITY;
-      ls[s] = on ? __ldcg(src + s * (HD + 2) + HD + 1) : 0.f;
-      os[s] = on ? __ldcg(src + s * (HD + 2) + dd) : 0.f;
+      const float2 ml = on ? __ldcg(reinterpret_cast<const float2 *>(src + s * (HD + 2) + HD)) : make_float2(-INFINITY, 0.f);
+      ms[s] = ml.x; ls[s] = ml.y;
+      os[s] = on ? __ldcg(reinterpret_cast<const float2 *>(src + s * (HD + 2) + dd)) : make_float2(0.f, 0.f);
     }
     float m = -INFINITY;
 #pragma unroll
     for (int s = 0; s < kAttnMaxSplits; ++s) m = fmaxf(m, ms[s]);
-    float l = 0.f, o = 0.f;
+    float l = 0.f, ox = 0.f, oy = 0.f;
 #pragma unroll
     for (int s = 0; s < kAttnMaxSplits; ++s) {
       const float w = (ms[s] > -INFINITY) ? __expf(ms[s] - m) : 0.f;
       l += w * ls[s];
-      o += w * os[s];
+      ox += w * os[s].x;
+      oy += w * os[s].y;
     }
-    a.att[(size_t)it * HD + dd] = __float2bfloat16_rn(o / l);
+    *reinterpret_cast<__nv_bfloat162 *>(a.att + (size_t)it * HD + dd) = __floats2bfloat162_rn(ox / l, oy / l);
   }
 }
 
