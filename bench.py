@@ -203,6 +203,8 @@ def run_ours(args):
     else:
         T, calib = list(wl["T"]), None
     eng = binding.Hsd(cfg, weights, wl["exits"], T, max_batch=B, max_seq=P + n_new + sum(T) + 16, page_size=wl["page"])
+    if args.coin > 0:                                    # A/B runs of two builds: the same accept decisions whatever the logits
+        eng.set_iid_acceptance([args.coin] * (len(wl["exits"]) - 1))
     if args.exit_heads:                                  # Section 5.1's other setting: one (random-init) head per drafting level
         eng.set_exit_heads(inputs.make_exit_heads(cfg, len(wl["exits"]), seed=4242, device="cuda"))
 
@@ -474,6 +476,9 @@ def main():
     ap.add_argument("--batch", type=int, default=1, help="sequences per GPU (the metric is quoted at 1)")
     ap.add_argument("--prompt-len", type=int, default=0, help="override the workload's prompt length (development runs)")
     ap.add_argument("--T", default="", help="fix T (comma separated) instead of calibrating / using the workload's")
+    ap.add_argument("--coin", type=float, default=0.0,
+                    help="accept every draft with this fixed probability instead of p/q (development: two builds then run "
+                         "the same passes; not the benchmark's metric)")
     ap.add_argument("--ablation", action="store_true",
                     help="add the four-way latency table (real / IID-coin acceptance x measured / artificial cost)")
     ap.add_argument("--exit-heads", action="store_true",

@@ -390,7 +390,8 @@ constexpr int kTcaTile = 64, kTcaKBufs = 3, kTcaVBufs = 2;
 constexpr int kTcaTileBytes = 2 * kTcaTile * 128;                 // two 64-column blocks of [64 keys][128 B]
 constexpr int kTcaOffK = 8192, kTcaOffV = kTcaOffK + 2 * kTcaKBufs * kTcaTileBytes, kTcaOffP = kTcaOffV + 2 * kTcaVBufs * kTcaTileBytes;
 constexpr int kTcaOffBar = kTcaOffP + 4 * 4096 + 12288, kTcaBytes = kTcaOffBar + 256;
-constexpr int kTcaMinKeys = 2048;                                 // shorter key ranges stay on the mma.sync path
+constexpr int kTcaMinKeys = 1920;                                 // shorter key ranges stay on the mma.sync path (the host plans splits of
+                                                                  // 2048 keys and more; the last split of a range may fall a little short)
 static_assert(kTcaBytes <= 4 * (kWBytes + 128 * kTcBlockK * 2) + kScratchBytes - 2 * 12 * 64 * 4, "tcgen05 attention buffers exceed the ring + scratch");
 
 __device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t lbo_bytes) {   // MN-major, 128-byte swizzle
@@ -418,7 +419,7 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const float *o) {
 struct TcaItem { int row0, nrows, seq, pos0, kvh, split, key_lo, key_hi, nqv, group; };
 
 __device__ __noinline__ void attn_item_tc(const FwdArgs &a, const __nv_bfloat16 *kpool, const __nv_bfloat16 *vpool, uint8_t *smem,
-                                          uint32_t tmem, const TcaItem it, int wt, volatile int *abort_flag) {
+                                          uint32_t tmem, const TcaItem it, int wt, volatile int *abort_flag, long long *dbg) {
   constexpr int HD = 128, TK = kTcaTile, NKB = kTcaKBufs, NVB = kTcaVBufs;
   const uint32_t s0 = smem_u32(smem), b0 = s0 + kTcaOffBar;
   // per stream s: k_free[3] (= S complete) k_full[3] v_full[2] v_free[2] p_ready[2]
@@ -428,6 +429,15 @@ __device__ __noinline__ void attn_item_tc(const FwdArgs &a, const __nv_bfloat16 
   auto v_free = [&](int s, int b) { return b0 + 8u * (s * 12 + 8 + b); };
   auto p_ready = [&](int s, int b) { return b0 + 8u * (s * 12 + 10 + b); };
   const int warp = wt >> 5, lane = wt & 31, s = warp >> 2, role = warp & 3;
+#ifdef HSD_PROFILE
+  // profiling build: CTA 0's first softmax warp laps its set-up [5], waits for S [6], softmax up to P ready [7] and the
+  // item's end [8]; [9] counts the items
+  long long cyc = clock64();
+  auto lap = [&](int k) { if (a.prof && wt == 0 && blockIdx.x == 0) { const long long n_ = clock64(); dbg[k] += n_ - cyc; cyc = n_; } };
+  if (a.prof && wt == 0 && blockIdx.x == 0) dbg[9] += 1;
+#else
+  auto lap = [](int) {};
+#endif
   if (wt == 0) {
     for (int ss = 0; ss < 2; ++ss) {
       for (int b = 0; b < NKB; ++b) { mbar_init(k_full(ss, b), 32); mbar_init(k_free(ss, b), 1); }
@@ -449,6 +459,7 @@ __device__ __noinline__ void attn_item_tc(const FwdArgs &a, const __nv_bfloat16 
   tc_fence_before();
   worker_sync();
   tc_fence_after();
+  lap(5);
   const int n_tiles = (it.key_hi - it.key_lo + TK - 1) / TK;
   const int n_mine = (n_tiles - s + 1) / 2;                      // tiles s, s + 2, ...
   const float sc = rsqrtf((float)HD) * 1.4426950408889634f;      // raw scores -> log2 units
@@ -562,6 +573,7 @@ __device__ __noinline__ void attn_item_tc(const FwdArgs &a, const __nv_bfloat16 
       if (lane == 0) ok = mbar_wait(k_free(s, t % NKB), (uint32_t)((t / NKB) & 1), abort_flag);
       sync_ok();
       if (!ok) break;
+      lap(6);
       tc_fence_after();
       float sv[TK];
 #pragma unroll
@@ -630,6 +642,7 @@ __device__ __noinline__ void attn_item_tc(const FwdArgs &a, const __nv_bfloat16 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(p_ready(s, t & 1));
+      lap(7);
     }
     if (ok && n_mine > 0) {                                       // the stream's last P V
       const int tl = n_mine - 1;
@@ -692,6 +705,7 @@ __device__ __noinline__ void attn_item_tc(const FwdArgs &a, const __nv_bfloat16 
     if (real && a.n_splits > 1) { dst[HD] = mm * rsqrtf((float)HD); dst[HD + 1] = lt; }   // m in natural-log units, as the merge phase expects
     tc_fence_before();
   }
+  lap(8);
 }
 
 // Phase A: warp-level online softmax.  A work item is (attention item, KV head, key split); its keys
@@ -751,7 +765,7 @@ __device__ __forceinline__ void attn_tiles_phase(const FwdArgs &a, const FwdLaye
       TcaItem ti;
       ti.row0 = row0; ti.nrows = nrows; ti.seq = seq; ti.pos0 = pos0; ti.kvh = kvh; ti.split = split;
       ti.key_lo = key_lo; ti.key_hi = key_hi; ti.nqv = nqv; ti.group = group;
-      attn_item_tc(a, kpool, vpool, tc_smem, tmem, ti, wt, abort_flag);
+      attn_item_tc(a, kpool, vpool, tc_smem, tmem, ti, wt, abort_flag, dbg);
       if (*abort_flag) return;
       continue;
     }
