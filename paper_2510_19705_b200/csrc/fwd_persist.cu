@@ -657,6 +657,9 @@ __device__ __noinline__ void attn_item_tc(const FwdArgs &a, const __nv_bfloat16 
   worker_sync();
   tc_fence_after();
   if (*abort_flag) return;
+  if (wt == 0)                                                    // nobody waits on the item's barriers any more: their memory
+    for (int i = 0; i < 24; ++i)                                  // goes back to the weight ring / the next item
+      asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(b0 + 8u * i) : "memory");
   float *xch = reinterpret_cast<float *>(smem + kTcaOffK);       // [32][HD + 2]
   if (role == 0 && s == 1) {
     if (n_mine > 0)
