@@ -294,6 +294,12 @@ def test_tensor_memory_attention_agrees_with_the_warp_level_path(lib, tmp_path):
         _, _, recs = _run_traced(lib, cfg, w, wl["exits"], T, prompts, 4, 6, wl["page"], tmp_path, tag="tca%d" % bool(on),
                                  setup=lambda eng: eng.set_tensor_attention(on))
         runs.append(recs)
+    # the page size changes where the tiles come from, not what is computed: 64-token pages give the same records
+    toks64, _, recs64 = _run_traced(lib, cfg, w, wl["exits"], T, prompts, 4, 6, 64, tmp_path, tag="tca64",
+                                    setup=lambda eng: eng.set_tensor_attention("prefer"))
+    assert len(recs64) == len(runs[0])
+    for ra, rb in zip(runs[0], recs64):
+        assert np.array_equal(ra["tokens"], rb["tokens"]) and np.array_equal(ra["logits"], rb["logits"])
     differs = False
     for b in range(B):
         for lvl in range(len(wl["exits"])):
