@@ -494,16 +494,19 @@ __global__ void __launch_bounds__(kFusedThreads, 1) verify_fused_kernel(const __
     group_sync();                                           // every thread holds its part of the row: the slot is free
     if (*abort_flag) break;                                 // uniform over the group: raised before the barrier
     if (gwarp == 0) fetch_ordinal(k + kFusedSlots);
-    float m = -INFINITY;
+    // the row maximum on the packed pairs (the maximum of bf16 values is one of them: exact)
+    __nv_bfloat162 mx2 = __floats2bfloat162_rn(-INFINITY, -INFINITY);
 #pragma unroll
     for (int j = 0; j < kFusedVecPerThread; ++j) {
       if (gtid + 512 * j < nvec) {
-        float f[8];
-        StatVec<__nv_bfloat16>::unpack(regs[j], f);
-#pragma unroll
-        for (int e = 0; e < 8; ++e) m = fmaxf(m, f[e]);
+        const uint4 r4 = regs[j];
+        mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162 *>(&r4.x));
+        mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162 *>(&r4.y));
+        mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162 *>(&r4.z));
+        mx2 = __hmax2(mx2, *reinterpret_cast<const __nv_bfloat162 *>(&r4.w));
       }
     }
+    float m = fmaxf(__low2float(mx2), __high2float(mx2));
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     if (lane == 0) shf[grp][gwarp] = m;
     group_sync();
